@@ -1,0 +1,166 @@
+/*
+ * ada.h -- C ABI of the B200 (sm_100a) Gram-threshold representative-token
+ * selection library (the selection hot path of Cascade ADA).
+ *
+ * Notation follows the paper: X in R^{T x d} is one layer's activation matrix
+ * (row t = token t), Xhat = D^-1 X its row-normalised form (Section 2.1),
+ * G = Xhat Xhat^T the cosine Gram, tau in (0,1) the Gram threshold,
+ * thr = 1 - tau^2, R^(l) the representative index set of layer l.
+ *
+ * Conventions shared by every call
+ *   - All data pointers are DEVICE pointers unless the function name ends in
+ *     `_host`.  `stream` is a cudaStream_t passed as void* (NULL = default
+ *     stream).  Device-pointer calls only enqueue work: they never synchronise
+ *     and never read a count back to the host, so the outputs of one layer can
+ *     feed the next call directly.
+ *   - X is row-major, B independent sequences stacked: element (b,t,k) lives at
+ *     X[(b*T + t)*ldx + k].  ldx >= d, and X, ldx*es and d*es must be multiples
+ *     of 16 bytes (es = 4 for ADA_F32, 2 for ADA_BF16); otherwise
+ *     ADA_ERR_UNSUPPORTED.  X is never written.
+ *   - Index lists are int32, strictly ascending token indices in [0,T), with a
+ *     capacity of T entries per sequence: sequence b uses list + b*T and
+ *     count[b].  Counts are int32 on the device.
+ *   - The caller owns every buffer it passes.  The library owns only the
+ *     context (workspace: inverse norms, gathered representative rows, gamma
+ *     scratch, role map, status word).  One context serves one stream at a
+ *     time: calls on the same context that overlap on the GPU race on the
+ *     workspace.
+ *   - Host-checkable faults (bad sizes, NULL required pointers, tau outside
+ *     (0,1), misalignment, sizes above the context's maxima) return an error
+ *     at once and enqueue nothing.  Device-detected faults (an inherited list
+ *     that is not strictly ascending or leaves [0,T), a count outside [0,T],
+ *     NaN/Inf in X, an expired bounded wait) set bits in the context's device
+ *     status word, leave the call's outputs in bounds but meaningless, and are
+ *     reported by ada_device_status.
+ *   - Arithmetic: squared norms and Gram accumulation in fp32.  ADA_BF16
+ *     multiplies the stored bf16 values on the tensor cores (products exact in
+ *     fp32) and applies 1/(|x_s| |x_t|) in the epilogue; a normalised bf16 copy
+ *     of X is never fed to the Gram.  gamma is compared in fp32 with
+ *     (float)(1 - tau*tau), strict "<".
+ */
+#ifndef ADA_H_
+#define ADA_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    ADA_OK = 0,
+    ADA_ERR_INVALID_ARG = 1,   /* NULL pointer, size < 1, tau outside (0,1), ldx < d        */
+    ADA_ERR_UNSUPPORTED = 2,   /* alignment rule broken, dtype differs from the context's   */
+    ADA_ERR_WORKSPACE = 3,     /* B, T or d above the maxima given to ada_create            */
+    ADA_ERR_CUDA = 4,          /* a CUDA runtime / driver call failed                       */
+    ADA_ERR_BAD_INDEX_SET = 5, /* device: inherited list not ascending / out of range       */
+    ADA_ERR_NONFINITE = 6,     /* device: NaN or Inf in X                                   */
+    ADA_ERR_TIMEOUT = 7        /* device: a bounded wait inside a kernel expired            */
+} ada_status;
+
+typedef enum { ADA_F32 = 0, ADA_BF16 = 1 } ada_dtype;
+
+/* flags of ada_cascade_step */
+#define ADA_CROSS_CAUSAL 1u /* restrict Algorithm 1 line 8 to valid representatives s < t */
+
+/* Which Gram kernel family a context uses.  AUTO: tensor cores (tcgen05) for
+ * ADA_BF16, fp32 FFMA for ADA_F32.  FFMA may be forced for bf16 input (a slow
+ * cross-check of the tensor-core path); TCGEN05 cannot be forced for fp32. */
+typedef enum { ADA_ENGINE_AUTO = 0, ADA_ENGINE_FFMA = 1, ADA_ENGINE_TCGEN05 = 2 } ada_engine;
+
+typedef struct ada_ctx ada_ctx; /* opaque */
+
+/* Create a context on `device` able to serve up to maxB sequences of maxT
+ * tokens of width maxd in storage type dt.  Allocates the workspace
+ * (cudaMalloc; about maxB*maxT*(maxd*es + 32) bytes).  *out is NULL on error. */
+ada_status ada_create(ada_ctx** out, int device, int64_t maxB, int64_t maxT, int64_t maxd,
+                      ada_dtype dt);
+ada_status ada_destroy(ada_ctx* ctx);
+ada_status ada_set_engine(ada_ctx* ctx, ada_engine e);
+
+/*
+ * Row normalisation and representative gather (Section 2.1; Algorithm 1
+ * lines 1-2).  Each output may be NULL:
+ *   inv_norm[B*T]  fp32, 1/||x_t||_2 (0 for a zero row; such rows are counted)
+ *   Xhat           same type/shape as X with row stride d: Xhat = D^-1 X
+ *   Xrep           if rep_idx/rep_cnt are given: Xrep[(b*T+i)*d + k] =
+ *                  X[b, rep_idx[b*T+i], k] for i < rep_cnt[b] (raw rows,
+ *                  same type as X, row stride d)
+ * One pass over X; rows are read once with 128-bit loads.
+ */
+ada_status ada_normalize(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d,
+                         int64_t ldx, ada_dtype dt, void* Xhat, float* inv_norm,
+                         const int32_t* rep_idx, const int32_t* rep_cnt, void* Xrep,
+                         void* stream);
+
+/*
+ * Full selection (Definition 1; used at layer 0, Section 4.1):
+ *   gamma_t = max_{s<t} |G_st|  (gamma_0 = 0),   R = { t : gamma_t < 1 - tau^2 }.
+ * The maximum runs over ALL earlier tokens.  The T x T Gram is never stored:
+ * mask, |.|, row maximum and compare are fused into the Gram kernel's epilogue.
+ * Outputs: rep_idx (B*T capacity) ascending, rep_cnt[B]; gamma[B*T] optional.
+ */
+ada_status ada_select_full(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d,
+                           int64_t ldx, ada_dtype dt, double tau, int32_t* rep_idx,
+                           int32_t* rep_cnt, float* gamma, void* stream);
+
+/*
+ * One cascade step (Algorithm 1, lines 1-11) on X = X^(l+1):
+ *   lines 3-5  gamma_rep_i = max_{j<i} |G(rho_i, rho_j)| over ALL inherited
+ *              representatives earlier in token order; valid iff < thr
+ *   lines 6-9  for every t outside the inherited set,
+ *              gamma_cross_t = max_{s in R_valid} |G_ts|; new iff < thr
+ *              (ADA_CROSS_CAUSAL: only s < t)
+ *   lines 10-11 rep_out = R_valid u R_new (ascending)
+ * plus the lists of Eq. (6): add = R_new, rem = R^(l) \ R_valid.
+ * rep_in_cnt[b] = 0 is legal (every token is added).  rep_out may not alias
+ * rep_in.  Optional outputs, both indexed by token and of size B*T:
+ * gamma_rep (0 for tokens outside the inherited set) and gamma_cross (0 for
+ * inherited representatives).
+ */
+ada_status ada_cascade_step(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d,
+                            int64_t ldx, ada_dtype dt, double tau, const int32_t* rep_in,
+                            const int32_t* rep_in_cnt, int32_t* rep_out, int32_t* rep_out_cnt,
+                            int32_t* add_idx, int32_t* add_cnt, int32_t* rem_idx,
+                            int32_t* rem_cnt, float* gamma_rep, float* gamma_cross,
+                            uint32_t flags, void* stream);
+
+/* Same operations with HOST buffers: inputs are copied to the device, the
+ * device-pointer call above runs, results are copied back, and the call
+ * returns after synchronising its own stream.  Counts are int32[B] on the
+ * host.  The context must have been created with maxima covering the sizes. */
+ada_status ada_select_full_host(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d,
+                                ada_dtype dt, double tau, int32_t* rep_idx, int32_t* rep_cnt,
+                                float* gamma);
+ada_status ada_cascade_step_host(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d,
+                                 ada_dtype dt, double tau, const int32_t* rep_in,
+                                 const int32_t* rep_in_cnt, int32_t* rep_out,
+                                 int32_t* rep_out_cnt, int32_t* add_idx, int32_t* add_cnt,
+                                 int32_t* rem_idx, int32_t* rem_cnt, float* gamma_rep,
+                                 float* gamma_cross, uint32_t flags);
+
+/* Gram operation counts of Eq. (4)/(5), d included: cascade == 0 -> T^2 d;
+ * cascade != 0 -> r^2 d + (T - r) r d with r the INHERITED count.  Pure host
+ * arithmetic; returns 0 for negative arguments or r > T. */
+uint64_t ada_gram_op_count(int cascade, int64_t T, int64_t d, int64_t r);
+
+/* Synchronise `stream`, then report and clear the device status word: returns
+ * ADA_OK or the most severe device-detected error since the last call.
+ * n_zero_norm_rows (optional, host) receives the number of zero rows seen. */
+ada_status ada_device_status(ada_ctx* ctx, void* stream, int64_t* n_zero_norm_rows);
+
+/* Per-kernel timing (for benchmarks): when enabled, every kernel launch of
+ * this context is bracketed by CUDA events on the launching stream.
+ * ada_profile_read synchronises those events, fills up to `cap` entries
+ * (kernel name, launches, total milliseconds), resets the counters and
+ * returns the number of kernels known. */
+ada_status ada_profile_enable(ada_ctx* ctx, int on);
+int ada_profile_read(ada_ctx* ctx, const char** names, int64_t* launches, double* total_ms,
+                     int cap);
+
+const char* ada_status_string(ada_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ADA_H_ */

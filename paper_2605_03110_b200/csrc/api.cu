@@ -1,0 +1,459 @@
+// C ABI of libada.so: argument checks, workspace, kernel sequencing.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+
+#include "common.cuh"
+
+using namespace ada;
+
+namespace {
+
+const char* const kKernelNames[K_COUNT] = {
+    "scatter_roles",   "norm_gather",      "gram_ffma_tri",  "gram_ffma_cross",
+    "gram_tc_tri",     "gram_tc_cross",    "compact_full",   "compact_cascade",
+};
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+ada_status check_common(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d, int64_t ldx,
+                        ada_dtype dt) {
+    if (ctx == nullptr || X == nullptr) return ADA_ERR_INVALID_ARG;
+    if (B < 1 || T < 1 || d < 1 || ldx < d) return ADA_ERR_INVALID_ARG;
+    if (dt != ADA_F32 && dt != ADA_BF16) return ADA_ERR_INVALID_ARG;
+    if (dt != ctx->dt) return ADA_ERR_UNSUPPORTED;
+    if (B > ctx->maxB || T > ctx->maxT || d > ctx->maxd) return ADA_ERR_WORKSPACE;
+    const int64_t es = dt == ADA_F32 ? 4 : 2;
+    if (!aligned16(X) || (ldx * es) % 16 != 0 || (d * es) % 16 != 0) return ADA_ERR_UNSUPPORTED;
+    return ADA_OK;
+}
+
+inline bool tau_ok(double tau) { return tau > 0.0 && tau < 1.0; }  // also rejects NaN
+
+struct DeviceGuard {
+    int prev = -1;
+    explicit DeviceGuard(int dev) {
+        cudaGetDevice(&prev);
+        if (prev != dev) cudaSetDevice(dev);
+        else prev = -1;
+    }
+    ~DeviceGuard() {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+bool use_tc(const ada_ctx* ctx, ada_dtype dt) {
+    if (dt != ADA_BF16) return false;
+    if (ctx->engine == ADA_ENGINE_FFMA) return false;
+    return gram_tc_available();
+}
+
+cudaError_t run_gram(ada_ctx* ctx, const GramProblem& p, ada_dtype dt, cudaStream_t s) {
+    if (use_tc(ctx, dt)) return launch_gram_tc(ctx, p, s);
+    return launch_gram_ffma(ctx, p, dt, s);
+}
+
+#define CU(x)                                  \
+    do {                                       \
+        cudaError_t e__ = (x);                 \
+        if (e__ != cudaSuccess) return ADA_ERR_CUDA; \
+    } while (0)
+
+}  // namespace
+
+namespace ada {
+
+void prof_begin(ada_ctx* ctx, int kid, cudaStream_t s) {
+    Profiler& pr = ctx->prof;
+    if (!pr.on || pr.n >= Profiler::MAXREC) return;
+    if (pr.n >= pr.created) {
+        cudaEventCreate(&pr.ev0[pr.n]);
+        cudaEventCreate(&pr.ev1[pr.n]);
+        pr.created = pr.n + 1;
+    }
+    pr.kid[pr.n] = kid;
+    cudaEventRecord(pr.ev0[pr.n], s);
+}
+
+void prof_end(ada_ctx* ctx, cudaStream_t s) {
+    Profiler& pr = ctx->prof;
+    if (!pr.on || pr.n >= Profiler::MAXREC) return;
+    cudaEventRecord(pr.ev1[pr.n], s);
+    ++pr.n;
+}
+
+}  // namespace ada
+
+extern "C" {
+
+const char* ada_status_string(ada_status s) {
+    switch (s) {
+        case ADA_OK: return "ADA_OK";
+        case ADA_ERR_INVALID_ARG: return "ADA_ERR_INVALID_ARG";
+        case ADA_ERR_UNSUPPORTED: return "ADA_ERR_UNSUPPORTED";
+        case ADA_ERR_WORKSPACE: return "ADA_ERR_WORKSPACE";
+        case ADA_ERR_CUDA: return "ADA_ERR_CUDA";
+        case ADA_ERR_BAD_INDEX_SET: return "ADA_ERR_BAD_INDEX_SET";
+        case ADA_ERR_NONFINITE: return "ADA_ERR_NONFINITE";
+        case ADA_ERR_TIMEOUT: return "ADA_ERR_TIMEOUT";
+    }
+    return "ADA_ERR_UNKNOWN";
+}
+
+uint64_t ada_gram_op_count(int cascade, int64_t T, int64_t d, int64_t r) {
+    if (T < 0 || d < 0 || r < 0) return 0;
+    const uint64_t t = (uint64_t)T, dd = (uint64_t)d, rr = (uint64_t)r;
+    if (!cascade) return t * t * dd;
+    if (r > T) return 0;
+    return rr * rr * dd + (t - rr) * rr * dd;
+}
+
+ada_status ada_create(ada_ctx** out, int device, int64_t maxB, int64_t maxT, int64_t maxd,
+                      ada_dtype dt) {
+    if (out == nullptr) return ADA_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (maxB < 1 || maxT < 1 || maxd < 1 || (dt != ADA_F32 && dt != ADA_BF16))
+        return ADA_ERR_INVALID_ARG;
+    if (maxT > (int64_t)1 << 24 || maxB * maxT > (int64_t)1 << 30) return ADA_ERR_INVALID_ARG;
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev)
+        return ADA_ERR_CUDA;
+    DeviceGuard guard(device);
+    ada_ctx* ctx = new (std::nothrow) ada_ctx();
+    if (ctx == nullptr) return ADA_ERR_CUDA;
+    ctx->device = device;
+    ctx->maxB = maxB; ctx->maxT = maxT; ctx->maxd = maxd;
+    ctx->dt = dt;
+    ctx->es = dt == ADA_F32 ? 4 : 2;
+    ctx->engine = ADA_ENGINE_AUTO;
+    ctx->stage = nullptr; ctx->stage_bytes = 0; ctx->host_stream = nullptr;
+    cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
+
+    const size_t n_tok = (size_t)maxB * (size_t)maxT;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    // role, g_tok, g_rep are contiguous so that one memset clears them
+    const size_t o_role = take(n_tok * 4), o_gtok = take(n_tok * 4), o_grep = take(n_tok * 4);
+    const size_t o_inv = take(n_tok * 4), o_invr = take(n_tok * 4);
+    const size_t o_reff = take((size_t)maxB * 4), o_stat = take(32), o_ctr = take(32);
+    const size_t o_xrep = take(n_tok * (size_t)maxd * ctx->es + 1024);
+    if (cudaMalloc(&ctx->ws, off) != cudaSuccess) {
+        cudaGetLastError();
+        delete ctx;
+        return ADA_ERR_CUDA;
+    }
+    ctx->role = reinterpret_cast<int32_t*>(ctx->ws + o_role);
+    ctx->g_tok = reinterpret_cast<unsigned*>(ctx->ws + o_gtok);
+    ctx->g_rep = reinterpret_cast<unsigned*>(ctx->ws + o_grep);
+    ctx->inv_norm = reinterpret_cast<float*>(ctx->ws + o_inv);
+    ctx->inv_rep = reinterpret_cast<float*>(ctx->ws + o_invr);
+    ctx->r_eff = reinterpret_cast<int32_t*>(ctx->ws + o_reff);
+    ctx->status = reinterpret_cast<unsigned*>(ctx->ws + o_stat);
+    ctx->tile_ctr = reinterpret_cast<unsigned*>(ctx->ws + o_ctr);
+    ctx->Xrep = ctx->ws + o_xrep;
+    if (cudaMemset(ctx->ws, 0, o_xrep) != cudaSuccess) {
+        cudaFree(ctx->ws);
+        delete ctx;
+        return ADA_ERR_CUDA;
+    }
+    *out = ctx;
+    return ADA_OK;
+}
+
+ada_status ada_destroy(ada_ctx* ctx) {
+    if (ctx == nullptr) return ADA_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaDeviceSynchronize();
+    for (int i = 0; i < ctx->prof.created; ++i) {
+        cudaEventDestroy(ctx->prof.ev0[i]);
+        cudaEventDestroy(ctx->prof.ev1[i]);
+    }
+    if (ctx->stage) cudaFree(ctx->stage);
+    if (ctx->host_stream) cudaStreamDestroy(ctx->host_stream);
+    cudaFree(ctx->ws);
+    delete ctx;
+    return ADA_OK;
+}
+
+ada_status ada_set_engine(ada_ctx* ctx, ada_engine e) {
+    if (ctx == nullptr) return ADA_ERR_INVALID_ARG;
+    if (e != ADA_ENGINE_AUTO && e != ADA_ENGINE_FFMA && e != ADA_ENGINE_TCGEN05)
+        return ADA_ERR_INVALID_ARG;
+    if (e == ADA_ENGINE_TCGEN05 && (ctx->dt != ADA_BF16 || !gram_tc_available()))
+        return ADA_ERR_UNSUPPORTED;
+    ctx->engine = e;
+    return ADA_OK;
+}
+
+ada_status ada_normalize(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d,
+                         int64_t ldx, ada_dtype dt, void* Xhat, float* inv_norm,
+                         const int32_t* rep_idx, const int32_t* rep_cnt, void* Xrep,
+                         void* stream) {
+    ada_status st = check_common(ctx, X, B, T, d, ldx, dt);
+    if (st != ADA_OK) return st;
+    const bool gather = rep_idx != nullptr || rep_cnt != nullptr || Xrep != nullptr;
+    if (gather && (rep_idx == nullptr || rep_cnt == nullptr || Xrep == nullptr))
+        return ADA_ERR_INVALID_ARG;
+    if ((Xhat != nullptr && !aligned16(Xhat)) || (Xrep != nullptr && !aligned16(Xrep)))
+        return ADA_ERR_UNSUPPORTED;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t n_tok = (size_t)B * T;
+    if (gather) {
+        CU(cudaMemsetAsync(ctx->role, 0, n_tok * 4, s));
+        CU(launch_scatter(ctx, rep_idx, rep_cnt, (int)B, (int)T, s));
+    }
+    CU(launch_norm_gather(ctx, X, (int)B, (int)T, (int)d, ldx, dt, inv_norm, Xhat,
+                          gather ? ctx->role : nullptr, Xrep, ctx->inv_rep, s));
+    return ADA_OK;
+}
+
+ada_status ada_select_full(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d,
+                           int64_t ldx, ada_dtype dt, double tau, int32_t* rep_idx,
+                           int32_t* rep_cnt, float* gamma, void* stream) {
+    ada_status st = check_common(ctx, X, B, T, d, ldx, dt);
+    if (st != ADA_OK) return st;
+    if (rep_idx == nullptr || rep_cnt == nullptr || !tau_ok(tau)) return ADA_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t n_tok = (size_t)B * T;
+    const float thr = (float)(1.0 - tau * tau);
+
+    CU(cudaMemsetAsync(ctx->g_tok, 0, n_tok * 4, s));
+    CU(launch_norm_gather(ctx, X, (int)B, (int)T, (int)d, ldx, dt, ctx->inv_norm, nullptr,
+                          nullptr, nullptr, nullptr, s));
+    GramProblem p;
+    memset(&p, 0, sizeof(p));
+    p.A = X; p.Bm = X;
+    p.lda = ldx; p.ldb = ldx;
+    p.a_batch = T * ldx; p.b_batch = T * ldx;
+    p.inv_a = ctx->inv_norm; p.inv_b = ctx->inv_norm;
+    p.out = ctx->g_tok;
+    p.n_dev = nullptr; p.n_host = (int)T;
+    p.rows = (int)T; p.cap = (int)T; p.d = (int)d; p.B = (int)B;
+    p.tri = 1;
+    CU(run_gram(ctx, p, dt, s));
+    CU(launch_compact_full(ctx, (int)B, (int)T, thr, rep_idx, rep_cnt, gamma, s));
+    return ADA_OK;
+}
+
+ada_status ada_cascade_step(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d,
+                            int64_t ldx, ada_dtype dt, double tau, const int32_t* rep_in,
+                            const int32_t* rep_in_cnt, int32_t* rep_out, int32_t* rep_out_cnt,
+                            int32_t* add_idx, int32_t* add_cnt, int32_t* rem_idx,
+                            int32_t* rem_cnt, float* gamma_rep, float* gamma_cross,
+                            uint32_t flags, void* stream) {
+    ada_status st = check_common(ctx, X, B, T, d, ldx, dt);
+    if (st != ADA_OK) return st;
+    if (rep_in == nullptr || rep_in_cnt == nullptr || rep_out == nullptr ||
+        rep_out_cnt == nullptr || add_idx == nullptr || add_cnt == nullptr ||
+        rem_idx == nullptr || rem_cnt == nullptr || !tau_ok(tau))
+        return ADA_ERR_INVALID_ARG;
+    if (rep_out == rep_in || (flags & ~ADA_CROSS_CAUSAL) != 0) return ADA_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t n_tok_cap = (size_t)ctx->maxB * ctx->maxT;
+    const size_t n_tok = (size_t)B * T;
+    const float thr = (float)(1.0 - tau * tau);
+    (void)n_tok;
+
+    // role, g_tok, g_rep are contiguous in the workspace: one memset clears all three
+    CU(cudaMemsetAsync(ctx->role, 0, (size_t)((char*)ctx->g_rep - (char*)ctx->role) + n_tok_cap * 4, s));
+    CU(launch_scatter(ctx, rep_in, rep_in_cnt, (int)B, (int)T, s));
+    // lines 1-2: inverse norms of all rows; inherited rows gathered into Xrep
+    CU(launch_norm_gather(ctx, X, (int)B, (int)T, (int)d, ldx, dt, ctx->inv_norm, nullptr,
+                          ctx->role, ctx->Xrep, ctx->inv_rep, s));
+    // lines 3-4: r x r Gram among inherited reps, max over earlier ones
+    GramProblem p;
+    memset(&p, 0, sizeof(p));
+    p.A = ctx->Xrep; p.Bm = ctx->Xrep;
+    p.lda = d; p.ldb = d;
+    p.a_batch = T * d; p.b_batch = T * d;
+    p.inv_a = ctx->inv_rep; p.inv_b = ctx->inv_rep;
+    p.out = ctx->g_rep;
+    p.n_dev = ctx->r_eff; p.n_host = 0;
+    p.rows = (int)T; p.cap = (int)T; p.d = (int)d; p.B = (int)B;
+    p.tri = 1;
+    CU(run_gram(ctx, p, dt, s));
+    // lines 6-8: cross-Gram of all rows against the valid inherited reps
+    GramProblem q;
+    memset(&q, 0, sizeof(q));
+    q.A = X; q.Bm = ctx->Xrep;
+    q.lda = ldx; q.ldb = d;
+    q.a_batch = T * ldx; q.b_batch = T * d;
+    q.inv_a = ctx->inv_norm; q.inv_b = ctx->inv_rep;
+    q.out = ctx->g_tok;
+    q.n_dev = ctx->r_eff; q.n_host = 0;
+    q.rows = (int)T; q.cap = (int)T; q.d = (int)d; q.B = (int)B;
+    q.tri = 0;
+    q.col_gate = ctx->g_rep;
+    q.thr_bits = 0;
+    memcpy(&q.thr_bits, &thr, 4);
+    q.col_token = rep_in;
+    q.row_role = ctx->role;
+    q.causal = (flags & ADA_CROSS_CAUSAL) ? 1 : 0;
+    CU(run_gram(ctx, q, dt, s));
+    // lines 5, 9, 10-11
+    CU(launch_compact_cascade(ctx, (int)B, (int)T, thr, rep_in, rep_out, rep_out_cnt, add_idx,
+                              add_cnt, rem_idx, rem_cnt, gamma_rep, gamma_cross, s));
+    return ADA_OK;
+}
+
+ada_status ada_device_status(ada_ctx* ctx, void* stream, int64_t* n_zero_norm_rows) {
+    if (ctx == nullptr) return ADA_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    unsigned h[8];
+    CU(cudaMemcpyAsync(h, ctx->status, sizeof(h), cudaMemcpyDeviceToHost, s));
+    CU(cudaMemsetAsync(ctx->status, 0, sizeof(h), s));
+    CU(cudaStreamSynchronize(s));
+    if (n_zero_norm_rows != nullptr) *n_zero_norm_rows = (int64_t)h[1];
+    if (h[0] & ST_TIMEOUT) return ADA_ERR_TIMEOUT;
+    if (h[0] & (ST_BAD_INDEX | ST_BAD_COUNT)) return ADA_ERR_BAD_INDEX_SET;
+    if (h[0] & ST_NONFINITE) return ADA_ERR_NONFINITE;
+    return ADA_OK;
+}
+
+// ---------------------------------------------------------------------------
+// host-buffer entry points
+// ---------------------------------------------------------------------------
+static ada_status ensure_stage(ada_ctx* ctx) {
+    if (ctx->stage != nullptr) return ADA_OK;
+    const size_t n_tok = (size_t)ctx->maxB * ctx->maxT;
+    // X | 5 index lists | 2 gamma arrays | 4 count arrays
+    const size_t bytes = align_up(n_tok * ctx->maxd * ctx->es, 256) + 7 * align_up(n_tok * 4, 256) +
+                         4 * align_up((size_t)ctx->maxB * 4, 256);
+    if (cudaMalloc(&ctx->stage, bytes) != cudaSuccess) {
+        cudaGetLastError();
+        return ADA_ERR_CUDA;
+    }
+    ctx->stage_bytes = bytes;
+    if (cudaStreamCreateWithFlags(&ctx->host_stream, cudaStreamNonBlocking) != cudaSuccess)
+        return ADA_ERR_CUDA;
+    return ADA_OK;
+}
+
+struct Stage {
+    char* X;
+    int32_t *l0, *l1, *l2, *l3;
+    float *g0, *g1;
+    int32_t *c0, *c1, *c2, *c3;
+};
+
+static Stage carve(ada_ctx* ctx) {
+    const size_t n_tok = (size_t)ctx->maxB * ctx->maxT;
+    const size_t lx = align_up(n_tok * ctx->maxd * ctx->es, 256), ll = align_up(n_tok * 4, 256),
+                 lc = align_up((size_t)ctx->maxB * 4, 256);
+    Stage st;
+    char* p = ctx->stage;
+    st.X = p; p += lx;
+    st.l0 = (int32_t*)p; p += ll;
+    st.l1 = (int32_t*)p; p += ll;
+    st.l2 = (int32_t*)p; p += ll;
+    st.l3 = (int32_t*)p; p += ll;
+    st.g0 = (float*)p; p += ll;
+    st.g1 = (float*)p; p += ll;
+    p += ll;
+    st.c0 = (int32_t*)p; p += lc;
+    st.c1 = (int32_t*)p; p += lc;
+    st.c2 = (int32_t*)p; p += lc;
+    st.c3 = (int32_t*)p;
+    return st;
+}
+
+ada_status ada_select_full_host(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d,
+                                ada_dtype dt, double tau, int32_t* rep_idx, int32_t* rep_cnt,
+                                float* gamma) {
+    if (ctx == nullptr || X == nullptr || rep_idx == nullptr || rep_cnt == nullptr)
+        return ADA_ERR_INVALID_ARG;
+    if (B < 1 || T < 1 || d < 1) return ADA_ERR_INVALID_ARG;
+    if (B > ctx->maxB || T > ctx->maxT || d > ctx->maxd) return ADA_ERR_WORKSPACE;
+    DeviceGuard guard(ctx->device);
+    ada_status st = ensure_stage(ctx);
+    if (st != ADA_OK) return st;
+    Stage sg = carve(ctx);
+    cudaStream_t s = ctx->host_stream;
+    const size_t n_tok = (size_t)B * T;
+    CU(cudaMemcpyAsync(sg.X, X, n_tok * d * ctx->es, cudaMemcpyHostToDevice, s));
+    st = ada_select_full(ctx, sg.X, B, T, d, d, dt, tau, sg.l0, sg.c0, gamma ? sg.g0 : nullptr, s);
+    if (st != ADA_OK) return st;
+    CU(cudaMemcpyAsync(rep_idx, sg.l0, n_tok * 4, cudaMemcpyDeviceToHost, s));
+    CU(cudaMemcpyAsync(rep_cnt, sg.c0, (size_t)B * 4, cudaMemcpyDeviceToHost, s));
+    if (gamma) CU(cudaMemcpyAsync(gamma, sg.g0, n_tok * 4, cudaMemcpyDeviceToHost, s));
+    CU(cudaStreamSynchronize(s));
+    return ADA_OK;
+}
+
+ada_status ada_cascade_step_host(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d,
+                                 ada_dtype dt, double tau, const int32_t* rep_in,
+                                 const int32_t* rep_in_cnt, int32_t* rep_out,
+                                 int32_t* rep_out_cnt, int32_t* add_idx, int32_t* add_cnt,
+                                 int32_t* rem_idx, int32_t* rem_cnt, float* gamma_rep,
+                                 float* gamma_cross, uint32_t flags) {
+    if (ctx == nullptr || X == nullptr || rep_in == nullptr || rep_in_cnt == nullptr ||
+        rep_out == nullptr || rep_out_cnt == nullptr || add_idx == nullptr ||
+        add_cnt == nullptr || rem_idx == nullptr || rem_cnt == nullptr)
+        return ADA_ERR_INVALID_ARG;
+    if (B < 1 || T < 1 || d < 1) return ADA_ERR_INVALID_ARG;
+    if (B > ctx->maxB || T > ctx->maxT || d > ctx->maxd) return ADA_ERR_WORKSPACE;
+    DeviceGuard guard(ctx->device);
+    ada_status st = ensure_stage(ctx);
+    if (st != ADA_OK) return st;
+    Stage sg = carve(ctx);
+    cudaStream_t s = ctx->host_stream;
+    const size_t n_tok = (size_t)B * T;
+    CU(cudaMemcpyAsync(sg.X, X, n_tok * d * ctx->es, cudaMemcpyHostToDevice, s));
+    CU(cudaMemcpyAsync(sg.l0, rep_in, n_tok * 4, cudaMemcpyHostToDevice, s));
+    CU(cudaMemcpyAsync(sg.c0, rep_in_cnt, (size_t)B * 4, cudaMemcpyHostToDevice, s));
+    st = ada_cascade_step(ctx, sg.X, B, T, d, d, dt, tau, sg.l0, sg.c0, sg.l1, sg.c1, sg.l2, sg.c2,
+                          sg.l3, sg.c3, gamma_rep ? sg.g0 : nullptr, gamma_cross ? sg.g1 : nullptr,
+                          flags, s);
+    if (st != ADA_OK) return st;
+    CU(cudaMemcpyAsync(rep_out, sg.l1, n_tok * 4, cudaMemcpyDeviceToHost, s));
+    CU(cudaMemcpyAsync(add_idx, sg.l2, n_tok * 4, cudaMemcpyDeviceToHost, s));
+    CU(cudaMemcpyAsync(rem_idx, sg.l3, n_tok * 4, cudaMemcpyDeviceToHost, s));
+    CU(cudaMemcpyAsync(rep_out_cnt, sg.c1, (size_t)B * 4, cudaMemcpyDeviceToHost, s));
+    CU(cudaMemcpyAsync(add_cnt, sg.c2, (size_t)B * 4, cudaMemcpyDeviceToHost, s));
+    CU(cudaMemcpyAsync(rem_cnt, sg.c3, (size_t)B * 4, cudaMemcpyDeviceToHost, s));
+    if (gamma_rep) CU(cudaMemcpyAsync(gamma_rep, sg.g0, n_tok * 4, cudaMemcpyDeviceToHost, s));
+    if (gamma_cross) CU(cudaMemcpyAsync(gamma_cross, sg.g1, n_tok * 4, cudaMemcpyDeviceToHost, s));
+    CU(cudaStreamSynchronize(s));
+    return ADA_OK;
+}
+
+ada_status ada_profile_enable(ada_ctx* ctx, int on) {
+    if (ctx == nullptr) return ADA_ERR_INVALID_ARG;
+    ctx->prof.on = on != 0;
+    ctx->prof.n = 0;
+    return ADA_OK;
+}
+
+int ada_profile_read(ada_ctx* ctx, const char** names, int64_t* launches, double* total_ms,
+                     int cap) {
+    if (ctx == nullptr) return 0;
+    DeviceGuard guard(ctx->device);
+    Profiler& pr = ctx->prof;
+    int64_t cnt[K_COUNT] = {0};
+    double ms[K_COUNT] = {0};
+    for (int i = 0; i < pr.n; ++i) {
+        cudaEventSynchronize(pr.ev1[i]);
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, pr.ev0[i], pr.ev1[i]) == cudaSuccess) {
+            cnt[pr.kid[i]] += 1;
+            ms[pr.kid[i]] += t;
+        }
+    }
+    pr.n = 0;
+    for (int k = 0; k < K_COUNT && k < cap; ++k) {
+        if (names) names[k] = kKernelNames[k];
+        if (launches) launches[k] = cnt[k];
+        if (total_ms) total_ms[k] = ms[k];
+    }
+    return K_COUNT;
+}
+
+}  // extern "C"

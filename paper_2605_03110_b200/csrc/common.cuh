@@ -1,0 +1,127 @@
+// Internal declarations shared by the translation units of libada.so.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/ada.h"
+
+namespace ada {
+
+// bits of the device status word (status[0])
+enum : unsigned {
+    ST_BAD_INDEX = 1u << 0,  // inherited list not strictly ascending / out of [0,T)
+    ST_BAD_COUNT = 1u << 1,  // a count outside [0,T]
+    ST_NONFINITE = 1u << 2,  // NaN / Inf met while normalising
+    ST_TIMEOUT = 1u << 3,    // a bounded wait in a kernel ran out
+};
+// status[1] counts zero-norm rows, status[2] records where a wait gave up.
+
+enum KernelId {
+    K_SCATTER = 0,
+    K_NORM_GATHER,
+    K_GRAM_FFMA_TRI,
+    K_GRAM_FFMA_CROSS,
+    K_GRAM_TC_TRI,
+    K_GRAM_TC_CROSS,
+    K_COMPACT_FULL,
+    K_COMPACT_CASCADE,
+    K_COUNT
+};
+
+// One masked-Gram-with-row-maximum problem, batched over B sequences.
+//   C(i,j) = a_i . b_j           a_i = row i of A, b_j = row j of Bm (both K-major)
+//   v(i,j) = |C(i,j)| * inv_a[i] * inv_b[j]
+//   out[i] = max over admissible j of v(i,j), combined with atomicMax on the
+//            IEEE bit pattern (v >= 0, so unsigned order == float order)
+// tri  : A == Bm, admissible j < i, i < n
+// cross: rows i < T of X against columns j < n of the gathered representative
+//        rows; admissible iff col_gate[j] < thr_bits (the representative is
+//        valid) and, when causal, col_token[j] < i; rows with row_role[i] != 0
+//        (inherited representatives) produce nothing.
+struct GramProblem {
+    const void* A;            // rows of the left operand
+    const void* Bm;           // rows of the right operand
+    int64_t lda, ldb;         // row strides in elements
+    int64_t a_batch, b_batch; // batch strides in elements
+    const float* inv_a;       // [B*cap]
+    const float* inv_b;       // [B*cap]
+    unsigned* out;            // [B*cap] gamma bit patterns (zero-initialised)
+    const int32_t* n_dev;     // [B] device-resident column/row count, or NULL
+    int n_host;               // used when n_dev == NULL
+    int rows;                 // number of A rows (cross); ignored for tri
+    int cap;                  // per-sequence capacity (= T) of the per-token arrays
+    int d;                    // contraction length
+    int B;
+    int tri;                  // 1: lower-triangular self Gram, 0: cross
+    // cross only
+    const unsigned* col_gate; // [B*cap] gamma_rep bits by position
+    unsigned thr_bits;        // bit pattern of (float)thr
+    const int32_t* col_token; // [B*cap] token index of each column (causal) or NULL
+    const int32_t* row_role;  // [B*cap] 0 for non-representatives
+    int causal;
+};
+
+struct Profiler {
+    bool on = false;
+    static const int MAXREC = 4096;
+    cudaEvent_t ev0[MAXREC], ev1[MAXREC];
+    int kid[MAXREC];
+    int n = 0, created = 0;
+};
+
+}  // namespace ada
+
+struct ada_ctx {
+    int device;
+    int64_t maxB, maxT, maxd;
+    ada_dtype dt;
+    int es;
+    ada_engine engine;
+    int sm_count;
+    // device workspace
+    char* ws;            // one allocation
+    float* inv_norm;     // [maxB*maxT] 1/||x_t||
+    float* inv_rep;      // [maxB*maxT] 1/||x|| of gathered rows, by position
+    unsigned* g_tok;     // [maxB*maxT] gamma (full) or gamma_cross, by token, bit patterns
+    unsigned* g_rep;     // [maxB*maxT] gamma_rep by position, bit patterns
+    int32_t* role;       // [maxB*maxT] 0 = not inherited, p+1 = position p in the inherited list
+    int32_t* r_eff;      // [maxB] sanitised inherited counts
+    unsigned* status;    // [8]
+    unsigned* tile_ctr;  // [8] persistent-kernel tile counters
+    void* Xrep;          // [maxB*maxT*maxd] gathered representative rows (raw values)
+    // staging for the *_host entry points (allocated on first use)
+    char* stage;
+    size_t stage_bytes;
+    cudaStream_t host_stream;
+    ada::Profiler prof;
+};
+
+namespace ada {
+
+// RAII-free launch bracket used by every launcher.
+void prof_begin(ada_ctx* ctx, int kid, cudaStream_t s);
+void prof_end(ada_ctx* ctx, cudaStream_t s);
+
+// prep_kernels.cu
+cudaError_t launch_scatter(ada_ctx* ctx, const int32_t* rep_in, const int32_t* rep_in_cnt, int B,
+                           int T, cudaStream_t s);
+cudaError_t launch_norm_gather(ada_ctx* ctx, const void* X, int B, int T, int d, int64_t ldx,
+                               ada_dtype dt, float* inv_norm, void* Xhat, const int32_t* role,
+                               void* Xrep, float* inv_rep, cudaStream_t s);
+cudaError_t launch_compact_full(ada_ctx* ctx, int B, int T, float thr, int32_t* rep_idx,
+                                int32_t* rep_cnt, float* gamma, cudaStream_t s);
+cudaError_t launch_compact_cascade(ada_ctx* ctx, int B, int T, float thr, const int32_t* rep_in,
+                                   int32_t* rep_out, int32_t* rep_out_cnt, int32_t* add_idx,
+                                   int32_t* add_cnt, int32_t* rem_idx, int32_t* rem_cnt,
+                                   float* gamma_rep, float* gamma_cross, cudaStream_t s);
+
+// gram_ffma.cu
+cudaError_t launch_gram_ffma(ada_ctx* ctx, const GramProblem& p, ada_dtype dt, cudaStream_t s);
+
+// gram_tc.cu (bf16, tcgen05 + TMA)
+cudaError_t launch_gram_tc(ada_ctx* ctx, const GramProblem& p, cudaStream_t s);
+bool gram_tc_available();
+
+}  // namespace ada

@@ -1,0 +1,292 @@
+"""GPU-vs-oracle parity of the selection path, through the C ABI (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_03110_b200 import workloads as wl
+from label_model import cascade_from_labels, full_from_labels
+
+pytestmark = pytest.mark.gpu
+
+TAU = 0.3
+
+
+@pytest.fixture(scope="module")
+def ada():
+    from paper_2605_03110_b200 import binding
+    assert torch.cuda.is_available()
+    binding.lib()
+    return binding
+
+
+def clustered(T, d, seed, dtype):
+    rng = np.random.default_rng(seed)
+    P = max(1, T // 5)
+    base = rng.standard_normal((P, d))
+    X = base[rng.integers(0, P, T)] + 0.05 * rng.standard_normal((T, d))
+    X[rng.integers(0, T, max(1, T // 10))] = rng.standard_normal((max(1, T // 10), d))
+    X = X.astype(np.float32)[None]
+    return wl.f32_to_bf16_bits(X) if dtype == "bf16" else X
+
+
+ENGINES = [("f32", 0), ("bf16", 0), ("bf16", 1)]   # (storage, engine): AUTO, AUTO, forced FFMA
+
+
+@pytest.mark.parametrize("dtype,engine", ENGINES)
+@pytest.mark.parametrize("T", [1, 2, 3, 127, 128, 129, 257, 600])
+@pytest.mark.parametrize("d", [8, 72, 768])
+def test_small_shapes_full_and_cascade(ada, dtype, engine, T, d):
+    from parity import check_cascade, check_full
+    ctx = ada.ada_create(1, T, d, ada.ADA_F32 if dtype == "f32" else ada.ADA_BF16)
+    ada.ada_set_engine(ctx, engine)
+    X0 = clustered(T, d, 1000 + T + d, dtype)
+    X1 = clustered(T, d, 1000 + T + d, dtype)       # same prototypes, then perturbed
+    rng = np.random.default_rng(T * 7 + d)
+    if dtype == "bf16":
+        X1 = wl.f32_to_bf16_bits(wl.bf16_bits_to_f32(X1) + 0.3 * rng.standard_normal(X1.shape).astype(np.float32))
+    else:
+        X1 = X1 + 0.3 * rng.standard_normal(X1.shape).astype(np.float32)
+    # the checks assert parity outside the tolerance band; at tiny d a gamma may
+    # land inside it by chance, which is tolerated (and counted) by design
+    band, reps = check_full(ctx, X0, TAU)
+    for causal in (False, True):
+        check_cascade(ctx, X1, TAU, reps, causal=causal)
+    # degenerate inherited sets: empty, everything, a single token
+    for R in ([], list(range(T)), [T - 1]):
+        check_cascade(ctx, X1, TAU, [R])
+    ada.ada_destroy(ctx)
+
+
+def run_config_chain(ada, cfg, n_layers=None, causal=False, engine=0):
+    """Step parity with the oracle chain's inherited sets fed to both sides,
+    plus the free-running GPU chain (its own sets fed forward)."""
+    from parity import check_cascade, check_full, lists, to_device
+    ctx = ada.ada_create(cfg.B, cfg.T, cfg.d, ada.ADA_F32 if cfg.dtype == "f32" else ada.ADA_BF16)
+    ada.ada_set_engine(ctx, engine)
+    band_total = 0
+    R_oracle = None
+    free_idx = free_cnt = None
+    for lb in wl.generate_layers(cfg, seed=0, n_layers=n_layers):
+        Xd = to_device(lb.X)
+        if lb.layer == 0:
+            band, reps = check_full(ctx, lb.X, cfg.tau)
+            R_oracle = reps if band == 0 else [oracle.select_full(wl.as_f64(lb.X[b]), cfg.tau)[0]
+                                               for b in range(cfg.B)]
+            free_idx, free_cnt, _ = ada.ada_select_full(ctx, Xd, cfg.tau)
+        else:
+            band, _, refs = check_cascade(ctx, lb.X, cfg.tau, R_oracle, causal=causal)
+            R_oracle = [r.rep for r in refs]
+            out = ada.ada_cascade_step(ctx, Xd, cfg.tau, free_idx, free_cnt,
+                                       flags=ada.ADA_CROSS_CAUSAL if causal else 0)
+            free_idx, free_cnt = out.rep_out, out.rep_out_cnt
+        band_total += band
+        for b in range(cfg.B):      # label-level prediction of the full selection (no Gram)
+            assert full_from_labels(lb.labels[b]).tolist() == \
+                oracle.select_full(wl.as_f64(lb.X[b]), cfg.tau)[0].tolist() or cfg.T > 4096
+    if band_total == 0:
+        free = lists(free_idx, free_cnt)
+        for b in range(cfg.B):
+            assert free[b].tolist() == R_oracle[b].tolist()
+    st, _ = ada.ada_device_status(ctx)
+    assert st == 0
+    ada.ada_destroy(ctx)
+    return band_total
+
+
+def test_config1_gpt2_shaped_fp32(ada):
+    assert run_config_chain(ada, wl.CONFIGS[1]) == 0
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_config2_batched_bf16(ada, causal):
+    assert run_config_chain(ada, wl.CONFIGS[2], n_layers=6, causal=causal) == 0
+
+
+def test_config3_gptj_shaped_bf16(ada):
+    assert run_config_chain(ada, wl.CONFIGS[3], n_layers=5) == 0
+
+
+def test_config2_ffma_engine_matches(ada):
+    assert run_config_chain(ada, wl.scaled(wl.CONFIGS[2], B=2), n_layers=3, engine=1) == 0
+
+
+def sampled_large(ada, cfg, n_layers, n_sample=48):
+    """Full-size check where the oracle cannot do a whole layer quickly: sets by the
+    label-level prediction (exact, no Gram), gamma on sampled rows by the oracle."""
+    from parity import TOL, lists, to_device
+    tol = TOL[cfg.dtype]
+    ctx = ada.ada_create(cfg.B, cfg.T, cfg.d, ada.ADA_BF16)
+    rng = np.random.default_rng(5)
+    R_lab = None
+    for lb in wl.generate_layers(cfg, seed=0, n_layers=n_layers):
+        Xd = to_device(lb.X)
+        lab = lb.labels[0]
+        X64 = wl.as_f64(lb.X[0])
+        rep_idx, rep_cnt, gamma = ada.ada_select_full(ctx, Xd, cfg.tau)
+        full = lists(rep_idx, rep_cnt)[0]
+        assert full.tolist() == full_from_labels(lab).tolist()
+        rows = np.sort(rng.choice(cfg.T, n_sample, replace=False)).astype(np.int32)
+        g_ref = oracle.full_rows(X64, rows)
+        assert np.max(np.abs(gamma.cpu().numpy()[0][rows] - g_ref)) <= tol
+        if lb.layer == 0:
+            R_lab = full
+            R_idx, R_cnt = rep_idx, rep_cnt
+            continue
+        out = ada.ada_cascade_step(ctx, Xd, cfg.tau, R_idx, R_cnt)
+        exp_rep, exp_add, exp_rem = cascade_from_labels(lab, R_lab)
+        assert lists(out.rep_out, out.rep_out_cnt)[0].tolist() == exp_rep.tolist()
+        assert lists(out.add_idx, out.add_cnt)[0].tolist() == exp_add.tolist()
+        assert lists(out.rem_idx, out.rem_cnt)[0].tolist() == exp_rem.tolist()
+        nonrep = np.setdiff1d(np.arange(cfg.T), R_lab)
+        rows = np.sort(rng.choice(nonrep, min(n_sample, nonrep.size), replace=False)).astype(np.int32)
+        ref = oracle.cascade_step(X64, cfg.tau, R_lab, only_rows=rows)
+        assert np.max(np.abs(out.gamma_cross.cpu().numpy()[0][rows] - ref.gamma_cross[rows])) <= tol
+        g_rep_tok = np.zeros(cfg.T)
+        g_rep_tok[R_lab] = ref.gamma_rep
+        assert np.max(np.abs(out.gamma_rep.cpu().numpy()[0] - g_rep_tok)) <= tol
+        assert lists(out.rem_idx, out.rem_cnt)[0].tolist() == ref.rem.tolist()
+        R_lab, R_idx, R_cnt = exp_rep, out.rep_out, out.rep_out_cnt
+    st, _ = ada.ada_device_status(ctx)
+    assert st == 0
+    ada.ada_destroy(ctx)
+
+
+def test_config4_opt_shaped_full_size_sampled(ada):
+    sampled_large(ada, wl.CONFIGS[4], n_layers=3)
+
+
+@pytest.mark.parametrize("T,q", [(512, 0.01), (1024, 0.5), (4096, 0.05), (16384, 0.01), (16384, 0.2)])
+def test_sweep_points_sampled(ada, T, q):
+    sampled_large(ada, wl.sweep_config(T, q), n_layers=2, n_sample=24)
+
+
+def test_threshold_band_adversarial(ada):
+    """Pairs built at cos = thr +- eps by a planar rotation embedded in d dims:
+    outside the tolerance the decision must match; inside it either answer is
+    accepted and counted."""
+    from parity import check_full
+    d, thr = 256, 1 - TAU * TAU
+    for dtype, tol in (("f32", 1e-5), ("bf16", 2e-3)):
+        ctx = ada.ada_create(1, 64, d, ada.ADA_F32 if dtype == "f32" else ada.ADA_BF16)
+        rows = []
+        rng = np.random.default_rng(11)
+        Q, _ = np.linalg.qr(rng.standard_normal((d, d)))
+        k = 0
+        for eps in (1e-2, 1e-3, 1e-4, 1e-6):
+            for sgn in (+1, -1):
+                theta = np.arccos(thr + sgn * eps)
+                a, b = Q[2 * k], Q[2 * k + 1]
+                rows.append(3.0 * a)
+                rows.append(0.7 * (np.cos(theta) * a + np.sin(theta) * b))
+                k += 1
+        X = np.asarray(rows, dtype=np.float32)[None]
+        Xs = wl.f32_to_bf16_bits(X) if dtype == "bf16" else X
+        band, reps = check_full(ctx, Xs, TAU)      # asserts gamma within tol, sets outside the band
+        _, g = oracle.select_full(wl.as_f64(Xs[0]), TAU)
+        n_in_band = int(np.sum(np.abs(g - thr) <= tol))
+        assert band <= n_in_band
+        ada.ada_destroy(ctx)
+
+
+def test_duplicates_orthogonal_and_zero_rows(ada):
+    from parity import check_full, to_device
+    d = 64
+    Q, _ = np.linalg.qr(np.random.default_rng(2).standard_normal((d, d)))
+    X = (Q[:40] * np.linspace(0.5, 4, 40)[:, None]).astype(np.float32)
+    X[13] = -2.0 * X[4]
+    X[29] = 0.0
+    ctx = ada.ada_create(1, 40, d, ada.ADA_F32)
+    band, reps = check_full(ctx, X[None], TAU)
+    assert band == 0 and reps[0].tolist() == [t for t in range(40) if t != 13]
+    ada.ada_select_full(ctx, to_device(X[None]), TAU)
+    st, nz = ada.ada_device_status(ctx)
+    assert st == 0 and nz == 1
+    ada.ada_destroy(ctx)
+
+
+def test_normalize_and_gather(ada):
+    from parity import to_device
+    cfg = wl.scaled(wl.CONFIGS[2], B=2, T=300, d=264, L=1)
+    X = next(wl.generate_layers(cfg)).X
+    Xd = to_device(X)
+    ctx = ada.ada_create(2, 300, 264, ada.ADA_BF16)
+    rep = np.zeros((2, 300), dtype=np.int32)
+    rep[0, :4] = [0, 7, 8, 299]
+    rep[1, :2] = [5, 100]
+    cnt = np.array([4, 2], dtype=np.int32)
+    inv, xhat, xrep = ada.ada_normalize(ctx, Xd, want_xhat=True, rep_idx=torch.from_numpy(rep).cuda(),
+                                        rep_cnt=torch.from_numpy(cnt).cuda())
+    for b in range(2):
+        X64 = wl.as_f64(X[b])
+        Xh, nrm = oracle.normalize(X64)
+        assert np.allclose(inv[b].cpu().numpy() * nrm, 1.0, atol=1e-6)
+        assert np.max(np.abs(xhat[b].float().cpu().numpy() - Xh)) <= 2.0 ** -8 * np.max(np.abs(Xh))
+        got = xrep[b, :cnt[b]].view(torch.int16).cpu().numpy().view(np.uint16)
+        assert np.array_equal(got, X[b][rep[b, :cnt[b]]])
+    ada.ada_destroy(ctx)
+
+
+def test_error_paths(ada):
+    from parity import to_device
+    ctx = ada.ada_create(1, 64, 32, ada.ADA_F32)
+    X = torch.randn(1, 64, 32, device="cuda")
+    for tau in (0.0, 1.0, -0.3, float("nan")):
+        with pytest.raises(ada.AdaError) as e:
+            ada.ada_select_full(ctx, X, tau)
+        assert e.value.status == 1
+    with pytest.raises(ada.AdaError) as e:                      # above the context maxima
+        ada.ada_select_full(ctx, torch.randn(1, 65, 32, device="cuda"), TAU)
+    assert e.value.status == 3
+    with pytest.raises(ada.AdaError) as e:                      # wrong storage type
+        ada.ada_select_full(ctx, X.bfloat16(), TAU)
+    assert e.value.status == 2
+    with pytest.raises(ada.AdaError) as e:                      # d*es not a multiple of 16
+        ada.ada_select_full(ctx, torch.randn(1, 64, 30, device="cuda"), TAU)
+    assert e.value.status == 2
+    # device-detected: unsorted inherited list, count out of range, NaN
+    bad = torch.tensor([[3, 2] + [0] * 62], dtype=torch.int32, device="cuda")
+    ada.ada_cascade_step(ctx, X, TAU, bad, torch.tensor([2], dtype=torch.int32, device="cuda"))
+    assert ada.ada_device_status(ctx)[0] == 5
+    ada.ada_cascade_step(ctx, X, TAU, bad, torch.tensor([65], dtype=torch.int32, device="cuda"))
+    assert ada.ada_device_status(ctx)[0] == 5
+    Xn = X.clone()
+    Xn[0, 3, 3] = float("nan")
+    ada.ada_select_full(ctx, Xn, TAU)
+    assert ada.ada_device_status(ctx)[0] == 6
+    ada.ada_select_full(ctx, X, TAU)                            # the context stays usable
+    assert ada.ada_device_status(ctx)[0] == 0
+    ada.ada_destroy(ctx)
+
+
+def test_host_entry_points_match_device_ones(ada):
+    from parity import lists, to_device
+    cfg = wl.scaled(wl.CONFIGS[2], B=3, T=700, d=256, L=2)
+    Xs, _ = wl.generate_all(cfg)
+    ctx = ada.ada_create(3, 700, 256, ada.ADA_BF16)
+    d0, d1 = to_device(Xs[0]), to_device(Xs[1])
+    ri, rc, g = ada.ada_select_full(ctx, d0, cfg.tau)
+    out = ada.ada_cascade_step(ctx, d1, cfg.tau, ri, rc)
+    h0, h1 = d0.cpu().pin_memory(), d1.cpu().pin_memory()
+    i32 = lambda *s: torch.empty(s, dtype=torch.int32).pin_memory()
+    hri, hrc, hg = i32(3, 700), i32(3), torch.empty(3, 700).pin_memory()
+    ada.ada_select_full_host(ctx, h0, cfg.tau, hri, hrc, hg)
+    assert [a.tolist() for a in lists(hri, hrc)] == [a.tolist() for a in lists(ri, rc)]
+    assert torch.equal(hg, g.cpu())
+    ro, roc, ai, ac, mi, mc = i32(3, 700), i32(3), i32(3, 700), i32(3), i32(3, 700), i32(3)
+    ada.ada_cascade_step_host(ctx, h1, cfg.tau, hri, hrc, ro, roc, ai, ac, mi, mc)
+    assert [a.tolist() for a in lists(ro, roc)] == [a.tolist() for a in lists(out.rep_out, out.rep_out_cnt)]
+    assert [a.tolist() for a in lists(ai, ac)] == [a.tolist() for a in lists(out.add_idx, out.add_cnt)]
+    assert [a.tolist() for a in lists(mi, mc)] == [a.tolist() for a in lists(out.rem_idx, out.rem_cnt)]
+    ada.ada_destroy(ctx)
+
+
+def test_repeated_runs_are_bit_identical(ada):
+    from parity import to_device
+    cfg = wl.scaled(wl.CONFIGS[3], T=1024, d=512, L=1, P=100)
+    Xd = to_device(next(wl.generate_layers(cfg)).X)
+    ctx = ada.ada_create(1, 1024, 512, ada.ADA_BF16)
+    a = ada.ada_select_full(ctx, Xd, cfg.tau)
+    b = ada.ada_select_full(ctx, Xd, cfg.tau)
+    assert torch.equal(a[2], b[2]) and torch.equal(a[1], b[1])
+    ada.ada_destroy(ctx)
