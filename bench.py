@@ -1,0 +1,431 @@
+#!/usr/bin/env python
+"""Benchmark of the selection hot path: selection tokens*layers/s on one B200 (or N replicas).
+
+A "step" is one pass of the whole path over one synthetic batch: full selection
+(Definition 1) at layer 0, then one cascade step (Algorithm 1) at each of the
+layers 1..L-1, every layer's X a distinct HBM-resident tensor.  The same layers
+are also pushed through full selection at every layer ("independent" selection)
+to report the cascade speedup.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1..4] [--impl reference]
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the fp64 CPU oracle
+on the host cores instead (a deliberately plain program: a reported baseline).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2605_03110_b200 import workloads as wl  # noqa: E402
+
+METRIC = "selection tokens*layers/s (full at layer 0 + cascade at layers 1..L-1)"
+UNIT = "tokens*layers/s"
+
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant
+# kernel, from the ncu captures summarised under profiles/ (None until captured).
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            m = json.load(f)
+        return dict(hbm_gbs=m["hbm_gbs"], bf16_burst=m["bf16_tflops"],
+                    bf16_sustained=m.get("bf16_tflops_sustained", m["bf16_tflops"]), src="measured")
+    return dict(hbm_gbs=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, src="fallback")
+
+
+# ------------------------------------------------------------------------------------------
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
+               0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, device_index: int):
+        super().__init__(daemon=True)
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.h = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            try:
+                uuid = "GPU-" + str(torch.cuda.get_device_properties(device_index).uuid)
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.h = None
+
+    def run(self):
+        if self.h is None:
+            return
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM))
+                bits = self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in self.REASONS.items():
+                    if bits & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop_evt.wait(0.05)
+
+    def finish(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def jaccard(a, b):
+    a, b = set(a), set(b)
+    return 1.0 if not (a or b) else len(a & b) / len(a | b)
+
+
+# ------------------------------------------------------------------------------------------
+def reference_arm(args, cfg):
+    """The fp64 CPU oracle on the host cores, same metric, bounded sample per step."""
+    import oracle
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n_lay = min(cfg.L, args.ref_layers)
+    layers = [lb.X for lb in wl.generate_layers(cfg, seed=0, n_layers=n_lay)]
+    X64 = [[wl.as_f64(X[b]) for b in range(cfg.B)] for X in layers]
+
+    def one_step():
+        t0 = time.perf_counter()
+        R = [oracle.select_full(X64[0][b], cfg.tau)[0] for b in range(cfg.B)]
+        t_full = time.perf_counter() - t0
+        t_c = []
+        for l in range(1, n_lay):
+            t1 = time.perf_counter()
+            R = [oracle.cascade_step(X64[l][b], cfg.tau, R[b]).rep for b in range(cfg.B)]
+            t_c.append(time.perf_counter() - t1)
+        return t_full, (float(np.mean(t_c)) if t_c else t_full)
+
+    for _ in range(args.ref_warmup):
+        one_step()
+    est = []
+    for _ in range(args.steps):
+        t_full, t_casc = one_step()
+        est.append(t_full + (cfg.L - 1) * t_casc)      # scaled to the L-layer pipeline
+    t_step = float(np.mean(est))
+    value = cfg.B * cfg.T * cfg.L / t_step
+    sample = (f"layers 0..{n_lay - 1} of workload {cfg.cfg_id} computed in full by the oracle; "
+              f"step time = t(full, layer 0) + {cfg.L - 1} x mean t(cascade step)")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.ref_warmup, "ms_per_step": 1e3 * t_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": workload_dict(cfg),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(),
+                         "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def workload_dict(cfg):
+    return {"workload": f"configs[{cfg.cfg_id - 1}] {cfg.name}", "B": cfg.B, "T": cfg.T, "d": cfg.d,
+            "L": cfg.L, "tau": cfg.tau, "prototypes": cfg.P, "storage": cfg.dtype,
+            "l2": "every layer is a distinct HBM-resident tensor; one step streams "
+                  f"{cfg.L * cfg.B * cfg.T * cfg.d * cfg.es / 2**20:.0f} MiB (> 126 MB L2)",
+            "seed": 0}
+
+
+# ------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=4, choices=[1, 2, 3, 4])
+    ap.add_argument("--layers", type=int, default=0, help="override L (0 = the configuration's)")
+    ap.add_argument("--engine", type=int, default=0, help="0 auto, 1 force FFMA Gram")
+    ap.add_argument("--ref-layers", type=int, default=4)
+    ap.add_argument("--ref-warmup", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+
+    cfg = wl.CONFIGS[args.workload]
+    if args.layers:
+        cfg = wl.scaled(cfg, L=args.layers)
+    if args.impl == "reference":
+        reference_arm(args, cfg)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2605_03110_b200 import binding as ada
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    ada.lib()                                                   # fail loudly if not built
+
+    # ---- inputs: every rank draws its own replica (weak scaling, no data-path collective) ----
+    host_layers = [lb.X for lb in wl.generate_layers(cfg, seed=rank)]
+    tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+
+    def as_torch(X):
+        if X.dtype == np.uint16:
+            return torch.from_numpy(X.view(np.int16)).view(torch.bfloat16)
+        return torch.from_numpy(X)
+
+    dev_layers = [as_torch(X).to(dev) for X in host_layers]
+    B, T, d, L = cfg.B, cfg.T, cfg.d, cfg.L
+    ctx = ada.ada_create(B, T, d, ada.ADA_BF16 if cfg.dtype == "bf16" else ada.ADA_F32, device=local)
+    ada.ada_set_engine(ctx, args.engine)
+    stream = torch.cuda.current_stream()
+
+    i32 = dict(dtype=torch.int32, device=dev)
+    idx = [torch.empty((B, T), **i32) for _ in range(2)]
+    cnt = [torch.empty((B,), **i32) for _ in range(2)]
+    outs = [ada.CascadeOut(B, T, dev, want_gamma=False) for _ in range(2)]
+    r_hist = torch.zeros((L, 3, B), **i32)                      # rep count, adds, removes per layer
+
+    def cascade_pipeline(record=False):
+        ada.ada_select_full(ctx, dev_layers[0], cfg.tau, outs[0].rep_out, outs[0].rep_out_cnt,
+                            want_gamma=False, stream=stream)
+        cur = 0
+        if record:
+            r_hist[0, 0].copy_(outs[0].rep_out_cnt)
+        for l in range(1, L):
+            nxt = 1 - cur
+            ada.ada_cascade_step(ctx, dev_layers[l], cfg.tau, outs[cur].rep_out, outs[cur].rep_out_cnt,
+                                 out=outs[nxt], stream=stream)
+            cur = nxt
+            if record:
+                r_hist[l, 0].copy_(outs[cur].rep_out_cnt)
+                r_hist[l, 1].copy_(outs[cur].add_cnt)
+                r_hist[l, 2].copy_(outs[cur].rem_cnt)
+        return outs[cur]
+
+    def independent_pipeline(keep=None):
+        for l in range(L):
+            ada.ada_select_full(ctx, dev_layers[l], cfg.tau, idx[0], cnt[0], want_gamma=False,
+                                stream=stream)
+            if keep is not None:
+                keep.append((idx[0].clone(), cnt[0].clone()))
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed(fn, steps, warmup):
+        for _ in range(warmup):
+            fn()
+        barrier()
+        sampler = ClockSampler(local)
+        sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            fn()
+        e1.record(stream)
+        barrier()
+        clocks = sampler.finish()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms / steps, clocks
+
+    # ---- headline: cascade pipeline, inputs resident in HBM ----
+    ms_step, clocks = timed(cascade_pipeline, args.steps, args.warmup)
+    value = world * B * T * L / (ms_step * 1e-3)
+
+    # ---- independent selection (full Gram at every layer) for the cascade speedup ----
+    ms_indep, _ = timed(independent_pipeline, max(1, args.steps // 5), 1)
+
+    # ---- per-kernel times (events on the launching stream) and roofline of the dominant kernel ----
+    cascade_pipeline(record=True)
+    torch.cuda.synchronize()
+    hist = r_hist.cpu().numpy().astype(np.int64)                # (L, 3, B)
+    ada.ada_profile_enable(ctx, True)
+    n_prof = 3
+    for _ in range(n_prof):
+        cascade_pipeline()
+    torch.cuda.synchronize()
+    prof = ada.ada_profile_read(ctx)
+    ada.ada_profile_enable(ctx, False)
+    kernels = {k: {"launches": c // n_prof, "ms_per_step": ms / n_prof}
+               for k, (c, ms) in prof.items() if c}
+    dom = max(kernels, key=lambda k: kernels[k]["ms_per_step"])
+    r_in = hist[:-1, 0, :]                                      # inherited count at layers 1..L-1
+    r_valid = r_in - hist[1:, 2, :]
+    flops = {
+        "tri_full": float(d) * T * (T - 1) * B,
+        "tri_rep": float(np.sum(d * r_in * (r_in - 1))),
+        "cross": float(np.sum(2.0 * d * (T - r_in) * r_valid)),
+    }
+    peaks = measured_peaks()
+    es = cfg.es
+    if "cross" in dom:
+        alg, bound, per = flops["cross"], "tensor", "2*d*(T-r)*r_valid flop per launch"
+    elif "tri" in dom:
+        alg, bound, per = flops["tri_full"] + flops["tri_rep"], "tensor", "d*n*(n-1) flop per launch"
+    else:
+        alg, bound, per = float(L * B * T * d * es), "hbm", "d*es bytes per token"
+    secs = kernels[dom]["ms_per_step"] * 1e-3
+    if bound == "tensor" and cfg.dtype == "bf16":
+        peak, unit, achieved = peaks["bf16_sustained"], "TFLOP/s", alg / secs / 1e12
+        peak_note = f"cuBLAS bf16 sustained, {peaks['src']}"
+    elif bound == "tensor":
+        # fp32 FFMA path: 148 SMs x 128 lanes x 2 flop x max SM clock
+        peak, unit, achieved = 148 * 128 * 2 * 1.965e9 / 1e12, "TFLOP/s", alg / secs / 1e12
+        bound, peak_note = "alu", "148 SMs x 128 FFMA lanes x 2 flop x 1.965 GHz (derived)"
+    else:
+        peak, unit, achieved = peaks["hbm_gbs"], "GB/s", alg / secs / 1e9
+        peak_note = f"copy bandwidth, {peaks['src']}"
+    roofline = {"kernel": dom, "bound": bound, "achieved": achieved, "peak": peak, "unit": unit,
+                "frac": achieved / peak, "peak_source": peak_note,
+                "algorithmic_per_launch": per,
+                "avg_launch_ms": kernels[dom]["ms_per_step"] / kernels[dom]["launches"],
+                "traffic": NCU_TRAFFIC_BYTES.get((dom, cfg.cfg_id))}
+
+    # ---- set statistics: consecutive-layer Jaccard (independent) and cascade-vs-full Jaccard ----
+    keep = []
+    independent_pipeline(keep)
+    torch.cuda.synchronize()
+    indep = [[i[b, :int(c[b])].cpu().numpy() for b in range(B)] for i, c in keep]
+    casc_sets = []
+    ada.ada_select_full(ctx, dev_layers[0], cfg.tau, outs[0].rep_out, outs[0].rep_out_cnt,
+                        want_gamma=False)
+    cur = 0
+    casc_sets.append([outs[0].rep_out[b, :int(outs[0].rep_out_cnt[b])].cpu().numpy() for b in range(B)])
+    for l in range(1, L):
+        ada.ada_cascade_step(ctx, dev_layers[l], cfg.tau, outs[cur].rep_out, outs[cur].rep_out_cnt,
+                             out=outs[1 - cur])
+        cur = 1 - cur
+        casc_sets.append([outs[cur].rep_out[b, :int(outs[cur].rep_out_cnt[b])].cpu().numpy()
+                          for b in range(B)])
+    j_consec = [float(np.mean([jaccard(indep[l][b], indep[l + 1][b]) for b in range(B)]))
+                for l in range(L - 1)]
+    j_cvf = [float(np.mean([jaccard(indep[l][b], casc_sets[l][b]) for b in range(B)]))
+             for l in range(L)]
+    st, n_zero = ada.ada_device_status(ctx)
+    assert st == 0, ada.status_string(st)
+    ops_indep = L * ada.ada_gram_op_count(False, T, d)
+    ops_casc = ada.ada_gram_op_count(False, T, d) + int(
+        np.mean([sum(ada.ada_gram_op_count(True, T, d, int(r_in[l, b])) for l in range(L - 1))
+                 for b in range(B)]))
+
+    # ---- end to end: HOST buffers through the C ABI, copies inside the timed region ----
+    e2e = None
+    if not args.no_e2e:
+        pin = [as_torch(X).pin_memory() for X in host_layers]
+        hi = lambda *s: torch.empty(s, dtype=torch.int32).pin_memory()  # noqa: E731
+        h_idx, h_cnt = [hi(B, T), hi(B, T)], [hi(B), hi(B)]
+        h_add, h_addc, h_rem, h_remc = hi(B, T), hi(B), hi(B, T), hi(B)
+
+        def e2e_pipeline():
+            ada.ada_select_full_host(ctx, pin[0], cfg.tau, h_idx[0], h_cnt[0])
+            c = 0
+            for l in range(1, L):
+                ada.ada_cascade_step_host(ctx, pin[l], cfg.tau, h_idx[c], h_cnt[c], h_idx[1 - c],
+                                          h_cnt[1 - c], h_add, h_addc, h_rem, h_remc)
+                c = 1 - c
+
+        for _ in range(2):
+            e2e_pipeline()
+        barrier()
+        n_e2e = max(3, args.steps // 2)
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            e2e_pipeline()
+        torch.cuda.synchronize()
+        t_e2e = (time.perf_counter() - t0) / n_e2e
+        if world > 1:
+            t = torch.tensor([t_e2e], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            t_e2e = float(t.item())
+        n_tok = B * T
+        h2d = L * n_tok * d * es + (L - 1) * (n_tok * 4 + B * 4)
+        d2h = (n_tok * 4 + B * 4) + (L - 1) * 3 * (n_tok * 4 + B * 4)
+        e2e = {"value": world * B * T * L / t_e2e, "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": 1e3 * t_e2e,
+               "api": "ada_select_full_host + ada_cascade_step_host, pinned host tensors"}
+
+    # ---- the oracle on this machine's host cores (rank 0, N = 1 only), bounded sample ----
+    cpu_baseline, parity_sample = None, None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        n_lay = min(L, args.ref_layers)
+        t_c, band, mism = [], 0, 0
+        t0 = time.perf_counter()
+        R = [oracle.select_full(wl.as_f64(host_layers[0][b]), cfg.tau)[0] for b in range(B)]
+        t_full = time.perf_counter() - t0
+        for l in range(n_lay):
+            if l > 0:
+                t1 = time.perf_counter()
+                R = [oracle.cascade_step(wl.as_f64(host_layers[l][b]), cfg.tau, R[b]).rep
+                     for b in range(B)]
+                t_c.append(time.perf_counter() - t1)
+            mism += sum(R[b].tolist() != casc_sets[l][b].tolist() for b in range(B))
+        t_est = t_full + (L - 1) * (float(np.mean(t_c)) if t_c else t_full)
+        cpu_baseline = {"value": B * T * L / t_est, "unit": UNIT, "cores": oracle.num_threads(),
+                        "kind": "oracle",
+                        "sample": f"layers 0..{n_lay - 1} computed in full (fp64); step time = "
+                                  f"t(full, layer 0) + {L - 1} x mean t(cascade step)",
+                        "t_full_s": t_full, "t_cascade_step_s": float(np.mean(t_c)) if t_c else None}
+        parity_sample = {"layers_checked": n_lay, "set_mismatches": mism}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16 x bf16 -> f32" if cfg.dtype == "bf16" else "f32",
+            "data": "synthetic", "config": workload_dict(cfg), "clocks": clocks, "e2e": e2e,
+            "gpu_launches": args.steps * (3 + 5 * (L - 1)),
+            "roofline": roofline, "cpu_baseline": cpu_baseline,
+            "independent": {"value": world * B * T * L / (ms_indep * 1e-3), "unit": UNIT,
+                            "ms_per_step": ms_indep},
+            "cascade_speedup": ms_indep / ms_step,
+            "kernels": kernels,
+            "algorithmic_gflop_per_step": {k: v / 1e9 for k, v in flops.items()},
+            "gram_ops": {"independent": ops_indep, "cascade": ops_casc,
+                         "saved_frac": 1.0 - ops_casc / ops_indep},
+            "sets": {"r_layer0": [int(x) for x in hist[0, 0]], "r_last": [int(x) for x in hist[-1, 0]],
+                     "jaccard_consecutive_independent_mean": float(np.mean(j_consec)) if j_consec else None,
+                     "jaccard_cascade_vs_full_mean": float(np.mean(j_cvf)),
+                     "jaccard_cascade_vs_full_last": j_cvf[-1]},
+            "parity_sample": parity_sample, "zero_norm_rows": n_zero,
+            "engine": "ffma" if args.engine == 1 else "auto",
+        }
+        print(json.dumps(line))
+    ada.ada_destroy(ctx)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
