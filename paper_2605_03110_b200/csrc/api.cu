@@ -131,6 +131,7 @@ ada_status ada_create(ada_ctx** out, int device, int64_t maxB, int64_t maxT, int
     ctx->es = dt == ADA_F32 ? 4 : 2;
     ctx->engine = ADA_ENGINE_AUTO;
     ctx->stage = nullptr; ctx->stage_bytes = 0; ctx->host_stream = nullptr;
+    ctx->tc_attr_set = false;
     cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
 
     const size_t n_tok = (size_t)maxB * (size_t)maxT;

@@ -80,6 +80,7 @@ struct ada_ctx {
     int es;
     ada_engine engine;
     int sm_count;
+    bool tc_attr_set;
     // device workspace
     char* ws;            // one allocation
     float* inv_norm;     // [maxB*maxT] 1/||x_t||
