@@ -289,7 +289,10 @@ def main():
     }
     peaks = measured_peaks()
     es = cfg.es
-    if "cross" in dom:
+    if "cascade" in dom:
+        alg, bound = flops["tri_rep"] + flops["cross"], "tensor"
+        per = "d*r*(r-1) + 2*d*(T-r)*r_valid flop per launch"
+    elif "cross" in dom:
         alg, bound, per = flops["cross"], "tensor", "2*d*(T-r)*r_valid flop per launch"
     elif "tri" in dom:
         alg, bound, per = flops["tri_full"] + flops["tri_rep"], "tensor", "d*n*(n-1) flop per launch"
@@ -405,7 +408,7 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16 x bf16 -> f32" if cfg.dtype == "bf16" else "f32",
             "data": "synthetic", "config": workload_dict(cfg), "clocks": clocks, "e2e": e2e,
-            "gpu_launches": args.steps * (3 + 5 * (L - 1)),
+            "gpu_launches": args.steps * sum(k["launches"] for k in kernels.values()),
             "roofline": roofline, "cpu_baseline": cpu_baseline,
             "independent": {"value": world * B * T * L / (ms_indep * 1e-3), "unit": UNIT,
                             "ms_per_step": ms_indep},

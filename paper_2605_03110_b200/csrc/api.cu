@@ -13,7 +13,8 @@ namespace {
 
 const char* const kKernelNames[K_COUNT] = {
     "scatter_roles",   "norm_gather",      "gram_ffma_tri",  "gram_ffma_cross",
-    "gram_tc_tri",     "gram_tc_cross",    "compact_full",   "compact_cascade",
+    "gram_tc_tri",     "gram_tc_cross",    "gram_tc_cascade", "compact_full",
+    "compact_cascade",
 };
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -53,7 +54,7 @@ bool use_tc(const ada_ctx* ctx, ada_dtype dt) {
 }
 
 cudaError_t run_gram(ada_ctx* ctx, const GramProblem& p, ada_dtype dt, cudaStream_t s) {
-    if (use_tc(ctx, dt)) return launch_gram_tc(ctx, p, s);
+    if (use_tc(ctx, dt)) return p.tri ? launch_gram_tc(ctx, &p, nullptr, s) : launch_gram_tc(ctx, nullptr, &p, s);
     return launch_gram_ffma(ctx, p, dt, s);
 }
 
@@ -139,8 +140,9 @@ ada_status ada_create(ada_ctx** out, int device, int64_t maxB, int64_t maxT, int
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
     // role, g_tok, g_rep are contiguous so that one memset clears them
     const size_t o_role = take(n_tok * 4), o_gtok = take(n_tok * 4), o_grep = take(n_tok * 4);
+    const size_t o_ctr = take(32);
     const size_t o_inv = take(n_tok * 4), o_invr = take(n_tok * 4);
-    const size_t o_reff = take((size_t)maxB * 4), o_stat = take(32), o_ctr = take(32);
+    const size_t o_reff = take((size_t)maxB * 4), o_stat = take(32);
     const size_t o_xrep = take(n_tok * (size_t)maxd * ctx->es + 1024);
     if (cudaMalloc(&ctx->ws, off) != cudaSuccess) {
         cudaGetLastError();
@@ -257,13 +259,12 @@ ada_status ada_cascade_step(ada_ctx* ctx, const void* X, int64_t B, int64_t T, i
     if (rep_out == rep_in || (flags & ~ADA_CROSS_CAUSAL) != 0) return ADA_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const size_t n_tok_cap = (size_t)ctx->maxB * ctx->maxT;
     const size_t n_tok = (size_t)B * T;
     const float thr = (float)(1.0 - tau * tau);
     (void)n_tok;
 
     // role, g_tok, g_rep are contiguous in the workspace: one memset clears all three
-    CU(cudaMemsetAsync(ctx->role, 0, (size_t)((char*)ctx->g_rep - (char*)ctx->role) + n_tok_cap * 4, s));
+    CU(cudaMemsetAsync(ctx->role, 0, (size_t)((char*)ctx->tile_ctr - (char*)ctx->role) + 32, s));
     CU(launch_scatter(ctx, rep_in, rep_in_cnt, (int)B, (int)T, s));
     // lines 1-2: inverse norms of all rows; inherited rows gathered into Xrep
     CU(launch_norm_gather(ctx, X, (int)B, (int)T, (int)d, ldx, dt, ctx->inv_norm, nullptr,
@@ -279,7 +280,8 @@ ada_status ada_cascade_step(ada_ctx* ctx, const void* X, int64_t B, int64_t T, i
     p.n_dev = ctx->r_eff; p.n_host = 0;
     p.rows = (int)T; p.cap = (int)T; p.d = (int)d; p.B = (int)B;
     p.tri = 1;
-    CU(run_gram(ctx, p, dt, s));
+    const bool fuse = use_tc(ctx, dt);   // one launch: the cross epilogues wait for lines 3-5 in-kernel
+    if (!fuse) CU(run_gram(ctx, p, dt, s));
     // lines 6-8: cross-Gram of all rows against the valid inherited reps
     GramProblem q;
     memset(&q, 0, sizeof(q));
@@ -297,7 +299,8 @@ ada_status ada_cascade_step(ada_ctx* ctx, const void* X, int64_t B, int64_t T, i
     q.col_token = rep_in;
     q.row_role = ctx->role;
     q.causal = (flags & ADA_CROSS_CAUSAL) ? 1 : 0;
-    CU(run_gram(ctx, q, dt, s));
+    if (fuse) CU(launch_gram_tc(ctx, &p, &q, s));
+    else CU(run_gram(ctx, q, dt, s));
     // lines 5, 9, 10-11
     CU(launch_compact_cascade(ctx, (int)B, (int)T, thr, rep_in, rep_out, rep_out_cnt, add_idx,
                               add_cnt, rem_idx, rem_cnt, gamma_rep, gamma_cross, s));

@@ -25,6 +25,7 @@ enum KernelId {
     K_GRAM_FFMA_CROSS,
     K_GRAM_TC_TRI,
     K_GRAM_TC_CROSS,
+    K_GRAM_TC_CASCADE,
     K_COMPACT_FULL,
     K_COMPACT_CASCADE,
     K_COUNT
@@ -122,7 +123,8 @@ cudaError_t launch_compact_cascade(ada_ctx* ctx, int B, int T, float thr, const 
 cudaError_t launch_gram_ffma(ada_ctx* ctx, const GramProblem& p, ada_dtype dt, cudaStream_t s);
 
 // gram_tc.cu (bf16, tcgen05 + TMA)
-cudaError_t launch_gram_tc(ada_ctx* ctx, const GramProblem& p, cudaStream_t s);
+cudaError_t launch_gram_tc(ada_ctx* ctx, const GramProblem* tri, const GramProblem* cross,
+                           cudaStream_t s);
 bool gram_tc_available();
 
 }  // namespace ada

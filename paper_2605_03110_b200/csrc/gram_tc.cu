@@ -8,7 +8,7 @@
 //
 // One persistent CTA per SM, 192 threads:
 //   warp 0      TMA producer: one lane issues cp.async.bulk.tensor loads of a 128 x 64
-//               A box and a 256 x 64 B box per K block into a 4-stage ring
+//               A box and up to four 64 x 64 B boxes per K block into a 4-stage ring
 //               (128-byte swizzle, completion on an mbarrier)
 //   warp 1      MMA issuer: one lane issues four tcgen05.mma (M=128, N<=256, K=16) per
 //               K block; tcgen05.commit releases the ring stage, and after the last K
@@ -22,6 +22,7 @@
 // status, drains its own outstanding copies and MMAs (again bounded), frees its TMEM
 // and returns.
 #include <cuda.h>
+#include <string.h>
 
 #include "common.cuh"
 
@@ -36,10 +37,17 @@ constexpr int STAGES = 4;
 constexpr int UMMA_K = 16;
 constexpr int A_BYTES = BM * BK * 2;                 // 16 KiB
 constexpr int B_BYTES = BN * BK * 2;                 // 32 KiB
+constexpr int BOX_N = 64;                            // B rows per TMA box
+constexpr int BOX_BYTES = BOX_N * BK * 2;            // 8 KiB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int NUM_THREADS = 192;
 constexpr int TMEM_COLS = 512;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // 2 s
+
+// one output tile: `ncols` (multiple of 16, <= 256) columns from col0 of the 128-row tile at row0
+struct Piece {
+    int b, row0, col0, ncols, n, m;
+};
 
 struct alignas(16) Shared {
     unsigned long long full[STAGES];
@@ -49,6 +57,7 @@ struct alignas(16) Shared {
     unsigned long long drain;
     unsigned tmem_base;
     int abort_flag;
+    int tiles0, tiles1;
     // per epilogue warp, so that staging needs no barrier across warps
     alignas(16) float col_scale[4][BN];
     alignas(16) int col_token[4][BN];
@@ -168,60 +177,91 @@ __device__ __forceinline__ unsigned instr_desc(int n) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((unsigned)(n >> 3) << 17) | ((unsigned)(BM >> 4) << 24);
 }
 
-// ---------------------------------------------------------------- tile schedule
-struct Tile {
-    int b, row0, col0, n, m;
-};
-
-// Lower-triangular schedule for BN = 2*BM: row tiles 2p and 2p+1 both need p+1 column tiles.
+// ---------------------------------------------------------------- work schedule
+// A launch covers up to two problems ("segments"): a triangular one (Definition 1 on X, or
+// Algorithm 1 lines 3-4 on the gathered representatives) and a cross one (lines 7-8).
+// Their output tiles form one list, triangular tiles first, dealt round-robin to the
+// persistent CTAs.  When both are present the cross epilogues need line 5's verdict on
+// every column, i.e. the finished triangular segment: each epilogue warp bumps a global
+// counter after publishing a triangular tile's maxima, and a cross epilogue waits (bounded)
+// for the counter to reach 4 x (number of triangular tiles) before it stages its column
+// factors.  The cross MAIN LOOPS do not wait, so the short r x r problem hides behind them.
+// Triangular tiles precede cross tiles in every CTA's order and wait on nothing, and the
+// launch is cooperative (all CTAs co-resident), so the wait always ends.
+__device__ __forceinline__ int seq_n(const GramProblem& p, int b) {
+    return p.n_dev != nullptr ? p.n_dev[b] : p.n_host;
+}
+// lower-triangular tile count for BN = 2*BM: row tiles 2P and 2P+1 both need P+1 column tiles
 __device__ __forceinline__ int tri_tiles(int n) {
     const int M = (n + BM - 1) / BM, P = M >> 1;
     return P * (P + 1) + ((M & 1) ? P + 1 : 0);
 }
-__device__ __forceinline__ bool decode_tile(const GramProblem& p, int id, Tile& t) {
+// cross: columns are cut into nct equal tiles of width w (multiple of 16, <= 256)
+__device__ __forceinline__ void cross_cols(int n, int& nct, int& w) {
+    nct = (n + BN - 1) / BN;
+    w = nct > 0 ? ((((n + nct - 1) / nct) + 15) & ~15) : 0;
+}
+__device__ __forceinline__ int seg_tiles(const GramProblem& p) {
+    int total = 0;
     for (int b = 0; b < p.B; ++b) {
-        const int n = p.n_dev != nullptr ? p.n_dev[b] : p.n_host;
-        int cnt;
-        if (p.tri) cnt = tri_tiles(n);
-        else cnt = n > 0 ? ((p.rows + BM - 1) / BM) * ((n + BN - 1) / BN) : 0;
-        if (id < cnt) {
-            t.b = b;
-            t.n = n;
-            if (p.tri) {
-                int P = (int)((sqrtf(4.0f * (float)id + 1.0f) - 1.0f) * 0.5f);
-                while (P * (P + 1) > id) --P;
-                while ((P + 1) * (P + 2) <= id) ++P;
-                const int rem = id - P * (P + 1);
-                const int mi = rem < P + 1 ? 2 * P : 2 * P + 1;
-                const int nj = rem < P + 1 ? rem : rem - (P + 1);
-                t.row0 = mi * BM;
-                t.col0 = nj * BN;
-                t.m = n;
-            } else {
-                const int nct = (n + BN - 1) / BN;
-                t.row0 = (id / nct) * BM;
-                t.col0 = (id % nct) * BN;
-                t.m = p.rows;
-            }
-            return true;
+        const int n = seq_n(p, b);
+        if (n <= 0) continue;
+        if (p.tri) total += tri_tiles(n);
+        else {
+            int nct, w;
+            cross_cols(n, nct, w);
+            total += ((p.rows + BM - 1) / BM) * nct;
         }
-        id -= cnt;
+    }
+    return total;
+}
+// tile `id` of segment p -> piece; false when id is past the segment's last tile
+__device__ __forceinline__ bool decode_tile(const GramProblem& p, int id, Piece& t) {
+    for (int b = 0; b < p.B; ++b) {
+        const int n = seq_n(p, b);
+        if (n <= 0) continue;
+        int cnt, nct = 0, w = 0;
+        if (p.tri) cnt = tri_tiles(n);
+        else {
+            cross_cols(n, nct, w);
+            cnt = ((p.rows + BM - 1) / BM) * nct;
+        }
+        if (id >= cnt) { id -= cnt; continue; }
+        t.b = b;
+        t.n = n;
+        int nc;
+        if (p.tri) {
+            int P = (int)((sqrtf(4.0f * (float)id + 1.0f) - 1.0f) * 0.5f);
+            while (P * (P + 1) > id) --P;
+            while ((P + 1) * (P + 2) <= id) ++P;
+            const int rem = id - P * (P + 1);
+            const int mi = rem < P + 1 ? 2 * P : 2 * P + 1;
+            const int nj = rem < P + 1 ? rem : rem - (P + 1);
+            t.row0 = mi * BM;
+            t.col0 = nj * BN;
+            t.m = n;
+            nc = min(min(n - t.col0, t.row0 + BM - t.col0), BN);   // nothing right of the tile's last row
+        } else {
+            t.row0 = (id / nct) * BM;
+            t.col0 = (id % nct) * w;
+            t.m = p.rows;
+            nc = min(n - t.col0, w);
+        }
+        t.ncols = max(16, (nc + 15) & ~15);                        // MMA N: multiple of 16
+        return true;
     }
     return false;
 }
-// Columns the MMA must produce for a tile: up to the matrix edge, and for the triangular
-// problem up to the last row of the tile; a multiple of 16 in [16, 256].
-__device__ __forceinline__ int tile_ncols(const GramProblem& p, const Tile& t) {
-    int nc = t.n - t.col0;
-    if (p.tri) nc = min(nc, t.row0 + BM - t.col0);
-    nc = min(nc, BN);
-    return max(16, (nc + 15) & ~15);
-}
 
 // ---------------------------------------------------------------- the kernel
+struct GramMaps {
+    CUtensorMap a[2], b[2];       // per segment: left operand (128-row boxes), right operand (64-row boxes)
+};
+
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-k_gram_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-          const GramProblem p, unsigned* __restrict__ status) {
+k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramProblem seg0,
+          const __grid_constant__ GramProblem seg1, const int nseg, unsigned* __restrict__ dep_ctr,
+          unsigned* __restrict__ status) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -229,7 +269,6 @@ k_gram_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     volatile int* abort_flag = &sh.abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int num_kb = (p.d + BK - 1) / BK;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -245,6 +284,10 @@ k_gram_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    if (threadIdx.x == 64) {
+        sh.tiles0 = seg_tiles(seg0);
+        sh.tiles1 = nseg > 1 ? seg_tiles(seg1) : 0;
+    }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(&sh.tmem_base)), "r"(TMEM_COLS)
@@ -255,28 +298,36 @@ k_gram_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     __syncthreads();
     tcgen05_fence_after();
     const unsigned tmem_base = sh.tmem_base;
+    const int tiles0 = sh.tiles0, total = sh.tiles0 + sh.tiles1;
+    Piece pc;
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
         if (lane == 0) {
             unsigned it = 0;      // running K-block counter over all of this CTA's tiles
-            Tile t;
             bool ok = true;
-            for (int id = blockIdx.x; ok && decode_tile(p, id, t); id += gridDim.x) {
+            for (int id = blockIdx.x; ok && id < total; id += gridDim.x) {
+                const int sg = id < tiles0 ? 0 : 1;
+                const GramProblem& p = sg ? seg1 : seg0;
+                if (!decode_tile(p, id - (sg ? tiles0 : 0), pc)) break;
+                const int num_kb = (p.d + BK - 1) / BK;
+                const int nbox = (pc.ncols + BOX_N - 1) / BOX_N;
+                const unsigned bytes = A_BYTES + nbox * BOX_BYTES;
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
                     const int s = it % STAGES;
                     const unsigned ph = (it / STAGES) & 1u;
                     if (!mbar_wait(&sh.empty[s], ph ^ 1u, abort_flag, 1)) { ok = false; break; }
                     unsigned char* sa = smem + s * STAGE_BYTES;
-                    mbar_expect_tx(&sh.full[s], STAGE_BYTES);
-                    tma_load_3d(&map_a, &sh.full[s], sa, kb * BK, t.row0, t.b);
-                    tma_load_3d(&map_b, &sh.full[s], sa + A_BYTES, kb * BK, t.col0, t.b);
+                    mbar_expect_tx(&sh.full[s], bytes);
+                    tma_load_3d(&maps.a[sg], &sh.full[s], sa, kb * BK, pc.row0, pc.b);
+                    for (int j = 0; j < nbox; ++j)
+                        tma_load_3d(&maps.b[sg], &sh.full[s], sa + A_BYTES + j * BOX_BYTES, kb * BK,
+                                    pc.col0 + j * BOX_N, pc.b);
                 }
             }
             // drain: every copy this lane issued must have landed before the CTA may exit
             const unsigned issued = it;
             for (int s = 0; s < STAGES; ++s) {
-                // number of fills issued to stage s
                 const unsigned fills = issued / STAGES + ((issued % STAGES) > (unsigned)s ? 1u : 0u);
                 if (fills == 0) continue;
                 const unsigned ph = (fills - 1) & 1u;
@@ -290,13 +341,16 @@ k_gram_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         // ------------------------------------------------ MMA issuer
         if (lane == 0) {
             unsigned it = 0, tile_it = 0;
-            Tile t;
             bool ok = true;
-            for (int id = blockIdx.x; ok && decode_tile(p, id, t); id += gridDim.x, ++tile_it) {
+            for (int id = blockIdx.x; ok && id < total; id += gridDim.x, ++tile_it) {
+                const int sg = id < tiles0 ? 0 : 1;
+                const GramProblem& p = sg ? seg1 : seg0;
+                if (!decode_tile(p, id - (sg ? tiles0 : 0), pc)) break;
+                const int num_kb = (p.d + BK - 1) / BK;
                 const unsigned acc = tile_it & 1u, acc_ph = (tile_it >> 1) & 1u;
                 if (!mbar_wait(&sh.tmem_empty[acc], acc_ph ^ 1u, abort_flag, 2)) { ok = false; break; }
                 tcgen05_fence_after();
-                const unsigned idesc = instr_desc(tile_ncols(p, t));
+                const unsigned idesc = instr_desc(pc.ncols);
                 const unsigned d_tmem = tmem_base + acc * BN;
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
                     const int s = it % STAGES;
@@ -327,23 +381,46 @@ k_gram_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         const int quad = warp & 3;                    // TMEM lane quadrant this warp may read
         float* cs = sh.col_scale[warp - 2];
         int* ct = sh.col_token[warp - 2];
+        const unsigned dep_total = 4u * (unsigned)tiles0;
+        bool dep_ok = !(nseg > 1 && tiles0 > 0);      // cross epilogues must see segment 0 finished
         unsigned tile_it = 0;
-        Tile t;
-        for (int id = blockIdx.x; decode_tile(p, id, t); id += gridDim.x, ++tile_it) {
+        for (int id = blockIdx.x; id < total; id += gridDim.x, ++tile_it) {
+            const int sg = id < tiles0 ? 0 : 1;
+            const GramProblem& p = sg ? seg1 : seg0;
+            if (!decode_tile(p, id - (sg ? tiles0 : 0), pc)) break;
             const unsigned acc = tile_it & 1u, acc_ph = (tile_it >> 1) & 1u;
-            const int64_t o = (int64_t)t.b * p.cap;
-            const int ncols = tile_ncols(p, t);
+            const int64_t o = (int64_t)pc.b * p.cap;
+            const int ncols = pc.ncols;
             const int ncols32 = (ncols + 31) & ~31;   // TMEM is read 32 columns at a time
+            if (sg == 1 && !dep_ok) {
+                // bounded wait for every triangular tile of this launch (line 5 before line 7)
+                int good = 1;
+                if (lane == 0) {
+                    const unsigned long long t0 = global_ns();
+                    unsigned seen;
+                    while (true) {
+                        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(dep_ctr) : "memory");
+                        if (seen >= dep_total) break;
+                        if (*abort_flag != 0) { good = 0; break; }
+                        if (global_ns() - t0 > WAIT_LIMIT_NS) { *abort_flag = 5; good = 0; break; }
+                        __nanosleep(64);
+                    }
+                }
+                good = __shfl_sync(0xffffffffu, good, 0);
+                if (!good) break;
+                dep_ok = true;
+            }
             // stage this tile's column factors (0 for inadmissible columns); warp-private copy
             __syncwarp();
             for (int c = lane; c < ncols32; c += 32) {
-                const int col = t.col0 + c;
+                const int col = pc.col0 + c;
                 float f = 0.f;
                 int tok = col;
-                if (c < ncols && col < t.n) {
+                if (c < ncols && col < pc.n) {
                     f = p.inv_b[o + col];
                     if (!p.tri) {
-                        if (!(p.col_gate[o + col] < p.thr_bits)) f = 0.f;   // representative removed at line 5
+                        // representative removed at line 5 (written earlier in this launch: read at L2)
+                        if (!(__ldcg(p.col_gate + o + col) < p.thr_bits)) f = 0.f;
                         if (p.causal) tok = p.col_token[o + col];
                     }
                 }
@@ -355,8 +432,8 @@ k_gram_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
             const bool got = mbar_wait(&sh.tmem_full[acc], acc_ph, abort_flag, 4);
             if (!__all_sync(0xffffffffu, got)) break;
             tcgen05_fence_after();
-            const int row = t.row0 + quad * 32 + lane;
-            const bool need_cmp = p.tri ? (t.col0 + ncols > t.row0) : (p.causal != 0);
+            const int row = pc.row0 + quad * 32 + lane;
+            const bool need_cmp = p.tri ? (pc.col0 + ncols > pc.row0) : (p.causal != 0);
             float mx = 0.f;
             for (int c0 = 0; c0 < ncols32; c0 += 32) {
                 float v[32];
@@ -382,12 +459,18 @@ k_gram_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
             tcgen05_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh.tmem_empty[acc]);
-            if (row < t.m) {
+            if (row < pc.m) {
                 const bool skip = !p.tri && p.row_role[o + row] != 0;   // inherited reps are not candidates
                 if (!skip) {
                     mx *= p.inv_a[o + row];
                     if (mx > 0.f) atomicMax(p.out + o + row, __float_as_uint(mx));
                 }
+            }
+            if (sg == 0 && nseg > 1) {
+                // publish: this warp's share of a triangular tile is in global memory
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) atomicAdd(dep_ctr, 1u);
             }
         }
     }
@@ -447,25 +530,53 @@ bool make_map(CUtensorMap* map, const void* base, int d, int rows, int B, int64_
 
 bool gram_tc_available() { return encode_fn() != nullptr; }
 
-cudaError_t launch_gram_tc(ada_ctx* ctx, const GramProblem& p, cudaStream_t s) {
+// tri and/or cross may be NULL.  With both, the cross epilogues wait inside the kernel for the
+// triangular segment (ctx->tile_ctr must be zero at launch) and the launch is cooperative.
+cudaError_t launch_gram_tc(ada_ctx* ctx, const GramProblem* tri, const GramProblem* cross,
+                           cudaStream_t s) {
     if (!ctx->tc_attr_set) {
         cudaError_t e = cudaFuncSetAttribute(k_gram_tc, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              SMEM_BYTES);
         if (e != cudaSuccess) return e;
         ctx->tc_attr_set = true;
     }
-    const int n_cap = p.n_dev != nullptr ? p.cap : p.n_host;
-    const int a_rows = p.tri ? n_cap : p.rows;
-    if (n_cap <= 0 || a_rows <= 0) return cudaSuccess;
-    CUtensorMap map_a, map_b;
-    // rows beyond the matrices (and k beyond d) are zero-filled by the TMA unit
-    if (!make_map(&map_a, p.A, p.d, p.tri ? p.cap : p.rows, p.B, p.lda, p.a_batch, BM) ||
-        !make_map(&map_b, p.Bm, p.d, p.cap, p.B, p.ldb, p.b_batch, BN))
-        return cudaErrorInvalidValue;
-    prof_begin(ctx, p.tri ? K_GRAM_TC_TRI : K_GRAM_TC_CROSS, s);
-    k_gram_tc<<<ctx->sm_count, NUM_THREADS, SMEM_BYTES, s>>>(map_a, map_b, p, ctx->status);
+    GramMaps maps;
+    memset(&maps, 0, sizeof(maps));
+    GramProblem segs[2];
+    memset(segs, 0, sizeof(segs));
+    int nseg = 0;
+    const GramProblem* in[2] = {tri, cross};
+    for (int i = 0; i < 2; ++i) {
+        const GramProblem* p = in[i];
+        if (p == nullptr) continue;
+        const int n_cap = p->n_dev != nullptr ? p->cap : p->n_host;
+        const int a_rows = p->tri ? n_cap : p->rows;
+        if (n_cap <= 0 || a_rows <= 0) continue;
+        // rows beyond the matrices (and k beyond d) are zero-filled by the TMA unit
+        if (!make_map(&maps.a[nseg], p->A, p->d, p->tri ? p->cap : p->rows, p->B, p->lda, p->a_batch, BM) ||
+            !make_map(&maps.b[nseg], p->Bm, p->d, p->cap, p->B, p->ldb, p->b_batch, BOX_N))
+            return cudaErrorInvalidValue;
+        segs[nseg++] = *p;
+    }
+    if (nseg == 0) return cudaSuccess;
+    if (nseg == 1) { maps.a[1] = maps.a[0]; maps.b[1] = maps.b[0]; segs[1] = segs[0]; segs[1].B = 0; }
+    const bool fused = nseg == 2;
+    prof_begin(ctx, fused ? K_GRAM_TC_CASCADE : (segs[0].tri ? K_GRAM_TC_TRI : K_GRAM_TC_CROSS), s);
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(ctx->sm_count);
+    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = fused ? 1 : 0;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, k_gram_tc, maps, segs[0], segs[1], nseg, ctx->tile_ctr,
+                                       ctx->status);
     prof_end(ctx, s);
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace ada
