@@ -12,7 +12,7 @@ using namespace ada;
 namespace {
 
 const char* const kKernelNames[K_COUNT] = {
-    "scatter_roles",   "norm_gather",      "gram_ffma_tri",  "gram_ffma_cross",
+    "norm_gather",     "gram_ffma_tri",    "gram_ffma_cross",
     "gram_tc_tri",     "gram_tc_cross",    "gram_tc_cascade", "compact_full",
     "compact_cascade",
 };
@@ -205,13 +205,9 @@ ada_status ada_normalize(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int6
         return ADA_ERR_UNSUPPORTED;
     DeviceGuard guard(ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const size_t n_tok = (size_t)B * T;
-    if (gather) {
-        CU(cudaMemsetAsync(ctx->role, 0, n_tok * 4, s));
-        CU(launch_scatter(ctx, rep_idx, rep_cnt, (int)B, (int)T, s));
-    }
     CU(launch_norm_gather(ctx, X, (int)B, (int)T, (int)d, ldx, dt, inv_norm, Xhat,
-                          gather ? ctx->role : nullptr, Xrep, ctx->inv_rep, s));
+                          gather ? rep_idx : nullptr, rep_cnt, nullptr, nullptr, Xrep, ctx->inv_rep,
+                          s));
     return ADA_OK;
 }
 
@@ -223,12 +219,11 @@ ada_status ada_select_full(ada_ctx* ctx, const void* X, int64_t B, int64_t T, in
     if (rep_idx == nullptr || rep_cnt == nullptr || !tau_ok(tau)) return ADA_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const size_t n_tok = (size_t)B * T;
     const float thr = (float)(1.0 - tau * tau);
 
-    CU(cudaMemsetAsync(ctx->g_tok, 0, n_tok * 4, s));
+    // the gamma scratch is zero on entry (workspace invariant kept by the compaction kernels)
     CU(launch_norm_gather(ctx, X, (int)B, (int)T, (int)d, ldx, dt, ctx->inv_norm, nullptr,
-                          nullptr, nullptr, nullptr, s));
+                          nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, s));
     GramProblem p;
     memset(&p, 0, sizeof(p));
     p.A = X; p.Bm = X;
@@ -259,16 +254,14 @@ ada_status ada_cascade_step(ada_ctx* ctx, const void* X, int64_t B, int64_t T, i
     if (rep_out == rep_in || (flags & ~ADA_CROSS_CAUSAL) != 0) return ADA_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const size_t n_tok = (size_t)B * T;
     const float thr = (float)(1.0 - tau * tau);
-    (void)n_tok;
 
-    // role, g_tok, g_rep are contiguous in the workspace: one memset clears all three
-    CU(cudaMemsetAsync(ctx->role, 0, (size_t)((char*)ctx->tile_ctr - (char*)ctx->role) + 32, s));
-    CU(launch_scatter(ctx, rep_in, rep_in_cnt, (int)B, (int)T, s));
-    // lines 1-2: inverse norms of all rows; inherited rows gathered into Xrep
-    CU(launch_norm_gather(ctx, X, (int)B, (int)T, (int)d, ldx, dt, ctx->inv_norm, nullptr,
-                          ctx->role, ctx->Xrep, ctx->inv_rep, s));
+    // role map, gamma scratch and dependency counter are zero on entry (workspace invariant
+    // kept by the compaction kernels).
+    // lines 1-2: inverse norms of all rows; inherited list validated, scattered into the role
+    // map and its rows gathered into Xrep
+    CU(launch_norm_gather(ctx, X, (int)B, (int)T, (int)d, ldx, dt, ctx->inv_norm, nullptr, rep_in,
+                          rep_in_cnt, ctx->role, ctx->r_eff, ctx->Xrep, ctx->inv_rep, s));
     // lines 3-4: r x r Gram among inherited reps, max over earlier ones
     GramProblem p;
     memset(&p, 0, sizeof(p));
@@ -302,8 +295,8 @@ ada_status ada_cascade_step(ada_ctx* ctx, const void* X, int64_t B, int64_t T, i
     if (fuse) CU(launch_gram_tc(ctx, &p, &q, s));
     else CU(run_gram(ctx, q, dt, s));
     // lines 5, 9, 10-11
-    CU(launch_compact_cascade(ctx, (int)B, (int)T, thr, rep_in, rep_out, rep_out_cnt, add_idx,
-                              add_cnt, rem_idx, rem_cnt, gamma_rep, gamma_cross, s));
+    CU(launch_compact_cascade(ctx, (int)B, (int)T, thr, rep_out, rep_out_cnt, add_idx, add_cnt,
+                              rem_idx, rem_cnt, gamma_rep, gamma_cross, s));
     return ADA_OK;
 }
 
@@ -316,6 +309,11 @@ ada_status ada_device_status(ada_ctx* ctx, void* stream, int64_t* n_zero_norm_ro
     CU(cudaMemsetAsync(ctx->status, 0, sizeof(h), s));
     CU(cudaStreamSynchronize(s));
     if (n_zero_norm_rows != nullptr) *n_zero_norm_rows = (int64_t)h[1];
+    if (h[0] != 0) {
+        // a faulted call may have left scratch behind: restore the all-zero workspace invariant
+        CU(cudaMemsetAsync(ctx->role, 0, (size_t)((char*)ctx->tile_ctr - (char*)ctx->role) + 32, s));
+        CU(cudaStreamSynchronize(s));
+    }
     if (h[0] & ST_TIMEOUT) return ADA_ERR_TIMEOUT;
     if (h[0] & (ST_BAD_INDEX | ST_BAD_COUNT)) return ADA_ERR_BAD_INDEX_SET;
     if (h[0] & ST_NONFINITE) return ADA_ERR_NONFINITE;

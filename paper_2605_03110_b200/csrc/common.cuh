@@ -19,8 +19,7 @@ enum : unsigned {
 // status[1] counts zero-norm rows, status[2] records where a wait gave up.
 
 enum KernelId {
-    K_SCATTER = 0,
-    K_NORM_GATHER,
+    K_NORM_GATHER = 0,
     K_GRAM_FFMA_TRI,
     K_GRAM_FFMA_CROSS,
     K_GRAM_TC_TRI,
@@ -107,17 +106,16 @@ void prof_begin(ada_ctx* ctx, int kid, cudaStream_t s);
 void prof_end(ada_ctx* ctx, cudaStream_t s);
 
 // prep_kernels.cu
-cudaError_t launch_scatter(ada_ctx* ctx, const int32_t* rep_in, const int32_t* rep_in_cnt, int B,
-                           int T, cudaStream_t s);
 cudaError_t launch_norm_gather(ada_ctx* ctx, const void* X, int B, int T, int d, int64_t ldx,
-                               ada_dtype dt, float* inv_norm, void* Xhat, const int32_t* role,
-                               void* Xrep, float* inv_rep, cudaStream_t s);
+                               ada_dtype dt, float* inv_norm, void* Xhat, const int32_t* rep_in,
+                               const int32_t* rep_in_cnt, int32_t* role, int32_t* r_eff, void* Xrep,
+                               float* inv_rep, cudaStream_t s);
 cudaError_t launch_compact_full(ada_ctx* ctx, int B, int T, float thr, int32_t* rep_idx,
                                 int32_t* rep_cnt, float* gamma, cudaStream_t s);
-cudaError_t launch_compact_cascade(ada_ctx* ctx, int B, int T, float thr, const int32_t* rep_in,
-                                   int32_t* rep_out, int32_t* rep_out_cnt, int32_t* add_idx,
-                                   int32_t* add_cnt, int32_t* rem_idx, int32_t* rem_cnt,
-                                   float* gamma_rep, float* gamma_cross, cudaStream_t s);
+cudaError_t launch_compact_cascade(ada_ctx* ctx, int B, int T, float thr, int32_t* rep_out,
+                                   int32_t* rep_out_cnt, int32_t* add_idx, int32_t* add_cnt,
+                                   int32_t* rem_idx, int32_t* rem_cnt, float* gamma_rep,
+                                   float* gamma_cross, cudaStream_t s);
 
 // gram_ffma.cu
 cudaError_t launch_gram_ffma(ada_ctx* ctx, const GramProblem& p, ada_dtype dt, cudaStream_t s);
