@@ -261,25 +261,34 @@ k_compact_cascade(unsigned* __restrict__ g_tok, unsigned* __restrict__ g_rep,
     __shared__ unsigned long long s_warp[33];
     const int b = blockIdx.x;
     const int64_t o = (int64_t)b * T;
+    const unsigned faulted = status[0];
     int base_keep = 0, base_add = 0, base_rem = 0;
     for (int t0 = 0; t0 < T; t0 += CHUNK) {
         const int first = t0 + threadIdx.x * CPT;
         unsigned keep = 0, add = 0, rem = 0;
         int pos[CPT];
+        unsigned gt[CPT], gp[CPT];
+        // independent loads first, the position-indexed gather second: two round trips in all
 #pragma unroll
-        for (int k = 0; k < CPT; ++k) pos[k] = (first + k < T) ? role[o + first + k] : 0;
+        for (int k = 0; k < CPT; ++k) {
+            const bool in = first + k < T;
+            pos[k] = in ? role[o + first + k] : 0;
+            gt[k] = in ? g_tok[o + first + k] : 0u;
+        }
+#pragma unroll
+        for (int k = 0; k < CPT; ++k) gp[k] = pos[k] > 0 ? g_rep[o + pos[k] - 1] : 0u;
 #pragma unroll
         for (int k = 0; k < CPT; ++k) {
             const int t = first + k;
             if (t >= T) continue;
             float gr = 0.f, gc = 0.f;
             if (pos[k] > 0) {       // inherited representative: line 5
-                gr = __uint_as_float(g_rep[o + pos[k] - 1]);
+                gr = __uint_as_float(gp[k]);
                 g_rep[o + pos[k] - 1] = 0u;
                 role[o + t] = 0;
                 if (gr < thr) keep |= 1u << k; else rem |= 1u << k;
             } else {                // line 9
-                gc = __uint_as_float(g_tok[o + t]);
+                gc = __uint_as_float(gt[k]);
                 if (gc < thr) { add |= 1u << k; keep |= 1u << k; }
             }
             g_tok[o + t] = 0u;      // rows of inherited reps are never written, clearing is harmless
@@ -306,7 +315,7 @@ k_compact_cascade(unsigned* __restrict__ g_tok, unsigned* __restrict__ g_rep,
         base_add += (int)((total >> 21) & 0x1FFFFFu);
         base_rem += (int)((total >> 42) & 0x1FFFFFu);
     }
-    if (status[0] != 0u) {
+    if (faulted != 0u) {
         // a rejected inherited list leaves positions without a token: clear them all
         for (int i = threadIdx.x; i < T; i += blockDim.x) g_rep[o + i] = 0u;
     }
