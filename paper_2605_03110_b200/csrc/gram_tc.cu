@@ -8,8 +8,9 @@
 //
 // One persistent CTA per SM, 192 threads:
 //   warp 0      TMA producer: one lane issues cp.async.bulk.tensor loads of a 128 x 64
-//               A box and up to four 64 x 64 B boxes per K block into a 4-stage ring
-//               (128-byte swizzle, completion on an mbarrier)
+//               A box and up to four 64 x 64 B boxes per K block into a ring of 4 to 9
+//               stages (fewer bytes per stage for narrow tiles, hence more K blocks in
+//               flight; 128-byte swizzle, completion on an mbarrier)
 //   warp 1      MMA issuer: one lane issues four tcgen05.mma (M=128, N<=256, K=16) per
 //               K block; tcgen05.commit releases the ring stage, and after the last K
 //               block hands the accumulator to the epilogue.  Owns the TMEM allocation
@@ -33,13 +34,12 @@ namespace {
 constexpr int BM = 128;          // accumulator rows per tile (TMEM lanes)
 constexpr int BN = 256;          // accumulator columns per tile
 constexpr int BK = 64;           // bf16 elements per K block = one 128-byte swizzle row
-constexpr int STAGES = 4;
+constexpr int MAX_STAGES = 9;
+constexpr int RING_BYTES = 216 * 1024;               // TMA ring: 4 stages of a 256-wide tile ... 9 of a 64-wide one
 constexpr int UMMA_K = 16;
 constexpr int A_BYTES = BM * BK * 2;                 // 16 KiB
-constexpr int B_BYTES = BN * BK * 2;                 // 32 KiB
 constexpr int BOX_N = 64;                            // B rows per TMA box
 constexpr int BOX_BYTES = BOX_N * BK * 2;            // 8 KiB
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int NUM_THREADS = 192;
 constexpr int TMEM_COLS = 512;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // 2 s
@@ -50,19 +50,20 @@ struct Piece {
 };
 
 struct alignas(16) Shared {
-    unsigned long long full[STAGES];
-    unsigned long long empty[STAGES];
+    unsigned long long full[MAX_STAGES];
+    unsigned long long empty[MAX_STAGES];
     unsigned long long tmem_full[2];
     unsigned long long tmem_empty[2];
     unsigned long long drain;
     unsigned tmem_base;
     int abort_flag;
-    int tiles0, tiles1;
+    int tiles0, tiles1, tw0;
     // per epilogue warp, so that staging needs no barrier across warps
     alignas(16) float col_scale[4][BN];
     alignas(16) int col_token[4][BN];
 };
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + (int)sizeof(Shared) + 1024;   // +1024: alignment slack
+constexpr int SMEM_BYTES = RING_BYTES + (int)sizeof(Shared) + 1024;   // +1024: alignment slack
+static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 
 // ---------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ unsigned smem_u32(const void* p) {
@@ -96,19 +97,24 @@ __device__ __forceinline__ unsigned long long global_ns() {
     return t;
 }
 // Bounded wait.  Returns false when the CTA is aborting (this or another wait ran out).
+// try_wait itself suspends the thread for a while before it reports failure, so the wall
+// clock (a slow special register) is consulted only once per 256 failed polls.
 __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity,
                                           volatile int* abort_flag, int where) {
-    if (mbar_try(bar, parity)) return true;
-    const unsigned long long t0 = global_ns();
     unsigned polls = 0;
-    while (true) {
-        if (mbar_try(bar, parity)) return true;
-        if (*abort_flag != 0) return false;
-        if ((++polls & 63u) == 0 && global_ns() - t0 > WAIT_LIMIT_NS) {
-            *abort_flag = where;
-            return false;
+    unsigned long long t0 = 0;
+    while (!mbar_try(bar, parity)) {
+        if ((++polls & 255u) == 0) {
+            if (*abort_flag != 0) return false;
+            const unsigned long long now = global_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > WAIT_LIMIT_NS) {
+                *abort_flag = where;
+                return false;
+            }
         }
     }
+    return true;
 }
 __device__ __forceinline__ void tma_load_3d(const CUtensorMap* map, unsigned long long* bar,
                                             void* dst, int c0, int c1, int c2) {
@@ -191,22 +197,34 @@ __device__ __forceinline__ unsigned instr_desc(int n) {
 __device__ __forceinline__ int seq_n(const GramProblem& p, int b) {
     return p.n_dev != nullptr ? p.n_dev[b] : p.n_host;
 }
-// lower-triangular tile count for BN = 2*BM: row tiles 2P and 2P+1 both need P+1 column tiles
-__device__ __forceinline__ int tri_tiles(int n) {
-    const int M = (n + BM - 1) / BM, P = M >> 1;
+// lower-triangular tile count for column tiles of width tw (128 or 256): the 128-row tile mi
+// needs the column tiles that start at or before its last row
+__device__ __forceinline__ int tri_tiles(int n, int tw) {
+    const int M = (n + BM - 1) / BM;
+    if (tw == BM) return M * (M + 1) / 2;
+    const int P = M >> 1;                                // row tiles 2P and 2P+1 both need P+1
     return P * (P + 1) + ((M & 1) ? P + 1 : 0);
+}
+// Stage geometry of the TMA ring for a tile of `ncols` columns: narrower tiles take fewer
+// bytes per K block, so more K blocks fit in flight and the loop stays ahead of the
+// load latency.
+__device__ __forceinline__ int stage_bytes(int ncols) {
+    return A_BYTES + ((ncols + BOX_N - 1) / BOX_N) * BOX_BYTES;
+}
+__device__ __forceinline__ int stage_count(int sbytes) {
+    return min(MAX_STAGES, RING_BYTES / sbytes);
 }
 // cross: columns are cut into nct equal tiles of width w (multiple of 16, <= 256)
 __device__ __forceinline__ void cross_cols(int n, int& nct, int& w) {
     nct = (n + BN - 1) / BN;
     w = nct > 0 ? ((((n + nct - 1) / nct) + 15) & ~15) : 0;
 }
-__device__ __forceinline__ int seg_tiles(const GramProblem& p) {
+__device__ __forceinline__ int seg_tiles(const GramProblem& p, int tw) {
     int total = 0;
     for (int b = 0; b < p.B; ++b) {
         const int n = seq_n(p, b);
         if (n <= 0) continue;
-        if (p.tri) total += tri_tiles(n);
+        if (p.tri) total += tri_tiles(n, tw);
         else {
             int nct, w;
             cross_cols(n, nct, w);
@@ -216,12 +234,12 @@ __device__ __forceinline__ int seg_tiles(const GramProblem& p) {
     return total;
 }
 // tile `id` of segment p -> piece; false when id is past the segment's last tile
-__device__ __forceinline__ bool decode_tile(const GramProblem& p, int id, Piece& t) {
+__device__ __forceinline__ bool decode_tile(const GramProblem& p, int tw, int id, Piece& t) {
     for (int b = 0; b < p.B; ++b) {
         const int n = seq_n(p, b);
         if (n <= 0) continue;
         int cnt, nct = 0, w = 0;
-        if (p.tri) cnt = tri_tiles(n);
+        if (p.tri) cnt = tri_tiles(n, tw);
         else {
             cross_cols(n, nct, w);
             cnt = ((p.rows + BM - 1) / BM) * nct;
@@ -231,16 +249,24 @@ __device__ __forceinline__ bool decode_tile(const GramProblem& p, int id, Piece&
         t.n = n;
         int nc;
         if (p.tri) {
-            int P = (int)((sqrtf(4.0f * (float)id + 1.0f) - 1.0f) * 0.5f);
-            while (P * (P + 1) > id) --P;
-            while ((P + 1) * (P + 2) <= id) ++P;
-            const int rem = id - P * (P + 1);
-            const int mi = rem < P + 1 ? 2 * P : 2 * P + 1;
-            const int nj = rem < P + 1 ? rem : rem - (P + 1);
+            int mi, nj;
+            if (tw == BM) {                              // row tile mi holds tiles mi(mi+1)/2 ... + mi
+                mi = (int)((sqrtf(8.0f * (float)id + 1.0f) - 1.0f) * 0.5f);
+                while (mi * (mi + 1) / 2 > id) --mi;
+                while ((mi + 1) * (mi + 2) / 2 <= id) ++mi;
+                nj = id - mi * (mi + 1) / 2;
+            } else {
+                int P = (int)((sqrtf(4.0f * (float)id + 1.0f) - 1.0f) * 0.5f);
+                while (P * (P + 1) > id) --P;
+                while ((P + 1) * (P + 2) <= id) ++P;
+                const int rem = id - P * (P + 1);
+                mi = rem < P + 1 ? 2 * P : 2 * P + 1;
+                nj = rem < P + 1 ? rem : rem - (P + 1);
+            }
             t.row0 = mi * BM;
-            t.col0 = nj * BN;
+            t.col0 = nj * tw;
             t.m = n;
-            nc = min(min(n - t.col0, t.row0 + BM - t.col0), BN);   // nothing right of the tile's last row
+            nc = min(min(n - t.col0, t.row0 + BM - t.col0), tw);   // nothing right of the tile's last row
         } else {
             t.row0 = (id / nct) * BM;
             t.col0 = (id % nct) * w;
@@ -265,13 +291,13 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-    Shared& sh = *reinterpret_cast<Shared*>(smem + STAGES * STAGE_BYTES);
+    Shared& sh = *reinterpret_cast<Shared*>(smem + RING_BYTES);
     volatile int* abort_flag = &sh.abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) {
+        for (int s = 0; s < MAX_STAGES; ++s) {
             mbar_init(&sh.full[s], 1);
             mbar_init(&sh.empty[s], 1);
         }
@@ -285,8 +311,13 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (threadIdx.x == 64) {
-        sh.tiles0 = seg_tiles(seg0);
-        sh.tiles1 = nseg > 1 ? seg_tiles(seg1) : 0;
+        // a triangular problem too small to give every CTA a 256-wide tile is cut 128 wide
+        int tw = BN;
+        int t0 = seg_tiles(seg0, tw);
+        if (seg0.tri && t0 < (int)gridDim.x) { tw = BM; t0 = seg_tiles(seg0, tw); }
+        sh.tw0 = tw;
+        sh.tiles0 = t0;
+        sh.tiles1 = nseg > 1 ? seg_tiles(seg1, BN) : 0;
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -298,41 +329,50 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
     __syncthreads();
     tcgen05_fence_after();
     const unsigned tmem_base = sh.tmem_base;
-    const int tiles0 = sh.tiles0, total = sh.tiles0 + sh.tiles1;
+    const int tiles0 = sh.tiles0, total = sh.tiles0 + sh.tiles1, tw0 = sh.tw0;
     Piece pc;
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
         if (lane == 0) {
-            unsigned it = 0;      // running K-block counter over all of this CTA's tiles
+            unsigned fills = 0;      // bit s: parity of the number of fills of stage s
+            unsigned used = 0;       // stages filled under the current geometry
+            unsigned ever = 0;       // stages ever filled
+            int cur_sb = 0, cur_nst = 0, s = 0;
             bool ok = true;
             for (int id = blockIdx.x; ok && id < total; id += gridDim.x) {
                 const int sg = id < tiles0 ? 0 : 1;
                 const GramProblem& p = sg ? seg1 : seg0;
-                if (!decode_tile(p, id - (sg ? tiles0 : 0), pc)) break;
+                if (!decode_tile(p, tw0, id - (sg ? tiles0 : 0), pc)) break;
                 const int num_kb = (p.d + BK - 1) / BK;
                 const int nbox = (pc.ncols + BOX_N - 1) / BOX_N;
-                const unsigned bytes = A_BYTES + nbox * BOX_BYTES;
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                    const int s = it % STAGES;
-                    const unsigned ph = (it / STAGES) & 1u;
-                    if (!mbar_wait(&sh.empty[s], ph ^ 1u, abort_flag, 1)) { ok = false; break; }
-                    unsigned char* sa = smem + s * STAGE_BYTES;
-                    mbar_expect_tx(&sh.full[s], bytes);
+                const int sb = stage_bytes(pc.ncols);
+                if (sb != cur_sb) {
+                    // new stage geometry: every stage of the old one must have been released
+                    for (int q = 0; q < cur_nst && ok; ++q)
+                        if ((used >> q) & 1u)
+                            ok = mbar_wait(&sh.empty[q], ((fills >> q) & 1u) ^ 1u, abort_flag, 6);
+                    if (!ok) break;
+                    cur_sb = sb; cur_nst = stage_count(sb); s = 0; used = 0;
+                }
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(&sh.empty[s], ((fills >> s) & 1u) ^ 1u, abort_flag, 1)) { ok = false; break; }
+                    unsigned char* sa = smem + s * sb;
+                    mbar_expect_tx(&sh.full[s], (unsigned)sb);
                     tma_load_3d(&maps.a[sg], &sh.full[s], sa, kb * BK, pc.row0, pc.b);
                     for (int j = 0; j < nbox; ++j)
                         tma_load_3d(&maps.b[sg], &sh.full[s], sa + A_BYTES + j * BOX_BYTES, kb * BK,
                                     pc.col0 + j * BOX_N, pc.b);
+                    fills ^= 1u << s; used |= 1u << s; ever |= 1u << s;
+                    s = (s + 1 == cur_nst) ? 0 : s + 1;
                 }
             }
             // drain: every copy this lane issued must have landed before the CTA may exit
-            const unsigned issued = it;
-            for (int s = 0; s < STAGES; ++s) {
-                const unsigned fills = issued / STAGES + ((issued % STAGES) > (unsigned)s ? 1u : 0u);
-                if (fills == 0) continue;
-                const unsigned ph = (fills - 1) & 1u;
+            for (int q = 0; q < MAX_STAGES; ++q) {
+                if (!((ever >> q) & 1u)) continue;
+                const unsigned ph = ((fills >> q) & 1u) ^ 1u;      // parity of the last fill's phase
                 const unsigned long long t0 = global_ns();
-                while (!mbar_try(&sh.full[s], ph)) {
+                while (!mbar_try(&sh.full[q], ph)) {
                     if (global_ns() - t0 > WAIT_LIMIT_NS / 2) { *abort_flag = 7; break; }
                 }
             }
@@ -340,24 +380,25 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer
         if (lane == 0) {
-            unsigned it = 0, tile_it = 0;
+            unsigned uses = 0, tile_it = 0;   // bit s of `uses`: parity of the number of uses of stage s
+            int cur_sb = 0, cur_nst = 0, s = 0;
             bool ok = true;
             for (int id = blockIdx.x; ok && id < total; id += gridDim.x, ++tile_it) {
                 const int sg = id < tiles0 ? 0 : 1;
                 const GramProblem& p = sg ? seg1 : seg0;
-                if (!decode_tile(p, id - (sg ? tiles0 : 0), pc)) break;
+                if (!decode_tile(p, tw0, id - (sg ? tiles0 : 0), pc)) break;
                 const int num_kb = (p.d + BK - 1) / BK;
+                const int sb = stage_bytes(pc.ncols);
+                if (sb != cur_sb) { cur_sb = sb; cur_nst = stage_count(sb); s = 0; }
                 const unsigned acc = tile_it & 1u, acc_ph = (tile_it >> 1) & 1u;
                 if (!mbar_wait(&sh.tmem_empty[acc], acc_ph ^ 1u, abort_flag, 2)) { ok = false; break; }
                 tcgen05_fence_after();
                 const unsigned idesc = instr_desc(pc.ncols);
                 const unsigned d_tmem = tmem_base + acc * BN;
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                    const int s = it % STAGES;
-                    const unsigned ph = (it / STAGES) & 1u;
-                    if (!mbar_wait(&sh.full[s], ph, abort_flag, 3)) { ok = false; break; }
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(&sh.full[s], (uses >> s) & 1u, abort_flag, 3)) { ok = false; break; }
                     tcgen05_fence_after();
-                    const unsigned a_addr = smem_u32(smem + s * STAGE_BYTES);
+                    const unsigned a_addr = smem_u32(smem + s * sb);
                     const unsigned long long adesc = smem_desc_sw128(a_addr);
                     const unsigned long long bdesc = smem_desc_sw128(a_addr + A_BYTES);
 #pragma unroll
@@ -366,6 +407,8 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
                         umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
                     }
                     umma_commit(&sh.empty[s]);          // stage reusable once these MMAs retire
+                    uses ^= 1u << s;
+                    s = (s + 1 == cur_nst) ? 0 : s + 1;
                 }
                 if (ok) umma_commit(&sh.tmem_full[acc]);  // accumulator complete
             }
@@ -387,7 +430,7 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
         for (int id = blockIdx.x; id < total; id += gridDim.x, ++tile_it) {
             const int sg = id < tiles0 ? 0 : 1;
             const GramProblem& p = sg ? seg1 : seg0;
-            if (!decode_tile(p, id - (sg ? tiles0 : 0), pc)) break;
+            if (!decode_tile(p, tw0, id - (sg ? tiles0 : 0), pc)) break;
             const unsigned acc = tile_it & 1u, acc_ph = (tile_it >> 1) & 1u;
             const int64_t o = (int64_t)pc.b * p.cap;
             const int ncols = pc.ncols;
