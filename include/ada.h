@@ -139,6 +139,37 @@ ada_status ada_cascade_step_host(ada_ctx* ctx, const void* X, int64_t B, int64_t
                                  int32_t* rem_idx, int32_t* rem_cnt, float* gamma_rep,
                                  float* gamma_cross, uint32_t flags);
 
+/*
+ * Full selection for callers that cannot allocate device memory (the paper has no
+ * counterpart; this is a deployment variant of ada_select_full for ONE sequence).
+ *
+ * Who needs it: a process whose device memory was handed in full to its own pool at
+ * start-up, a latency-critical loop that cannot take the device-wide synchronisation an
+ * allocation implies, a plug-in whose host forbids allocator calls.  None of them can
+ * create an ada_ctx, because its workspace is one cudaMalloc.  This call takes no context
+ * and performs no cudaMalloc / cudaFree and calls no allocating library routine: its
+ * scratch (gamma bit patterns, inverse norms, a few status words; about 128 KiB) is a fixed
+ * array inside the library image, present on every GPU that loads the library until the
+ * process exits.
+ *
+ * Arguments as ada_select_full with B = 1: device pointers, X row-major T x d with row
+ * stride ldx, rep_idx capacity T, rep_cnt one int32, gamma optional (T floats); the work
+ * is enqueued on `stream` for the CURRENT device and the call does not synchronise.
+ *   - T above ADA_NOALLOC_MAX_T returns ADA_ERR_WORKSPACE and enqueues nothing.
+ *   - The first call on each device also performs a one-time set-up (it looks up the
+ *     scratch array's device address and the SM count); make that first call before any
+ *     stream capture begins.
+ *   - All calls on a device share the one scratch array, and it keeps the previous call's
+ *     contents; the call itself clears what must start at zero.  Two calls whose kernels
+ *     overlap on the GPU (different streams) race on it: keep them stream-ordered.
+ *   - Device-detected faults (NaN/Inf) cannot be read back through a context here; check
+ *     the inputs upstream if that matters.
+ */
+#define ADA_NOALLOC_MAX_T 16384
+ada_status ada_select_full_noalloc(const void* X, int64_t T, int64_t d, int64_t ldx,
+                                   ada_dtype dt, double tau, int32_t* rep_idx, int32_t* rep_cnt,
+                                   float* gamma, void* stream);
+
 /* Gram operation counts of Eq. (4)/(5), d included: cascade == 0 -> T^2 d;
  * cascade != 0 -> r^2 d + (T - r) r d with r the INHERITED count.  Pure host
  * arithmetic; returns 0 for negative arguments or r > T. */

@@ -25,7 +25,9 @@ SYMBOLS = [
     "ada_create", "ada_destroy", "ada_set_engine", "ada_normalize", "ada_select_full",
     "ada_cascade_step", "ada_select_full_host", "ada_cascade_step_host", "ada_gram_op_count",
     "ada_device_status", "ada_profile_enable", "ada_profile_read", "ada_status_string",
+    "ada_select_full_noalloc",
 ]
+ADA_NOALLOC_MAX_T = 16384
 
 _lib = None
 
@@ -58,6 +60,8 @@ def lib() -> C.CDLL:
         L.ada_cascade_step_host.argtypes = [vp, vp, i64, i64, i64, C.c_int, C.c_double,
                                             i32p, i32p, i32p, i32p, i32p, i32p, i32p, i32p, fp, fp,
                                             C.c_uint32]
+        L.ada_select_full_noalloc.argtypes = [vp, i64, i64, i64, C.c_int, C.c_double, i32p, i32p,
+                                              fp, vp]
         L.ada_gram_op_count.argtypes = [C.c_int, i64, i64, i64]
         L.ada_gram_op_count.restype = C.c_uint64
         L.ada_device_status.argtypes = [vp, vp, C.POINTER(i64)]
@@ -236,6 +240,28 @@ def ada_cascade_step_host(ctx: Context, X: torch.Tensor, tau: float, rep_in, rep
                                        rep_out_cnt.data_ptr(), add_idx.data_ptr(), add_cnt.data_ptr(),
                                        rem_idx.data_ptr(), rem_cnt.data_ptr(), _ptr(gamma_rep),
                                        _ptr(gamma_cross), flags), "ada_cascade_step_host")
+
+
+def ada_select_full_noalloc(X: torch.Tensor, tau: float, rep_idx: torch.Tensor,
+                            rep_cnt: torch.Tensor, gamma: Optional[torch.Tensor] = None,
+                            stream=None) -> None:
+    """Full selection of ONE sequence (T x d) with no context and no allocation inside the
+    library: the caller passes every buffer (rep_idx: T int32, rep_cnt: 1 int32, gamma:
+    optional T float32) and the library's scratch is a fixed device array, so this is the
+    call for code that may not allocate device memory.  T <= ADA_NOALLOC_MAX_T; calls on
+    one device must not overlap on the GPU (they share the scratch)."""
+    if X.dim() == 3 and X.shape[0] == 1:
+        X = X[0]
+    if X.dim() != 2 or X.stride(1) != 1:
+        raise ValueError("X must be T x d with unit inner stride")
+    T, d = X.shape
+    st = lib().ada_select_full_noalloc(X.data_ptr(), T, d, X.stride(0), dtype_of(X), float(tau),
+                                       rep_idx.data_ptr(), rep_cnt.data_ptr(), _ptr(gamma),
+                                       _stream(stream))
+    if st == 3:
+        raise AdaError(st, f"ada_select_full_noalloc: T={T} exceeds ADA_NOALLOC_MAX_T="
+                           f"{ADA_NOALLOC_MAX_T}")
+    _check(st, "ada_select_full_noalloc")
 
 
 def ada_profile_enable(ctx: Context, on: bool) -> None:
