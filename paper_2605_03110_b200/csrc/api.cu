@@ -141,6 +141,8 @@ ada_status ada_create(ada_ctx** out, int device, int64_t maxB, int64_t maxT, int
     // role, g_tok, g_rep are contiguous so that one memset clears them
     const size_t o_role = take(n_tok * 4), o_gtok = take(n_tok * 4), o_grep = take(n_tok * 4);
     const size_t o_ctr = take(32);
+    const int agg_stride = (int)((maxT + 1023) / 1024);
+    const size_t o_done = take(32), o_agg = take((size_t)maxB * agg_stride * 8);
     const size_t o_inv = take(n_tok * 4), o_invr = take(n_tok * 4);
     const size_t o_reff = take((size_t)maxB * 4), o_stat = take(32);
     const size_t o_xrep = take(n_tok * (size_t)maxd * ctx->es + 1024);
@@ -157,6 +159,9 @@ ada_status ada_create(ada_ctx** out, int device, int64_t maxB, int64_t maxT, int
     ctx->r_eff = reinterpret_cast<int32_t*>(ctx->ws + o_reff);
     ctx->status = reinterpret_cast<unsigned*>(ctx->ws + o_stat);
     ctx->tile_ctr = reinterpret_cast<unsigned*>(ctx->ws + o_ctr);
+    ctx->done_ctr = reinterpret_cast<unsigned*>(ctx->ws + o_done);
+    ctx->agg = reinterpret_cast<unsigned long long*>(ctx->ws + o_agg);
+    ctx->agg_stride = agg_stride;
     ctx->Xrep = ctx->ws + o_xrep;
     if (cudaMemset(ctx->ws, 0, o_xrep) != cudaSuccess) {
         cudaFree(ctx->ws);
@@ -311,7 +316,7 @@ ada_status ada_device_status(ada_ctx* ctx, void* stream, int64_t* n_zero_norm_ro
     if (n_zero_norm_rows != nullptr) *n_zero_norm_rows = (int64_t)h[1];
     if (h[0] != 0) {
         // a faulted call may have left scratch behind: restore the all-zero workspace invariant
-        CU(cudaMemsetAsync(ctx->role, 0, (size_t)((char*)ctx->tile_ctr - (char*)ctx->role) + 32, s));
+        CU(cudaMemsetAsync(ctx->role, 0, (size_t)((char*)ctx->inv_norm - (char*)ctx->role), s));
         CU(cudaStreamSynchronize(s));
     }
     if (h[0] & ST_TIMEOUT) return ADA_ERR_TIMEOUT;

@@ -90,7 +90,10 @@ struct ada_ctx {
     int32_t* role;       // [maxB*maxT] 0 = not inherited, p+1 = position p in the inherited list
     int32_t* r_eff;      // [maxB] sanitised inherited counts
     unsigned* status;    // [8]
-    unsigned* tile_ctr;  // [8] persistent-kernel tile counters
+    unsigned* tile_ctr;  // [8] dependency counter of the fused Gram launch
+    unsigned long long* agg;  // [maxB][agg_stride] block counts published by the compaction
+    unsigned* done_ctr;  // compaction blocks finished
+    int agg_stride;
     void* Xrep;          // [maxB*maxT*maxd] gathered representative rows (raw values)
     // staging for the *_host entry points (allocated on first use)
     char* stage;

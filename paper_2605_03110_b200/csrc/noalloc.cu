@@ -14,7 +14,8 @@ using namespace ada;
 
 namespace {
 
-// gamma bit patterns [ADA_NOALLOC_MAX_T] | inverse norms [ADA_NOALLOC_MAX_T] | status + counters
+// gamma bit patterns [ADA_NOALLOC_MAX_T] | inverse norms [ADA_NOALLOC_MAX_T] | status words,
+// counters and the compaction's 16 published block counts (256 bytes)
 constexpr size_t kGammaBytes = (size_t)ADA_NOALLOC_MAX_T * 4;
 constexpr size_t kInvBytes = (size_t)ADA_NOALLOC_MAX_T * 4;
 constexpr size_t kTailBytes = 256;
@@ -59,7 +60,10 @@ ada_status setup_device(int device, PerDevice** out) {
         c.g_tok = reinterpret_cast<unsigned*>(pd.scratch);
         c.inv_norm = reinterpret_cast<float*>(pd.scratch + kGammaBytes);
         c.status = reinterpret_cast<unsigned*>(pd.scratch + kGammaBytes + kInvBytes);
-        c.tile_ctr = c.status + 8;
+        c.tile_ctr = c.status + 8;                                           // +32 bytes
+        c.done_ctr = c.status + 16;                                          // +64 bytes
+        c.agg = reinterpret_cast<unsigned long long*>(c.status + 32);        // +128 bytes: 16 words
+        c.agg_stride = ADA_NOALLOC_MAX_T / 1024;
         c.g_rep = nullptr;
         c.inv_rep = nullptr;
         c.role = nullptr;

@@ -165,16 +165,32 @@ cudaError_t launch_norm_gather(ada_ctx* ctx, const void* X, int B, int T, int d,
 }
 
 // ---------------------------------------------------------------------------
-// Compaction.  One 1024-thread block per sequence.  Each thread owns 8 consecutive
-// tokens of an 8192-token chunk, so a chunk needs one block-wide prefix sum (warp
-// shuffles + 32 warp totals) and the lists come out ascending.  The three running
-// counts of the cascade update travel through the scan packed in one 64-bit word.
-// The kernels also restore the workspace invariant: the gamma scratch, the role map
-// and the dependency counter are zero again when they finish, so no memset is needed
-// between calls.
+// Compaction (Definition 1's threshold; Algorithm 1 lines 5, 9, 10-11 and the lists of
+// Eq. 6).  Every 1024-thread block owns 1024 consecutive tokens of one sequence, one token
+// per thread, so all loads are coalesced and the whole sequence is in flight at once.
+// A block reduces its own counts, publishes them (one 64-bit word: three 21-bit counts
+// and a READY bit), then sums the words of the blocks before it -- those never wait on
+// anything, so the look-back is one round trip -- and writes its slice of the ascending
+// lists.  The last block to finish clears the published words and the counters, and every
+// thread clears the scratch it read, so the workspace is all-zero again when the kernel
+// ends and no memset is needed between calls.
 // ---------------------------------------------------------------------------
-constexpr int CPT = 8;                       // tokens per thread per chunk
-constexpr int CHUNK = 1024 * CPT;
+constexpr unsigned long long AGG_READY = 1ull << 63;
+constexpr unsigned long long AGG_MASK = (1ull << 21) - 1;
+
+struct CompactArgs {
+    unsigned* g_tok;             // gamma (full) / gamma_cross by token, bit patterns
+    unsigned* g_rep;             // gamma_rep by position (cascade) or NULL
+    int32_t* role;               // 0 / position+1 (cascade) or NULL
+    unsigned long long* agg;     // [B][agg_stride] published block counts
+    unsigned* done_ctr;          // blocks finished
+    unsigned* dep_ctr;           // dependency counter of the fused Gram launch (cleared here)
+    unsigned* status;
+    int agg_stride, T;
+    float thr;
+    int32_t *keep_idx, *keep_cnt, *add_idx, *add_cnt, *rem_idx, *rem_cnt;
+    float *gamma_a, *gamma_b;    // full: gamma | cascade: gamma_rep, gamma_cross (optional)
+};
 
 __device__ __forceinline__ unsigned long long block_exclusive_scan(unsigned long long v,
                                                                    unsigned long long* s_warp,
@@ -202,141 +218,133 @@ __device__ __forceinline__ unsigned long long block_exclusive_scan(unsigned long
     __syncthreads();
     const unsigned long long off = s_warp[warp] + incl - v;
     total = s_warp[32];
-    __syncthreads();   // s_warp is reused by the next chunk
+    __syncthreads();   // s_warp is reused
     return off;
 }
 
-// Definition 1: R = { t : gamma_t < thr }.
-__global__ void __launch_bounds__(1024)
-k_compact_full(unsigned* __restrict__ g_tok, int T, float thr, int32_t* __restrict__ rep_idx,
-               int32_t* __restrict__ rep_cnt, float* __restrict__ gamma) {
+__global__ void __launch_bounds__(1024) k_compact(const CompactArgs a) {
     __shared__ unsigned long long s_warp[33];
-    const int b = blockIdx.x;
-    unsigned* g = g_tok + (int64_t)b * T;
-    int32_t* out = rep_idx + (int64_t)b * T;
-    float* go = gamma != nullptr ? gamma + (int64_t)b * T : nullptr;
-    int base = 0;
-    for (int t0 = 0; t0 < T; t0 += CHUNK) {
-        const int first = t0 + threadIdx.x * CPT;
-        float gv[CPT];
-        unsigned flags = 0;
-#pragma unroll
-        for (int k = 0; k < CPT; ++k) {
-            const int t = first + k;
-            gv[k] = 0.f;
-            if (t < T) {
-                gv[k] = __uint_as_float(g[t]);
-                g[t] = 0u;                                   // leave the scratch clean
-                if (gv[k] < thr) flags |= 1u << k;
-                if (go != nullptr) go[t] = gv[k];
+    const int b = blockIdx.y, blk = blockIdx.x, nblk = gridDim.x;
+    const int t = blk * 1024 + threadIdx.x;
+    const int64_t o = (int64_t)b * a.T;
+    const bool in = t < a.T;
+    const bool cascade = a.role != nullptr;
+    const unsigned faulted = a.status[0];
+
+    // independent loads first, the position-indexed gather second
+    const int pos = (cascade && in) ? a.role[o + t] : 0;
+    const unsigned gt = in ? a.g_tok[o + t] : 0u;
+    const unsigned gp = pos > 0 ? a.g_rep[o + pos - 1] : 0u;
+    bool keep = false, add = false, rem = false;
+    if (in) {
+        float ga = 0.f, gb = 0.f;
+        if (pos > 0) {                    // inherited representative: line 5
+            ga = __uint_as_float(gp);
+            keep = ga < a.thr;
+            rem = !keep;
+            a.g_rep[o + pos - 1] = 0u;
+            a.role[o + t] = 0;
+        } else {                          // Definition 1 / line 9
+            gb = __uint_as_float(gt);
+            keep = gb < a.thr;
+            add = cascade && keep;
+        }
+        a.g_tok[o + t] = 0u;
+        if (cascade) {
+            if (a.gamma_a != nullptr) a.gamma_a[o + t] = ga;
+            if (a.gamma_b != nullptr) a.gamma_b[o + t] = gb;
+            if (faulted != 0u) a.g_rep[o + t] = 0u;   // a rejected list leaves positions without a token
+        } else if (a.gamma_a != nullptr) {
+            a.gamma_a[o + t] = gb;
+        }
+    }
+    const unsigned long long mine = (keep ? 1ull : 0ull) | (add ? 1ull << 21 : 0ull) | (rem ? 1ull << 42 : 0ull);
+    unsigned long long total;
+    const unsigned long long off = block_exclusive_scan(mine, s_warp, total);
+
+    unsigned long long* agg = a.agg + (int64_t)b * a.agg_stride;
+    if (threadIdx.x == 0) atomicExch(agg + blk, total | AGG_READY);
+    // look-back over the blocks before this one (bounded spin; they wait on nothing)
+    unsigned long long before = 0;
+    for (int j = threadIdx.x; j < blk; j += 1024) {
+        unsigned long long v;
+        unsigned polls = 0;
+        long long t0 = 0;
+        while (true) {
+            v = *reinterpret_cast<volatile unsigned long long*>(agg + j);
+            if (v & AGG_READY) break;
+            if ((++polls & 1023u) == 0) {
+                const long long now = clock64();
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > 4000000000ll) { atomicOr(a.status, ST_TIMEOUT); v = 0; break; }
             }
         }
-        unsigned long long total;
-        int off = base + (int)block_exclusive_scan((unsigned long long)__popc(flags), s_warp, total);
-#pragma unroll
-        for (int k = 0; k < CPT; ++k)
-            if (flags & (1u << k)) out[off++] = first + k;
-        base += (int)total;
+        before += v & ~AGG_READY;
     }
-    if (threadIdx.x == 0) rep_cnt[b] = base;
+    unsigned long long base;
+    block_exclusive_scan(before, s_warp, base);
+
+    const int nk = (int)((base + off) & AGG_MASK);
+    const int na = (int)(((base + off) >> 21) & AGG_MASK);
+    const int nr = (int)(((base + off) >> 42) & AGG_MASK);
+    if (keep) a.keep_idx[o + nk] = t;
+    if (add) a.add_idx[o + na] = t;
+    if (rem) a.rem_idx[o + nr] = t;
+    if (blk == nblk - 1 && threadIdx.x == 0) {
+        const unsigned long long all = base + total;
+        a.keep_cnt[b] = (int)(all & AGG_MASK);
+        if (cascade) {
+            a.add_cnt[b] = (int)((all >> 21) & AGG_MASK);
+            a.rem_cnt[b] = (int)((all >> 42) & AGG_MASK);
+        }
+    }
+    // the last block to finish restores the zero state of the shared words
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        const unsigned n_blocks = gridDim.x * gridDim.y;
+        if (atomicAdd(a.done_ctr, 1u) == n_blocks - 1) {
+            for (unsigned q = 0; q < gridDim.y; ++q)
+                for (unsigned j = 0; j < gridDim.x; ++j) a.agg[(int64_t)q * a.agg_stride + j] = 0ull;
+            *a.done_ctr = 0u;
+            *a.dep_ctr = 0u;
+        }
+    }
 }
 
-cudaError_t launch_compact_full(ada_ctx* ctx, int B, int T, float thr, int32_t* rep_idx,
-                                int32_t* rep_cnt, float* gamma, cudaStream_t s) {
-    prof_begin(ctx, K_COMPACT_FULL, s);
-    k_compact_full<<<B, 1024, 0, s>>>(ctx->g_tok, T, thr, rep_idx, rep_cnt, gamma);
+static cudaError_t launch_compact(ada_ctx* ctx, int kid, const CompactArgs& a, int B, cudaStream_t s) {
+    const int nblk = (a.T + 1023) / 1024;
+    if (nblk > a.agg_stride) return cudaErrorInvalidValue;
+    prof_begin(ctx, kid, s);
+    k_compact<<<dim3(nblk, B), 1024, 0, s>>>(a);
     prof_end(ctx, s);
     return cudaGetLastError();
 }
 
-// Algorithm 1 lines 5, 9, 10-11 and the lists of Eq. (6).
-__global__ void __launch_bounds__(1024)
-k_compact_cascade(unsigned* __restrict__ g_tok, unsigned* __restrict__ g_rep,
-                  int32_t* __restrict__ role, unsigned* __restrict__ dep_ctr,
-                  const unsigned* __restrict__ status, int T, float thr,
-                  int32_t* __restrict__ rep_out, int32_t* __restrict__ rep_out_cnt,
-                  int32_t* __restrict__ add_idx, int32_t* __restrict__ add_cnt,
-                  int32_t* __restrict__ rem_idx, int32_t* __restrict__ rem_cnt,
-                  float* __restrict__ gamma_rep, float* __restrict__ gamma_cross) {
-    __shared__ unsigned long long s_warp[33];
-    const int b = blockIdx.x;
-    const int64_t o = (int64_t)b * T;
-    const unsigned faulted = status[0];
-    int base_keep = 0, base_add = 0, base_rem = 0;
-    for (int t0 = 0; t0 < T; t0 += CHUNK) {
-        const int first = t0 + threadIdx.x * CPT;
-        unsigned keep = 0, add = 0, rem = 0;
-        int pos[CPT];
-        unsigned gt[CPT], gp[CPT];
-        // independent loads first, the position-indexed gather second: two round trips in all
-#pragma unroll
-        for (int k = 0; k < CPT; ++k) {
-            const bool in = first + k < T;
-            pos[k] = in ? role[o + first + k] : 0;
-            gt[k] = in ? g_tok[o + first + k] : 0u;
-        }
-#pragma unroll
-        for (int k = 0; k < CPT; ++k) gp[k] = pos[k] > 0 ? g_rep[o + pos[k] - 1] : 0u;
-#pragma unroll
-        for (int k = 0; k < CPT; ++k) {
-            const int t = first + k;
-            if (t >= T) continue;
-            float gr = 0.f, gc = 0.f;
-            if (pos[k] > 0) {       // inherited representative: line 5
-                gr = __uint_as_float(gp[k]);
-                g_rep[o + pos[k] - 1] = 0u;
-                role[o + t] = 0;
-                if (gr < thr) keep |= 1u << k; else rem |= 1u << k;
-            } else {                // line 9
-                gc = __uint_as_float(gt[k]);
-                if (gc < thr) { add |= 1u << k; keep |= 1u << k; }
-            }
-            g_tok[o + t] = 0u;      // rows of inherited reps are never written, clearing is harmless
-            if (gamma_rep != nullptr) gamma_rep[o + t] = gr;
-            if (gamma_cross != nullptr) gamma_cross[o + t] = gc;
-        }
-        // three counts (each <= 8192 per chunk, running totals < 2^21) in one scan
-        const unsigned long long packed = (unsigned long long)__popc(keep) |
-                                          ((unsigned long long)__popc(add) << 21) |
-                                          ((unsigned long long)__popc(rem) << 42);
-        unsigned long long total;
-        const unsigned long long off = block_exclusive_scan(packed, s_warp, total);
-        int ok = base_keep + (int)(off & 0x1FFFFFu);
-        int oa = base_add + (int)((off >> 21) & 0x1FFFFFu);
-        int om = base_rem + (int)((off >> 42) & 0x1FFFFFu);
-#pragma unroll
-        for (int k = 0; k < CPT; ++k) {
-            const int t = first + k;
-            if (keep & (1u << k)) rep_out[o + ok++] = t;
-            if (add & (1u << k)) add_idx[o + oa++] = t;
-            if (rem & (1u << k)) rem_idx[o + om++] = t;
-        }
-        base_keep += (int)(total & 0x1FFFFFu);
-        base_add += (int)((total >> 21) & 0x1FFFFFu);
-        base_rem += (int)((total >> 42) & 0x1FFFFFu);
-    }
-    if (faulted != 0u) {
-        // a rejected inherited list leaves positions without a token: clear them all
-        for (int i = threadIdx.x; i < T; i += blockDim.x) g_rep[o + i] = 0u;
-    }
-    if (threadIdx.x == 0) {
-        rep_out_cnt[b] = base_keep;
-        add_cnt[b] = base_add;
-        rem_cnt[b] = base_rem;
-        if (b == 0) *dep_ctr = 0u;
-    }
+cudaError_t launch_compact_full(ada_ctx* ctx, int B, int T, float thr, int32_t* rep_idx,
+                                int32_t* rep_cnt, float* gamma, cudaStream_t s) {
+    CompactArgs a;
+    a.g_tok = ctx->g_tok; a.g_rep = nullptr; a.role = nullptr;
+    a.agg = ctx->agg; a.done_ctr = ctx->done_ctr; a.dep_ctr = ctx->tile_ctr; a.status = ctx->status;
+    a.agg_stride = ctx->agg_stride; a.T = T; a.thr = thr;
+    a.keep_idx = rep_idx; a.keep_cnt = rep_cnt;
+    a.add_idx = nullptr; a.add_cnt = nullptr; a.rem_idx = nullptr; a.rem_cnt = nullptr;
+    a.gamma_a = gamma; a.gamma_b = nullptr;
+    return launch_compact(ctx, K_COMPACT_FULL, a, B, s);
 }
 
 cudaError_t launch_compact_cascade(ada_ctx* ctx, int B, int T, float thr, int32_t* rep_out,
                                    int32_t* rep_out_cnt, int32_t* add_idx, int32_t* add_cnt,
                                    int32_t* rem_idx, int32_t* rem_cnt, float* gamma_rep,
                                    float* gamma_cross, cudaStream_t s) {
-    prof_begin(ctx, K_COMPACT_CASCADE, s);
-    k_compact_cascade<<<B, 1024, 0, s>>>(ctx->g_tok, ctx->g_rep, ctx->role, ctx->tile_ctr, ctx->status, T, thr,
-                                         rep_out, rep_out_cnt, add_idx, add_cnt, rem_idx, rem_cnt,
-                                         gamma_rep, gamma_cross);
-    prof_end(ctx, s);
-    return cudaGetLastError();
+    CompactArgs a;
+    a.g_tok = ctx->g_tok; a.g_rep = ctx->g_rep; a.role = ctx->role;
+    a.agg = ctx->agg; a.done_ctr = ctx->done_ctr; a.dep_ctr = ctx->tile_ctr; a.status = ctx->status;
+    a.agg_stride = ctx->agg_stride; a.T = T; a.thr = thr;
+    a.keep_idx = rep_out; a.keep_cnt = rep_out_cnt;
+    a.add_idx = add_idx; a.add_cnt = add_cnt; a.rem_idx = rem_idx; a.rem_cnt = rem_cnt;
+    a.gamma_a = gamma_rep; a.gamma_b = gamma_cross;
+    return launch_compact(ctx, K_COMPACT_CASCADE, a, B, s);
 }
 
 }  // namespace ada
