@@ -65,8 +65,15 @@ typedef enum { ADA_F32 = 0, ADA_BF16 = 1 } ada_dtype;
 
 /* Which Gram kernel family a context uses.  AUTO: tensor cores (tcgen05) for
  * ADA_BF16, fp32 FFMA for ADA_F32.  FFMA may be forced for bf16 input (a slow
- * cross-check of the tensor-core path); TCGEN05 cannot be forced for fp32. */
-typedef enum { ADA_ENGINE_AUTO = 0, ADA_ENGINE_FFMA = 1, ADA_ENGINE_TCGEN05 = 2 } ada_engine;
+ * cross-check of the tensor-core path); the tensor-core forms cannot be forced
+ * for fp32.  TCGEN05 is the one-CTA kernel (128-row tiles), TCGEN05_PAIR the
+ * two-CTA kernel (cta_group::2, 256-row tiles shared by the two SMs of a TPC). */
+typedef enum {
+    ADA_ENGINE_AUTO = 0,
+    ADA_ENGINE_FFMA = 1,
+    ADA_ENGINE_TCGEN05 = 2,
+    ADA_ENGINE_TCGEN05_PAIR = 3
+} ada_engine;
 
 typedef struct ada_ctx ada_ctx; /* opaque */
 

@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libada.so")
 ADA_OK = 0
 ADA_F32, ADA_BF16 = 0, 1
 ADA_CROSS_CAUSAL = 1
-ADA_ENGINE_AUTO, ADA_ENGINE_FFMA, ADA_ENGINE_TCGEN05 = 0, 1, 2
+ADA_ENGINE_AUTO, ADA_ENGINE_FFMA, ADA_ENGINE_TCGEN05, ADA_ENGINE_TCGEN05_PAIR = 0, 1, 2, 3
 
 SYMBOLS = [
     "ada_create", "ada_destroy", "ada_set_engine", "ada_normalize", "ada_select_full",

@@ -53,8 +53,14 @@ bool use_tc(const ada_ctx* ctx, ada_dtype dt) {
     return gram_tc_available();
 }
 
+// tensor-core launch of one or two segments, in the one-CTA or the pair-CTA form
+cudaError_t launch_tc(ada_ctx* ctx, const GramProblem* tri, const GramProblem* cross, cudaStream_t s) {
+    if (ctx->engine == ADA_ENGINE_TCGEN05_PAIR) return launch_gram_tc2(ctx, tri, cross, s);
+    return launch_gram_tc(ctx, tri, cross, s);
+}
+
 cudaError_t run_gram(ada_ctx* ctx, const GramProblem& p, ada_dtype dt, cudaStream_t s) {
-    if (use_tc(ctx, dt)) return p.tri ? launch_gram_tc(ctx, &p, nullptr, s) : launch_gram_tc(ctx, nullptr, &p, s);
+    if (use_tc(ctx, dt)) return p.tri ? launch_tc(ctx, &p, nullptr, s) : launch_tc(ctx, nullptr, &p, s);
     return launch_gram_ffma(ctx, p, dt, s);
 }
 
@@ -133,6 +139,8 @@ ada_status ada_create(ada_ctx** out, int device, int64_t maxB, int64_t maxT, int
     ctx->engine = ADA_ENGINE_AUTO;
     ctx->stage = nullptr; ctx->stage_bytes = 0; ctx->host_stream = nullptr;
     ctx->tc_attr_set = false;
+    ctx->tc2_attr_set = false;
+    ctx->tc2_pairs = 0;
     cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
 
     const size_t n_tok = (size_t)maxB * (size_t)maxT;
@@ -189,9 +197,11 @@ ada_status ada_destroy(ada_ctx* ctx) {
 
 ada_status ada_set_engine(ada_ctx* ctx, ada_engine e) {
     if (ctx == nullptr) return ADA_ERR_INVALID_ARG;
-    if (e != ADA_ENGINE_AUTO && e != ADA_ENGINE_FFMA && e != ADA_ENGINE_TCGEN05)
+    if (e != ADA_ENGINE_AUTO && e != ADA_ENGINE_FFMA && e != ADA_ENGINE_TCGEN05 &&
+        e != ADA_ENGINE_TCGEN05_PAIR)
         return ADA_ERR_INVALID_ARG;
-    if (e == ADA_ENGINE_TCGEN05 && (ctx->dt != ADA_BF16 || !gram_tc_available()))
+    if ((e == ADA_ENGINE_TCGEN05 || e == ADA_ENGINE_TCGEN05_PAIR) &&
+        (ctx->dt != ADA_BF16 || !gram_tc_available()))
         return ADA_ERR_UNSUPPORTED;
     ctx->engine = e;
     return ADA_OK;
@@ -297,7 +307,7 @@ ada_status ada_cascade_step(ada_ctx* ctx, const void* X, int64_t B, int64_t T, i
     q.col_token = rep_in;
     q.row_role = ctx->role;
     q.causal = (flags & ADA_CROSS_CAUSAL) ? 1 : 0;
-    if (fuse) CU(launch_gram_tc(ctx, &p, &q, s));
+    if (fuse) CU(launch_tc(ctx, &p, &q, s));
     else CU(run_gram(ctx, q, dt, s));
     // lines 5, 9, 10-11
     CU(launch_compact_cascade(ctx, (int)B, (int)T, thr, rep_out, rep_out_cnt, add_idx, add_cnt,

@@ -81,6 +81,8 @@ struct ada_ctx {
     ada_engine engine;
     int sm_count;
     bool tc_attr_set;
+    bool tc2_attr_set;   // pair-CTA kernel configured
+    int tc2_pairs;       // clusters of two that fit on the device at once
     // device workspace
     char* ws;            // one allocation
     float* inv_norm;     // [maxB*maxT] 1/||x_t||
@@ -127,5 +129,9 @@ cudaError_t launch_gram_ffma(ada_ctx* ctx, const GramProblem& p, ada_dtype dt, c
 cudaError_t launch_gram_tc(ada_ctx* ctx, const GramProblem* tri, const GramProblem* cross,
                            cudaStream_t s);
 bool gram_tc_available();
+
+// gram_tc2.cu (bf16, tcgen05.cta_group::2: two CTAs per 256-row tile)
+cudaError_t launch_gram_tc2(ada_ctx* ctx, const GramProblem* tri, const GramProblem* cross,
+                            cudaStream_t s);
 
 }  // namespace ada

@@ -22,166 +22,14 @@
 // Every wait is bounded: when a limit expires the CTA raises the context's TIMEOUT
 // status, drains its own outstanding copies and MMAs (again bounded), frees its TMEM
 // and returns.
-#include <cuda.h>
-#include <string.h>
+#include "gram_tc_dev.cuh"
 
-#include "common.cuh"
 
 namespace ada {
 
+using namespace tc;
+
 namespace {
-
-constexpr int BM = 128;          // accumulator rows per tile (TMEM lanes)
-constexpr int BN = 256;          // accumulator columns per tile
-constexpr int BK = 64;           // bf16 elements per K block = one 128-byte swizzle row
-constexpr int MAX_STAGES = 9;
-constexpr int RING_BYTES = 216 * 1024;               // TMA ring: 4 stages of a 256-wide tile ... 9 of a 64-wide one
-constexpr int UMMA_K = 16;
-constexpr int A_BYTES = BM * BK * 2;                 // 16 KiB
-constexpr int BOX_N = 64;                            // B rows per TMA box
-constexpr int BOX_BYTES = BOX_N * BK * 2;            // 8 KiB
-constexpr int NUM_THREADS = 192;
-constexpr int TMEM_COLS = 512;
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // 2 s
-
-// one output tile: `ncols` (multiple of 16, <= 256) columns from col0 of the 128-row tile at row0
-struct Piece {
-    int b, row0, col0, ncols, n, m;
-};
-
-struct alignas(16) Shared {
-    unsigned long long full[MAX_STAGES];
-    unsigned long long empty[MAX_STAGES];
-    unsigned long long tmem_full[2];
-    unsigned long long tmem_empty[2];
-    unsigned long long drain;
-    unsigned tmem_base;
-    int abort_flag;
-    int tiles0, tiles1, tw0;
-    // per epilogue warp, so that staging needs no barrier across warps
-    alignas(16) float col_scale[4][BN];
-    alignas(16) int col_token[4][BN];
-};
-constexpr int SMEM_BYTES = RING_BYTES + (int)sizeof(Shared) + 1024;   // +1024: alignment slack
-static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
-
-// ---------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ unsigned smem_u32(const void* p) {
-    return static_cast<unsigned>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ void mbar_init(unsigned long long* bar, unsigned count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, unsigned bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)),
-                 "r"(bytes)
-                 : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(unsigned long long* bar, unsigned parity) {
-    unsigned ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ unsigned long long global_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-// Bounded wait.  Returns false when the CTA is aborting (this or another wait ran out).
-// try_wait itself suspends the thread for a while before it reports failure, so the wall
-// clock (a slow special register) is consulted only once per 256 failed polls.
-__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity,
-                                          volatile int* abort_flag, int where) {
-    unsigned polls = 0;
-    unsigned long long t0 = 0;
-    while (!mbar_try(bar, parity)) {
-        if ((++polls & 255u) == 0) {
-            if (*abort_flag != 0) return false;
-            const unsigned long long now = global_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > WAIT_LIMIT_NS) {
-                *abort_flag = where;
-                return false;
-            }
-        }
-    }
-    return true;
-}
-__device__ __forceinline__ void tma_load_3d(const CUtensorMap* map, unsigned long long* bar,
-                                            void* dst, int c0, int c1, int c2) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
-        " [%0], [%1, {%3, %4, %5}], [%2];"
-        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<unsigned long long>(map)), "r"(smem_u32(bar)),
-          "r"(c0), "r"(c1), "r"(c2)
-        : "memory");
-}
-__device__ __forceinline__ void tcgen05_fence_before() {
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-}
-__device__ __forceinline__ void tcgen05_fence_after() {
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-}
-__device__ __forceinline__ void umma_commit(unsigned long long* bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
-                 ::"r"(smem_u32(bar))
-                 : "memory");
-}
-__device__ __forceinline__ void umma_bf16(unsigned tmem_d, unsigned long long adesc,
-                                          unsigned long long bdesc, unsigned idesc,
-                                          unsigned accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(unsigned taddr, float (&v)[32]) {
-    unsigned r[32];
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n\t"
-        // the wait sits in the same statement so that no use of the registers can be
-        // scheduled ahead of it
-        "tcgen05.wait::ld.sync.aligned;"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
-          "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
-          "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]),
-          "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]),
-          "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr)
-        : "memory");
-#pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-}
-
-// Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes wide and
-// stored with the 128-byte swizzle: 8-row groups are 1024 bytes apart (stride byte offset),
-// the leading byte offset is unused for swizzled K-major tiles, descriptor version 1.
-__device__ __forceinline__ unsigned long long smem_desc_sw128(unsigned addr) {
-    unsigned long long d = 0;
-    d |= (unsigned long long)((addr & 0x3FFFFu) >> 4);        // start address, 16-byte units
-    d |= (unsigned long long)1 << 16;                         // leading byte offset (ignored)
-    d |= (unsigned long long)(1024 >> 4) << 32;               // stride byte offset
-    d |= (unsigned long long)1 << 46;                         // descriptor version (sm_100)
-    d |= (unsigned long long)2 << 61;                         // layout: 128-byte swizzle
-    return d;
-}
-// Instruction descriptor: D = fp32, A = B = bf16, both K-major, M = 128, N = n.
-__device__ __forceinline__ unsigned instr_desc(int n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((unsigned)(n >> 3) << 17) | ((unsigned)(BM >> 4) << 24);
-}
 
 // ---------------------------------------------------------------- work schedule
 // A launch covers up to two problems ("segments"): a triangular one (Definition 1 on X, or
@@ -530,43 +378,6 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
         atomicOr(status, ST_TIMEOUT);
         status[2] = (unsigned)sh.abort_flag;
     }
-}
-
-// ---------------------------------------------------------------- host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
-                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
-                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) ==
-                cudaSuccess && q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-        else
-            cudaGetLastError();
-    }
-    return fn;
-}
-
-// 3-D map over a stack of K-major bf16 matrices: (k, row, sequence).
-bool make_map(CUtensorMap* map, const void* base, int d, int rows, int B, int64_t ld,
-              int64_t batch, int box_rows) {
-    EncodeTiledFn fn = encode_fn();
-    if (fn == nullptr) return false;
-    const cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)rows, (cuuint64_t)B};
-    // the stride of the last dimension is unused when B == 1 but must still be legal
-    const cuuint64_t strides[2] = {(cuuint64_t)ld * 2, (cuuint64_t)(B > 1 ? batch : (int64_t)rows * ld) * 2};
-    const cuuint32_t box[3] = {(cuuint32_t)BK, (cuuint32_t)box_rows, 1};
-    const cuuint32_t estr[3] = {1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box,
-              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 }  // namespace

@@ -1,0 +1,469 @@
+// bf16 masked-Gram kernel for sm_100a, two-CTA form: the CTAs of a cluster of two
+// (one per SM of a TPC) share one 256-row output tile.  Each CTA loads its own 128 rows
+// of the left operand but only HALF of the right operand's columns; the leader CTA
+// issues tcgen05.mma.cta_group::2 (M = 256), which reads both halves from the two shared
+// memories and writes each CTA's 128 x N accumulator into its own TMEM.  Per CTA and
+// K block that is 16 KiB + N*64 bytes of TMA traffic instead of 16 KiB + N*128: the
+// one-CTA kernel is bound by what one SM can pull out of L2, this one by the tensor pipe.
+//
+// Same contract as the one-CTA kernel (out[i] = max_j |a_i.b_j| inv_a[i] inv_b[j] over the
+// admissible j; Definition 1, Algorithm 1 lines 3-4 and 7-8; the Gram never leaves TMEM),
+// same tile list (triangular segment first, cross epilogues wait for it), same warp roles:
+//   warp 0      TMA producer in BOTH CTAs (completion bytes of both land on the leader's
+//               mbarrier; no multicast is used)
+//   warp 1      leader: MMA issuer; releases ring stages and hands over accumulators with
+//               tcgen05.commit multicast to both CTAs.  Both CTAs: TMEM allocation
+//   warps 2..5  epilogue in both CTAs, each on its own 128 rows; the peer's epilogue
+//               returns the accumulator by a remote arrive on the leader's mbarrier
+// Every wait is bounded; the two CTAs meet at a cluster barrier before either frees TMEM
+// or exits.
+#include "gram_tc_dev.cuh"
+
+namespace ada {
+
+using namespace tc;
+
+namespace {
+
+constexpr int PM = 2 * BM;     // rows of a pair tile
+
+// ---------------------------------------------------------------- PTX, pair forms
+__device__ __forceinline__ unsigned cluster_rank() {
+    unsigned r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// address of the same shared-memory location in CTA `rank` of this cluster
+__device__ __forceinline__ unsigned map_to_cta(unsigned addr, unsigned rank) {
+    unsigned r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_remote(unsigned cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr)
+                 : "memory");
+}
+// TMA load whose completion bytes go to the LEADER's barrier: bit 24 of a shared::cluster
+// address selects the CTA within the pair, clearing it names the even (leader) CTA.
+__device__ __forceinline__ void tma_load_3d_pair(const CUtensorMap* map, unsigned long long* bar,
+                                                 void* dst, int c0, int c1, int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<unsigned long long>(map)),
+          "r"(smem_u32(bar) & 0xFEFFFFFFu), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(unsigned tmem_d, unsigned long long adesc,
+                                               unsigned long long bdesc, unsigned idesc,
+                                               unsigned accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// commit: arrive on the barrier at this offset in BOTH CTAs once the MMAs issued so far retire
+__device__ __forceinline__ void umma_commit_pair_both(unsigned long long* bar) {
+    const unsigned short mask = 3;
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(smem_u32(bar)), "h"(mask)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit_pair_local(unsigned long long* bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                 ::"r"(smem_u32(bar))
+                 : "memory");
+}
+// instruction descriptor of the pair MMA: M = 256
+__device__ __forceinline__ unsigned instr_desc_pair(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((unsigned)(n >> 3) << 17) | ((unsigned)(PM >> 4) << 24);
+}
+
+// ---------------------------------------------------------------- tile list (256-row tiles)
+__device__ __forceinline__ int seq_n(const GramProblem& p, int b) {
+    return p.n_dev != nullptr ? p.n_dev[b] : p.n_host;
+}
+__device__ __forceinline__ int tri_tiles(int n) {           // row pair P needs column tiles 0..P
+    const int M = (n + PM - 1) / PM;
+    return M * (M + 1) / 2;
+}
+__device__ __forceinline__ void cross_cols(int n, int& nct, int& w) {
+    nct = (n + BN - 1) / BN;
+    w = nct > 0 ? ((((n + nct - 1) / nct) + 31) & ~31) : 0;    // each CTA holds w/2 columns: keep w/2 a multiple of 16
+}
+__device__ __forceinline__ int seg_tiles(const GramProblem& p) {
+    int total = 0;
+    for (int b = 0; b < p.B; ++b) {
+        const int n = seq_n(p, b);
+        if (n <= 0) continue;
+        if (p.tri) total += tri_tiles(n);
+        else {
+            int nct, w;
+            cross_cols(n, nct, w);
+            total += ((p.rows + PM - 1) / PM) * nct;
+        }
+    }
+    return total;
+}
+__device__ __forceinline__ bool decode_tile(const GramProblem& p, int id, Piece& t) {
+    for (int b = 0; b < p.B; ++b) {
+        const int n = seq_n(p, b);
+        if (n <= 0) continue;
+        int cnt, nct = 0, w = 0;
+        if (p.tri) cnt = tri_tiles(n);
+        else {
+            cross_cols(n, nct, w);
+            cnt = ((p.rows + PM - 1) / PM) * nct;
+        }
+        if (id >= cnt) { id -= cnt; continue; }
+        t.b = b;
+        t.n = n;
+        int nc;
+        if (p.tri) {
+            int mi = (int)((sqrtf(8.0f * (float)id + 1.0f) - 1.0f) * 0.5f);
+            while (mi * (mi + 1) / 2 > id) --mi;
+            while ((mi + 1) * (mi + 2) / 2 <= id) ++mi;
+            t.row0 = mi * PM;
+            t.col0 = (id - mi * (mi + 1) / 2) * BN;
+            t.m = n;
+            nc = min(n - t.col0, BN);
+        } else {
+            t.row0 = (id / nct) * PM;
+            t.col0 = (id % nct) * w;
+            t.m = p.rows;
+            nc = min(n - t.col0, w);
+        }
+        t.ncols = max(32, (nc + 31) & ~31);
+        return true;
+    }
+    return false;
+}
+// per-CTA stage: 128 rows of A and ncols/2 rows of B (in 64-row boxes)
+__device__ __forceinline__ int stage_bytes_pair(int ncols) {
+    return A_BYTES + (((ncols >> 1) + BOX_N - 1) / BOX_N) * BOX_BYTES;
+}
+__device__ __forceinline__ int stage_count(int sbytes) {
+    return min(MAX_STAGES, RING_BYTES / sbytes);
+}
+
+struct GramMaps {
+    CUtensorMap a[2], b[2];
+};
+
+// ---------------------------------------------------------------- the kernel
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramProblem seg0,
+           const __grid_constant__ GramProblem seg1, const int nseg, unsigned* __restrict__ dep_ctr,
+           unsigned* __restrict__ status) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>(
+        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    Shared& sh = *reinterpret_cast<Shared*>(smem + RING_BYTES);
+    volatile int* abort_flag = &sh.abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const unsigned rank = cluster_rank();            // 0 = leader
+    const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < MAX_STAGES; ++s) {
+            mbar_init(&sh.full[s], 1);
+            mbar_init(&sh.empty[s], 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(&sh.tmem_full[a], 1);
+            mbar_init(&sh.tmem_empty[a], 8);      // four epilogue warps in each CTA
+        }
+        mbar_init(&sh.drain, 1);
+        sh.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (threadIdx.x == 64) {
+        sh.tiles0 = seg_tiles(seg0);
+        sh.tiles1 = nseg > 1 ? seg_tiles(seg1) : 0;
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&sh.tmem_base)), "r"(TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    cluster_sync_all();          // the peer's barriers exist before anything signals them
+    tcgen05_fence_after();
+    const unsigned tmem_base = sh.tmem_base;
+    const int tiles0 = sh.tiles0, total = sh.tiles0 + sh.tiles1;
+    Piece pc;
+
+    if (warp == 0) {
+        // ------------------------------------------------ TMA producer (both CTAs)
+        if (lane == 0) {
+            unsigned fills = 0, used = 0, ever = 0;
+            int cur_sb = 0, cur_nst = 0, s = 0;
+            bool ok = true;
+            for (int id = pair; ok && id < total; id += npairs) {
+                const int sg = id < tiles0 ? 0 : 1;
+                const GramProblem& p = sg ? seg1 : seg0;
+                if (!decode_tile(p, id - (sg ? tiles0 : 0), pc)) break;
+                const int num_kb = (p.d + BK - 1) / BK;
+                const int half = pc.ncols >> 1;
+                const int nbox = (half + BOX_N - 1) / BOX_N;
+                const int sb = stage_bytes_pair(pc.ncols);
+                if (sb != cur_sb) {
+                    for (int q = 0; q < cur_nst && ok; ++q)
+                        if ((used >> q) & 1u)
+                            ok = mbar_wait(&sh.empty[q], ((fills >> q) & 1u) ^ 1u, abort_flag, 6);
+                    if (!ok) break;
+                    cur_sb = sb; cur_nst = stage_count(sb); s = 0; used = 0;
+                }
+                const int a_row = pc.row0 + (int)rank * BM;
+                const int b_row = pc.col0 + (int)rank * half;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(&sh.empty[s], ((fills >> s) & 1u) ^ 1u, abort_flag, 1)) { ok = false; break; }
+                    unsigned char* sa = smem + s * sb;
+                    // the leader's barrier counts the bytes of both CTAs
+                    if (rank == 0) mbar_expect_tx(&sh.full[s], 2u * (unsigned)sb);
+                    tma_load_3d_pair(&maps.a[sg], &sh.full[s], sa, kb * BK, a_row, pc.b);
+                    for (int j = 0; j < nbox; ++j)
+                        tma_load_3d_pair(&maps.b[sg], &sh.full[s], sa + A_BYTES + j * BOX_BYTES, kb * BK,
+                                         b_row + j * BOX_N, pc.b);
+                    fills ^= 1u << s; used |= 1u << s; ever |= 1u << s;
+                    s = (s + 1 == cur_nst) ? 0 : s + 1;
+                }
+            }
+            // drain: a stage's release (empty) implies its copy landed and was consumed
+            for (int q = 0; q < MAX_STAGES; ++q) {
+                if (!((ever >> q) & 1u)) continue;
+                const unsigned ph = ((fills >> q) & 1u) ^ 1u;
+                const unsigned long long t0 = global_ns();
+                while (!mbar_try(&sh.empty[q], ph)) {
+                    if (*abort_flag != 0 || global_ns() - t0 > WAIT_LIMIT_NS / 2) { *abort_flag = 7; break; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer (leader CTA only)
+        if (lane == 0 && rank == 0) {
+            unsigned uses = 0, tile_it = 0;
+            int cur_sb = 0, cur_nst = 0, s = 0;
+            bool ok = true;
+            for (int id = pair; ok && id < total; id += npairs, ++tile_it) {
+                const int sg = id < tiles0 ? 0 : 1;
+                const GramProblem& p = sg ? seg1 : seg0;
+                if (!decode_tile(p, id - (sg ? tiles0 : 0), pc)) break;
+                const int num_kb = (p.d + BK - 1) / BK;
+                const int sb = stage_bytes_pair(pc.ncols);
+                if (sb != cur_sb) { cur_sb = sb; cur_nst = stage_count(sb); s = 0; }
+                const unsigned acc = tile_it & 1u, acc_ph = (tile_it >> 1) & 1u;
+                if (!mbar_wait(&sh.tmem_empty[acc], acc_ph ^ 1u, abort_flag, 2)) { ok = false; break; }
+                tcgen05_fence_after();
+                const unsigned idesc = instr_desc_pair(pc.ncols);
+                const unsigned d_tmem = tmem_base + acc * BN;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(&sh.full[s], (uses >> s) & 1u, abort_flag, 3)) { ok = false; break; }
+                    tcgen05_fence_after();
+                    const unsigned a_addr = smem_u32(smem + s * sb);
+                    const unsigned long long adesc = smem_desc_sw128(a_addr);
+                    const unsigned long long bdesc = smem_desc_sw128(a_addr + A_BYTES);
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; ++k)
+                        umma_bf16_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+                    umma_commit_pair_both(&sh.empty[s]);   // both producers may refill this stage
+                    uses ^= 1u << s;
+                    s = (s + 1 == cur_nst) ? 0 : s + 1;
+                }
+                if (ok) umma_commit_pair_both(&sh.tmem_full[acc]);   // both epilogues may read
+            }
+            umma_commit_pair_local(&sh.drain);
+            const unsigned long long t0 = global_ns();
+            while (!mbar_try(&sh.drain, 0)) {
+                if (global_ns() - t0 > WAIT_LIMIT_NS / 2) { *abort_flag = 8; break; }
+            }
+        }
+    } else {
+        // ------------------------------------------------ epilogue (warps 2..5, both CTAs)
+        const int quad = warp & 3;
+        float* cs = sh.col_scale[warp - 2];
+        int* ct = sh.col_token[warp - 2];
+        const unsigned dep_total = 8u * (unsigned)tiles0;
+        bool dep_ok = !(nseg > 1 && tiles0 > 0);
+        // the accumulator goes back to the leader's barrier
+        const unsigned empty_addr[2] = {map_to_cta(smem_u32(&sh.tmem_empty[0]), 0),
+                                        map_to_cta(smem_u32(&sh.tmem_empty[1]), 0)};
+        unsigned tile_it = 0;
+        for (int id = pair; id < total; id += npairs, ++tile_it) {
+            const int sg = id < tiles0 ? 0 : 1;
+            const GramProblem& p = sg ? seg1 : seg0;
+            if (!decode_tile(p, id - (sg ? tiles0 : 0), pc)) break;
+            const unsigned acc = tile_it & 1u, acc_ph = (tile_it >> 1) & 1u;
+            const int64_t o = (int64_t)pc.b * p.cap;
+            const int ncols = pc.ncols;
+            if (sg == 1 && !dep_ok) {
+                int good = 1;
+                if (lane == 0) {
+                    const unsigned long long t0 = global_ns();
+                    unsigned seen;
+                    while (true) {
+                        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(dep_ctr) : "memory");
+                        if (seen >= dep_total) break;
+                        if (*abort_flag != 0) { good = 0; break; }
+                        if (global_ns() - t0 > WAIT_LIMIT_NS) { *abort_flag = 5; good = 0; break; }
+                        __nanosleep(64);
+                    }
+                }
+                good = __shfl_sync(0xffffffffu, good, 0);
+                if (!good) break;
+                dep_ok = true;
+            }
+            __syncwarp();
+            for (int c = lane; c < ncols; c += 32) {
+                const int col = pc.col0 + c;
+                float f = 0.f;
+                int tok = col;
+                if (col < pc.n) {
+                    f = p.inv_b[o + col];
+                    if (!p.tri) {
+                        if (!(__ldcg(p.col_gate + o + col) < p.thr_bits)) f = 0.f;
+                        if (p.causal) tok = p.col_token[o + col];
+                    }
+                }
+                cs[c] = f;
+                ct[c] = tok;
+            }
+            __syncwarp();
+            const bool got = mbar_wait(&sh.tmem_full[acc], acc_ph, abort_flag, 4);
+            if (!__all_sync(0xffffffffu, got)) break;
+            tcgen05_fence_after();
+            const int row_base = pc.row0 + (int)rank * BM;
+            const int row = row_base + quad * 32 + lane;
+            const bool need_cmp = p.tri ? (pc.col0 + ncols > row_base) : (p.causal != 0);
+            float mx = 0.f;
+            for (int c0 = 0; c0 < ncols; c0 += 32) {
+                float v[32];
+                tmem_ld32(tmem_base + ((unsigned)(quad * 32) << 16) + acc * BN + c0, v);
+                if (!need_cmp) {
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4) {
+                        const float4 f = *reinterpret_cast<const float4*>(cs + c0 + j);
+                        mx = fmaxf(mx, fabsf(v[j]) * f.x);
+                        mx = fmaxf(mx, fabsf(v[j + 1]) * f.y);
+                        mx = fmaxf(mx, fabsf(v[j + 2]) * f.z);
+                        mx = fmaxf(mx, fabsf(v[j + 3]) * f.w);
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const float x = fabsf(v[j]) * cs[c0 + j];
+                        if (ct[c0 + j] < row) mx = fmaxf(mx, x);
+                    }
+                }
+            }
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_remote(empty_addr[acc]);
+            if (row < pc.m) {
+                const bool skip = !p.tri && p.row_role[o + row] != 0;
+                if (!skip) {
+                    mx *= p.inv_a[o + row];
+                    if (mx > 0.f) atomicMax(p.out + o + row, __float_as_uint(mx));
+                }
+            }
+            if (sg == 0 && nseg > 1) {
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) atomicAdd(dep_ctr, 1u);
+            }
+        }
+    }
+
+    tcgen05_fence_before();
+    __syncthreads();
+    cluster_sync_all();          // neither CTA frees TMEM or exits while the other may still touch it
+    if (warp == 1) {
+        tcgen05_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                     "r"(TMEM_COLS)
+                     : "memory");
+    }
+    if (threadIdx.x == 0 && sh.abort_flag != 0) {
+        atomicOr(status, ST_TIMEOUT);
+        status[2] = 100u + (unsigned)sh.abort_flag;
+    }
+}
+
+}  // namespace
+
+// Pair-CTA launch.  tri and/or cross may be NULL; with both the cross epilogues wait in-kernel
+// for the triangular segment (ctx->tile_ctr must be zero at launch).
+cudaError_t launch_gram_tc2(ada_ctx* ctx, const GramProblem* tri, const GramProblem* cross,
+                            cudaStream_t s) {
+    if (!ctx->tc2_attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(k_gram_tc2, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        // how many clusters of two fit on the device at once
+        cudaLaunchConfig_t q;
+        memset(&q, 0, sizeof(q));
+        q.gridDim = dim3(2 * (ctx->sm_count / 2));
+        q.blockDim = dim3(NUM_THREADS);
+        q.dynamicSmemBytes = SMEM_BYTES;
+        cudaLaunchAttribute qa[1];
+        qa[0].id = cudaLaunchAttributeClusterDimension;
+        qa[0].val.clusterDim.x = 2; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
+        q.attrs = qa; q.numAttrs = 1;
+        int nclusters = 0;
+        e = cudaOccupancyMaxActiveClusters(&nclusters, k_gram_tc2, &q);
+        if (e != cudaSuccess || nclusters < 1) { cudaGetLastError(); return cudaErrorLaunchOutOfResources; }
+        ctx->tc2_pairs = nclusters < ctx->sm_count / 2 ? nclusters : ctx->sm_count / 2;
+        ctx->tc2_attr_set = true;
+    }
+    GramMaps maps;
+    memset(&maps, 0, sizeof(maps));
+    GramProblem segs[2];
+    memset(segs, 0, sizeof(segs));
+    int nseg = 0;
+    const GramProblem* in[2] = {tri, cross};
+    for (int i = 0; i < 2; ++i) {
+        const GramProblem* p = in[i];
+        if (p == nullptr) continue;
+        const int n_cap = p->n_dev != nullptr ? p->cap : p->n_host;
+        const int a_rows = p->tri ? n_cap : p->rows;
+        if (n_cap <= 0 || a_rows <= 0) continue;
+        if (!make_map(&maps.a[nseg], p->A, p->d, p->tri ? p->cap : p->rows, p->B, p->lda, p->a_batch, BM) ||
+            !make_map(&maps.b[nseg], p->Bm, p->d, p->cap, p->B, p->ldb, p->b_batch, BOX_N))
+            return cudaErrorInvalidValue;
+        segs[nseg++] = *p;
+    }
+    if (nseg == 0) return cudaSuccess;
+    if (nseg == 1) { maps.a[1] = maps.a[0]; maps.b[1] = maps.b[0]; segs[1] = segs[0]; segs[1].B = 0; }
+    const bool fused = nseg == 2;
+    prof_begin(ctx, fused ? K_GRAM_TC_CASCADE : (segs[0].tri ? K_GRAM_TC_TRI : K_GRAM_TC_CROSS), s);
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(2 * ctx->tc2_pairs);
+    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeCooperative;
+    attr[1].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = fused ? 2 : 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, k_gram_tc2, maps, segs[0], segs[1], nseg, ctx->tile_ctr,
+                                       ctx->status);
+    prof_end(ctx, s);
+    return e;
+}
+
+}  // namespace ada

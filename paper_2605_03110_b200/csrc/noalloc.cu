@@ -51,6 +51,8 @@ ada_status setup_device(int device, PerDevice** out) {
         c.maxd = 0;
         c.engine = ADA_ENGINE_AUTO;
         c.tc_attr_set = false;
+        c.tc2_attr_set = false;
+        c.tc2_pairs = 0;
         c.ws = nullptr;
         c.stage = nullptr;
         c.stage_bytes = 0;

@@ -30,7 +30,8 @@ def clustered(T, d, seed, dtype):
     return wl.f32_to_bf16_bits(X) if dtype == "bf16" else X
 
 
-ENGINES = [("f32", 0), ("bf16", 0), ("bf16", 1)]   # (storage, engine): AUTO, AUTO, forced FFMA
+# (storage, engine): AUTO, AUTO, forced FFMA, forced one-CTA tcgen05, forced pair-CTA tcgen05
+ENGINES = [("f32", 0), ("bf16", 0), ("bf16", 1), ("bf16", 2), ("bf16", 3)]
 
 
 @pytest.mark.parametrize("dtype,engine", ENGINES)
@@ -111,12 +112,19 @@ def test_config2_ffma_engine_matches(ada):
     assert run_config_chain(ada, wl.scaled(wl.CONFIGS[2], B=2), n_layers=3, engine=1) == 0
 
 
-def sampled_large(ada, cfg, n_layers, n_sample=48):
+@pytest.mark.parametrize("engine", [2, 3])
+def test_config2_and_3_on_both_tensor_core_kernels(ada, engine):
+    assert run_config_chain(ada, wl.CONFIGS[2], n_layers=4, causal=True, engine=engine) == 0
+    assert run_config_chain(ada, wl.CONFIGS[3], n_layers=4, engine=engine) == 0
+
+
+def sampled_large(ada, cfg, n_layers, n_sample=48, engine=0):
     """Full-size check where the oracle cannot do a whole layer quickly: sets by the
     label-level prediction (exact, no Gram), gamma on sampled rows by the oracle."""
     from parity import TOL, lists, to_device
     tol = TOL[cfg.dtype]
     ctx = ada.ada_create(cfg.B, cfg.T, cfg.d, ada.ADA_BF16)
+    ada.ada_set_engine(ctx, engine)
     rng = np.random.default_rng(5)
     R_lab = None
     for lb in wl.generate_layers(cfg, seed=0, n_layers=n_layers):
@@ -152,8 +160,9 @@ def sampled_large(ada, cfg, n_layers, n_sample=48):
     ada.ada_destroy(ctx)
 
 
-def test_config4_opt_shaped_full_size_sampled(ada):
-    sampled_large(ada, wl.CONFIGS[4], n_layers=3)
+@pytest.mark.parametrize("engine", [2, 3])
+def test_config4_opt_shaped_full_size_sampled(ada, engine):
+    sampled_large(ada, wl.CONFIGS[4], n_layers=3, engine=engine)
 
 
 @pytest.mark.parametrize("T,q", [(512, 0.01), (1024, 0.5), (4096, 0.05), (16384, 0.01), (16384, 0.2)])
