@@ -55,7 +55,14 @@ bool use_tc(const ada_ctx* ctx, ada_dtype dt) {
 
 // tensor-core launch of one or two segments, in the one-CTA or the pair-CTA form
 cudaError_t launch_tc(ada_ctx* ctx, const GramProblem* tri, const GramProblem* cross, cudaStream_t s) {
-    if (ctx->engine == ADA_ENGINE_TCGEN05_PAIR) return launch_gram_tc2(ctx, tri, cross, s);
+    bool pair = ctx->engine == ADA_ENGINE_TCGEN05_PAIR;
+    if (ctx->engine == ADA_ENGINE_AUTO) {
+        // The pair kernel pays off once there are several 256-row tiles per SM pair and a long
+        // contraction; small problems are covered better by the finer one-CTA tiles.
+        const GramProblem* p = cross != nullptr ? cross : tri;
+        pair = (int64_t)p->B * p->rows >= 8192 && p->d >= 2048;
+    }
+    if (pair) return launch_gram_tc2(ctx, tri, cross, s);
     return launch_gram_tc(ctx, tri, cross, s);
 }
 

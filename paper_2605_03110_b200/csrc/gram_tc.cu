@@ -45,11 +45,12 @@ namespace {
 __device__ __forceinline__ int seq_n(const GramProblem& p, int b) {
     return p.n_dev != nullptr ? p.n_dev[b] : p.n_host;
 }
-// lower-triangular tile count for column tiles of width tw (128 or 256): the 128-row tile mi
-// needs the column tiles that start at or before its last row
+// lower-triangular tile count for column tiles of width tw (64, 128 or 256): the 128-row
+// tile mi needs the column tiles that start at or before its last row
 __device__ __forceinline__ int tri_tiles(int n, int tw) {
     const int M = (n + BM - 1) / BM;
-    if (tw == BM) return M * (M + 1) / 2;
+    if (tw == BM) return M * (M + 1) / 2;                // mi + 1 each
+    if (tw == BM / 2) return M * (M + 1);                // 2 (mi + 1) each
     const int P = M >> 1;                                // row tiles 2P and 2P+1 both need P+1
     return P * (P + 1) + ((M & 1) ? P + 1 : 0);
 }
@@ -62,34 +63,47 @@ __device__ __forceinline__ int stage_bytes(int ncols) {
 __device__ __forceinline__ int stage_count(int sbytes) {
     return min(MAX_STAGES, RING_BYTES / sbytes);
 }
-// cross: columns are cut into nct equal tiles of width w (multiple of 16, <= 256)
-__device__ __forceinline__ void cross_cols(int n, int& nct, int& w) {
-    nct = (n + BN - 1) / BN;
+// cross: columns are cut into nct equal tiles of width w (multiple of 16, <= 256).  `want` is
+// the number of column tiles per row tile that would give every CTA one tile: a problem
+// with few row tiles is cut finer (down to 64 columns), since a narrow tile moves fewer
+// bytes per K block and finishes sooner, while a large one keeps 256-wide tiles.
+__device__ __forceinline__ void cross_cols(int n, int want, int& nct, int& w) {
+    const int lo = (n + BN - 1) / BN, hi = (n + BOX_N - 1) / BOX_N;
+    nct = min(max(want, lo), hi);
     w = nct > 0 ? ((((n + nct - 1) / nct) + 15) & ~15) : 0;
 }
-__device__ __forceinline__ int seg_tiles(const GramProblem& p, int tw) {
+// column tiles per row tile that fill the grid once (cross segment)
+__device__ __forceinline__ int cross_want(const GramProblem& p, int G) {
+    int row_tiles = 0;
+    for (int b = 0; b < p.B; ++b)
+        if (seq_n(p, b) > 0) row_tiles += (p.rows + BM - 1) / BM;
+    return row_tiles > 0 ? max(1, G / row_tiles) : 1;
+}
+// `par`: column tile width (triangular segment) or wanted column tiles per row tile (cross)
+__device__ __forceinline__ int seg_tiles(const GramProblem& p, int par) {
     int total = 0;
     for (int b = 0; b < p.B; ++b) {
         const int n = seq_n(p, b);
         if (n <= 0) continue;
-        if (p.tri) total += tri_tiles(n, tw);
+        if (p.tri) total += tri_tiles(n, par);
         else {
             int nct, w;
-            cross_cols(n, nct, w);
+            cross_cols(n, par, nct, w);
             total += ((p.rows + BM - 1) / BM) * nct;
         }
     }
     return total;
 }
 // tile `id` of segment p -> piece; false when id is past the segment's last tile
-__device__ __forceinline__ bool decode_tile(const GramProblem& p, int tw, int id, Piece& t) {
+__device__ __forceinline__ bool decode_tile(const GramProblem& p, int par, int id, Piece& t) {
+    const int tw = par;
     for (int b = 0; b < p.B; ++b) {
         const int n = seq_n(p, b);
         if (n <= 0) continue;
         int cnt, nct = 0, w = 0;
         if (p.tri) cnt = tri_tiles(n, tw);
         else {
-            cross_cols(n, nct, w);
+            cross_cols(n, par, nct, w);
             cnt = ((p.rows + BM - 1) / BM) * nct;
         }
         if (id >= cnt) { id -= cnt; continue; }
@@ -98,7 +112,12 @@ __device__ __forceinline__ bool decode_tile(const GramProblem& p, int tw, int id
         int nc;
         if (p.tri) {
             int mi, nj;
-            if (tw == BM) {                              // row tile mi holds tiles mi(mi+1)/2 ... + mi
+            if (tw == BM / 2) {                          // row tile mi holds tiles mi(mi+1) ... + 2mi+1
+                mi = (int)((sqrtf(4.0f * (float)id + 1.0f) - 1.0f) * 0.5f);
+                while (mi * (mi + 1) > id) --mi;
+                while ((mi + 1) * (mi + 2) <= id) ++mi;
+                nj = id - mi * (mi + 1);
+            } else if (tw == BM) {                       // row tile mi holds tiles mi(mi+1)/2 ... + mi
                 mi = (int)((sqrtf(8.0f * (float)id + 1.0f) - 1.0f) * 0.5f);
                 while (mi * (mi + 1) / 2 > id) --mi;
                 while ((mi + 1) * (mi + 2) / 2 <= id) ++mi;
@@ -159,13 +178,22 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (threadIdx.x == 64) {
-        // a triangular problem too small to give every CTA a 256-wide tile is cut 128 wide
+        // a triangular problem too small to give every CTA a 256-wide tile is cut 128 or 64 wide
         int tw = BN;
         int t0 = seg_tiles(seg0, tw);
-        if (seg0.tri && t0 < (int)gridDim.x) { tw = BM; t0 = seg_tiles(seg0, tw); }
-        sh.tw0 = tw;
+        // (narrower tiles move fewer bytes per K block and finish sooner) as long as that
+        // still fits in one round of the grid
+        if (seg0.tri && 2 * t0 < (int)gridDim.x) { tw = BM; t0 = seg_tiles(seg0, tw); }
+        if (seg0.tri && 2 * t0 < (int)gridDim.x) { tw = BM / 2; t0 = seg_tiles(seg0, tw); }
+        if (!seg0.tri) { tw = cross_want(seg0, gridDim.x); t0 = seg_tiles(seg0, tw); }
+        sh.par0 = tw;
         sh.tiles0 = t0;
-        sh.tiles1 = nseg > 1 ? seg_tiles(seg1, BN) : 0;
+        sh.par1 = 1;
+        sh.tiles1 = 0;
+        if (nseg > 1) {
+            sh.par1 = seg1.tri ? BN : cross_want(seg1, gridDim.x);
+            sh.tiles1 = seg_tiles(seg1, sh.par1);
+        }
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -177,7 +205,7 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
     __syncthreads();
     tcgen05_fence_after();
     const unsigned tmem_base = sh.tmem_base;
-    const int tiles0 = sh.tiles0, total = sh.tiles0 + sh.tiles1, tw0 = sh.tw0;
+    const int tiles0 = sh.tiles0, total = sh.tiles0 + sh.tiles1, par0 = sh.par0, par1 = sh.par1;
     Piece pc;
 
     if (warp == 0) {
@@ -191,7 +219,7 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
             for (int id = blockIdx.x; ok && id < total; id += gridDim.x) {
                 const int sg = id < tiles0 ? 0 : 1;
                 const GramProblem& p = sg ? seg1 : seg0;
-                if (!decode_tile(p, tw0, id - (sg ? tiles0 : 0), pc)) break;
+                if (!decode_tile(p, sg ? par1 : par0, id - (sg ? tiles0 : 0), pc)) break;
                 const int num_kb = (p.d + BK - 1) / BK;
                 const int nbox = (pc.ncols + BOX_N - 1) / BOX_N;
                 const int sb = stage_bytes(pc.ncols);
@@ -234,7 +262,7 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
             for (int id = blockIdx.x; ok && id < total; id += gridDim.x, ++tile_it) {
                 const int sg = id < tiles0 ? 0 : 1;
                 const GramProblem& p = sg ? seg1 : seg0;
-                if (!decode_tile(p, tw0, id - (sg ? tiles0 : 0), pc)) break;
+                if (!decode_tile(p, sg ? par1 : par0, id - (sg ? tiles0 : 0), pc)) break;
                 const int num_kb = (p.d + BK - 1) / BK;
                 const int sb = stage_bytes(pc.ncols);
                 if (sb != cur_sb) { cur_sb = sb; cur_nst = stage_count(sb); s = 0; }
@@ -278,7 +306,7 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
         for (int id = blockIdx.x; id < total; id += gridDim.x, ++tile_it) {
             const int sg = id < tiles0 ? 0 : 1;
             const GramProblem& p = sg ? seg1 : seg0;
-            if (!decode_tile(p, tw0, id - (sg ? tiles0 : 0), pc)) break;
+            if (!decode_tile(p, sg ? par1 : par0, id - (sg ? tiles0 : 0), pc)) break;
             const unsigned acc = tile_it & 1u, acc_ph = (tile_it >> 1) & 1u;
             const int64_t o = (int64_t)pc.b * p.cap;
             const int ncols = pc.ncols;

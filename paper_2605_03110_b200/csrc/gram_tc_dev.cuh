@@ -37,7 +37,7 @@ struct alignas(16) Shared {
     unsigned long long drain;
     unsigned tmem_base;
     int abort_flag;
-    int tiles0, tiles1, tw0;
+    int tiles0, tiles1, par0, par1;
     // per epilogue warp, so that staging needs no barrier across warps
     alignas(16) float col_scale[4][BN];
     alignas(16) int col_token[4][BN];
