@@ -166,6 +166,8 @@ def main():
     ap.add_argument("--ref-warmup", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cooperative", action="store_true",
+                    help="launch the fused cascade kernel as an ordinary grid (for profilers)")
     ap.add_argument("--no-graph", action="store_true",
                     help="launch every call from Python instead of replaying a CUDA graph of one step")
     args = ap.parse_args()
@@ -203,6 +205,8 @@ def main():
     B, T, d, L = cfg.B, cfg.T, cfg.d, cfg.L
     ctx = ada.ada_create(B, T, d, ada.ADA_BF16 if cfg.dtype == "bf16" else ada.ADA_F32, device=local)
     ada.ada_set_engine(ctx, args.engine)
+    if args.no_cooperative:
+        ada.ada_set_cooperative(ctx, False)
     stream = torch.cuda.current_stream()
 
     i32 = dict(dtype=torch.int32, device=dev)

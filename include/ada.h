@@ -84,6 +84,13 @@ ada_status ada_create(ada_ctx** out, int device, int64_t maxB, int64_t maxT, int
                       ada_dtype dt);
 ada_status ada_destroy(ada_ctx* ctx);
 ada_status ada_set_engine(ada_ctx* ctx, ada_engine e);
+/* The fused cascade launch has CTAs that wait on results of other CTAs of the same grid, so
+ * it is launched cooperatively (the driver guarantees that all CTAs are resident, or refuses
+ * the launch).  on = 0 launches it as an ordinary grid of one CTA per SM instead: same
+ * kernel and results, but if other work keeps some SMs busy for long the in-kernel waits
+ * can expire (ADA_ERR_TIMEOUT).  Meant for profilers that cannot replay cooperative
+ * launches.  Default: on. */
+ada_status ada_set_cooperative(ada_ctx* ctx, int on);
 
 /*
  * Row normalisation and representative gather (Section 2.1; Algorithm 1

@@ -54,7 +54,8 @@ bool use_tc(const ada_ctx* ctx, ada_dtype dt) {
 }
 
 // tensor-core launch of one or two segments, in the one-CTA or the pair-CTA form
-cudaError_t launch_tc(ada_ctx* ctx, const GramProblem* tri, const GramProblem* cross, cudaStream_t s) {
+cudaError_t launch_tc(ada_ctx* ctx, const GramProblem* tri, const GramProblem* cross,
+                      const NormJob* norms, cudaStream_t s) {
     bool pair = ctx->engine == ADA_ENGINE_TCGEN05_PAIR;
     if (ctx->engine == ADA_ENGINE_AUTO) {
         // The pair kernel pays off once there are several 256-row tiles per SM pair and a long
@@ -62,12 +63,12 @@ cudaError_t launch_tc(ada_ctx* ctx, const GramProblem* tri, const GramProblem* c
         const GramProblem* p = cross != nullptr ? cross : tri;
         pair = (int64_t)p->B * p->rows >= 8192 && p->d >= 2048;
     }
-    if (pair) return launch_gram_tc2(ctx, tri, cross, s);
-    return launch_gram_tc(ctx, tri, cross, s);
+    if (pair) return launch_gram_tc2(ctx, tri, cross, norms, s);
+    return launch_gram_tc(ctx, tri, cross, norms, s);
 }
 
 cudaError_t run_gram(ada_ctx* ctx, const GramProblem& p, ada_dtype dt, cudaStream_t s) {
-    if (use_tc(ctx, dt)) return p.tri ? launch_tc(ctx, &p, nullptr, s) : launch_tc(ctx, nullptr, &p, s);
+    if (use_tc(ctx, dt)) return p.tri ? launch_tc(ctx, &p, nullptr, nullptr, s) : launch_tc(ctx, nullptr, &p, nullptr, s);
     return launch_gram_ffma(ctx, p, dt, s);
 }
 
@@ -146,6 +147,7 @@ ada_status ada_create(ada_ctx** out, int device, int64_t maxB, int64_t maxT, int
     ctx->engine = ADA_ENGINE_AUTO;
     ctx->stage = nullptr; ctx->stage_bytes = 0; ctx->host_stream = nullptr;
     ctx->tc_attr_set = false;
+    ctx->cooperative = true;
     ctx->tc2_attr_set = false;
     ctx->tc2_pairs = 0;
     cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
@@ -214,6 +216,12 @@ ada_status ada_set_engine(ada_ctx* ctx, ada_engine e) {
     return ADA_OK;
 }
 
+ada_status ada_set_cooperative(ada_ctx* ctx, int on) {
+    if (ctx == nullptr) return ADA_ERR_INVALID_ARG;
+    ctx->cooperative = on != 0;
+    return ADA_OK;
+}
+
 ada_status ada_normalize(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d,
                          int64_t ldx, ada_dtype dt, void* Xhat, float* inv_norm,
                          const int32_t* rep_idx, const int32_t* rep_cnt, void* Xrep,
@@ -244,8 +252,13 @@ ada_status ada_select_full(ada_ctx* ctx, const void* X, int64_t B, int64_t T, in
     const float thr = (float)(1.0 - tau * tau);
 
     // the gamma scratch is zero on entry (workspace invariant kept by the compaction kernels)
-    CU(launch_norm_gather(ctx, X, (int)B, (int)T, (int)d, ldx, dt, ctx->inv_norm, nullptr,
-                          nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, s));
+    // long-K tensor-core launches compute the row norms themselves, hidden behind the MMAs
+    const bool tc = use_tc(ctx, dt), fuse = tc && d >= 2048 && B * T >= 4096;
+    if (!fuse)
+        CU(launch_norm_gather(ctx, X, (int)B, (int)T, (int)d, ldx, dt, ctx->inv_norm, nullptr,
+                              nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, s));
+    NormJob nj;
+    nj.X = X; nj.ldx = ldx; nj.n_rows = B * T; nj.d = (int)d; nj.inv_norm = ctx->inv_norm;
     GramProblem p;
     memset(&p, 0, sizeof(p));
     p.A = X; p.Bm = X;
@@ -256,7 +269,9 @@ ada_status ada_select_full(ada_ctx* ctx, const void* X, int64_t B, int64_t T, in
     p.n_dev = nullptr; p.n_host = (int)T;
     p.rows = (int)T; p.cap = (int)T; p.d = (int)d; p.B = (int)B;
     p.tri = 1;
-    CU(run_gram(ctx, p, dt, s));
+    p.wait_norm_a = p.wait_norm_b = fuse ? 1 : 0;
+    if (tc) CU(launch_tc(ctx, &p, nullptr, fuse ? &nj : nullptr, s));
+    else CU(run_gram(ctx, p, dt, s));
     CU(launch_compact_full(ctx, (int)B, (int)T, thr, rep_idx, rep_cnt, gamma, s));
     return ADA_OK;
 }
@@ -282,8 +297,13 @@ ada_status ada_cascade_step(ada_ctx* ctx, const void* X, int64_t B, int64_t T, i
     // kept by the compaction kernels).
     // lines 1-2: inverse norms of all rows; inherited list validated, scattered into the role
     // map and its rows gathered into Xrep
-    CU(launch_norm_gather(ctx, X, (int)B, (int)T, (int)d, ldx, dt, ctx->inv_norm, nullptr, rep_in,
-                          rep_in_cnt, ctx->role, ctx->r_eff, ctx->Xrep, ctx->inv_rep, s));
+    // tensor cores: one launch does lines 3-8; for long K it also computes line 1's row norms
+    const bool fuse = use_tc(ctx, dt), fuse_norm = fuse && d >= 2048 && B * T >= 4096;
+    CU(launch_norm_gather(ctx, X, (int)B, (int)T, (int)d, ldx, dt, fuse_norm ? nullptr : ctx->inv_norm,
+                          nullptr, rep_in, rep_in_cnt, ctx->role, ctx->r_eff, ctx->Xrep,
+                          ctx->inv_rep, s));
+    NormJob nj;
+    nj.X = X; nj.ldx = ldx; nj.n_rows = B * T; nj.d = (int)d; nj.inv_norm = ctx->inv_norm;
     // lines 3-4: r x r Gram among inherited reps, max over earlier ones
     GramProblem p;
     memset(&p, 0, sizeof(p));
@@ -295,7 +315,6 @@ ada_status ada_cascade_step(ada_ctx* ctx, const void* X, int64_t B, int64_t T, i
     p.n_dev = ctx->r_eff; p.n_host = 0;
     p.rows = (int)T; p.cap = (int)T; p.d = (int)d; p.B = (int)B;
     p.tri = 1;
-    const bool fuse = use_tc(ctx, dt);   // one launch: the cross epilogues wait for lines 3-5 in-kernel
     if (!fuse) CU(run_gram(ctx, p, dt, s));
     // lines 6-8: cross-Gram of all rows against the valid inherited reps
     GramProblem q;
@@ -314,7 +333,8 @@ ada_status ada_cascade_step(ada_ctx* ctx, const void* X, int64_t B, int64_t T, i
     q.col_token = rep_in;
     q.row_role = ctx->role;
     q.causal = (flags & ADA_CROSS_CAUSAL) ? 1 : 0;
-    if (fuse) CU(launch_tc(ctx, &p, &q, s));
+    q.wait_norm_a = fuse_norm ? 1 : 0;
+    if (fuse) CU(launch_tc(ctx, &p, &q, fuse_norm ? &nj : nullptr, s));
     else CU(run_gram(ctx, q, dt, s));
     // lines 5, 9, 10-11
     CU(launch_compact_cascade(ctx, (int)B, (int)T, thr, rep_out, rep_out_cnt, add_idx, add_cnt,

@@ -61,6 +61,20 @@ struct GramProblem {
     const int32_t* col_token; // [B*cap] token index of each column (causal) or NULL
     const int32_t* row_role;  // [B*cap] 0 for non-representatives
     int causal;
+    // set when inv_a / inv_b are produced inside the same launch (NormJob): the epilogue
+    // waits for the norm warps before it reads them
+    int wait_norm_a, wait_norm_b;
+};
+
+// Row norms computed inside a tensor-core Gram launch by four extra warps per CTA
+// (Section 2.1; Algorithm 1 line 1): inv_norm[row] = 1/||x_row|| for all n_rows rows of X.
+// X == NULL: nothing to do.
+struct NormJob {
+    const void* X;
+    int64_t ldx;
+    int64_t n_rows;
+    int d;
+    float* inv_norm;
 };
 
 struct Profiler {
@@ -81,6 +95,7 @@ struct ada_ctx {
     ada_engine engine;
     int sm_count;
     bool tc_attr_set;
+    bool cooperative;    // fused launches use the cooperative attribute
     bool tc2_attr_set;   // pair-CTA kernel configured
     int tc2_pairs;       // clusters of two that fit on the device at once
     // device workspace
@@ -127,11 +142,11 @@ cudaError_t launch_gram_ffma(ada_ctx* ctx, const GramProblem& p, ada_dtype dt, c
 
 // gram_tc.cu (bf16, tcgen05 + TMA)
 cudaError_t launch_gram_tc(ada_ctx* ctx, const GramProblem* tri, const GramProblem* cross,
-                           cudaStream_t s);
+                           const NormJob* norms, cudaStream_t s);
 bool gram_tc_available();
 
 // gram_tc2.cu (bf16, tcgen05.cta_group::2: two CTAs per 256-row tile)
 cudaError_t launch_gram_tc2(ada_ctx* ctx, const GramProblem* tri, const GramProblem* cross,
-                            cudaStream_t s);
+                            const NormJob* norms, cudaStream_t s);
 
 }  // namespace ada

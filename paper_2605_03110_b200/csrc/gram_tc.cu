@@ -6,7 +6,7 @@
 // admissible columns j (Definition 1; Algorithm 1 lines 3-4 and 7-8).  Both operands
 // are row-major (K-major) bf16 matrices, so G = A B^T needs no transpose.
 //
-// One persistent CTA per SM, 192 threads:
+// One persistent CTA per SM, 14 warps:
 //   warp 0      TMA producer: one lane issues cp.async.bulk.tensor loads of a 128 x 64
 //               A box and up to four 64 x 64 B boxes per K block into a ring of 4 to 9
 //               stages (fewer bytes per stage for narrow tiles, hence more K blocks in
@@ -19,6 +19,9 @@
 //   warps 2..5  epilogue: tcgen05.ld 32 lanes x 32 columns at a time (one accumulator
 //               row per thread, so the row maximum is thread-local), then one
 //               atomicMax per row and tile on the IEEE bit pattern (values are >= 0).
+//   warps 6..13 optional row norms (Section 2.1): 1/||x_t|| of every row of X with plain
+//               128-bit loads, overlapped with the main loops; the epilogues wait (bounded)
+//               for them before they scale, so a long-K call needs no separate norm pass
 // Every wait is bounded: when a limit expires the CTA raises the context's TIMEOUT
 // status, drains its own outstanding copies and MMAs (again bounded), frees its TMEM
 // and returns.
@@ -153,7 +156,8 @@ struct GramMaps {
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramProblem seg0,
-          const __grid_constant__ GramProblem seg1, const int nseg, unsigned* __restrict__ dep_ctr,
+          const __grid_constant__ GramProblem seg1, const int nseg,
+          const __grid_constant__ NormJob norms, unsigned* __restrict__ dep_ctr,
           unsigned* __restrict__ status) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>(
@@ -295,13 +299,15 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
                 if (global_ns() - t0 > WAIT_LIMIT_NS / 2) { *abort_flag = 8; break; }
             }
         }
-    } else {
+    } else if (warp < 6) {
         // ------------------------------------------------ epilogue (warps 2..5)
         const int quad = warp & 3;                    // TMEM lane quadrant this warp may read
         float* cs = sh.col_scale[warp - 2];
         int* ct = sh.col_token[warp - 2];
         const unsigned dep_total = 4u * (unsigned)tiles0;
-        bool dep_ok = !(nseg > 1 && tiles0 > 0);      // cross epilogues must see segment 0 finished
+        bool dep_ok = !(nseg > 1 && tiles0 > 0);
+        bool norm_ok = norms.X == nullptr;           // row norms computed by this launch's norm warps
+        const unsigned norm_total = (unsigned)(gridDim.x * NORM_WARPS);      // cross epilogues must see segment 0 finished
         unsigned tile_it = 0;
         for (int id = blockIdx.x; id < total; id += gridDim.x, ++tile_it) {
             const int sg = id < tiles0 ? 0 : 1;
@@ -312,22 +318,13 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
             const int ncols = pc.ncols;
             const int ncols32 = (ncols + 31) & ~31;   // TMEM is read 32 columns at a time
             if (sg == 1 && !dep_ok) {
-                // bounded wait for every triangular tile of this launch (line 5 before line 7)
-                int good = 1;
-                if (lane == 0) {
-                    const unsigned long long t0 = global_ns();
-                    unsigned seen;
-                    while (true) {
-                        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(dep_ctr) : "memory");
-                        if (seen >= dep_total) break;
-                        if (*abort_flag != 0) { good = 0; break; }
-                        if (global_ns() - t0 > WAIT_LIMIT_NS) { *abort_flag = 5; good = 0; break; }
-                        __nanosleep(64);
-                    }
-                }
-                good = __shfl_sync(0xffffffffu, good, 0);
-                if (!good) break;
+                // every triangular tile of this launch first (line 5 before line 7)
+                if (!wait_counter(dep_ctr, dep_total, lane, abort_flag, 5)) break;
                 dep_ok = true;
+            }
+            if (p.wait_norm_b && !norm_ok) {
+                if (!wait_counter(dep_ctr + 1, norm_total, lane, abort_flag, 9)) break;
+                norm_ok = true;
             }
             // stage this tile's column factors (0 for inadmissible columns); warp-private copy
             __syncwarp();
@@ -336,7 +333,7 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
                 float f = 0.f;
                 int tok = col;
                 if (c < ncols && col < pc.n) {
-                    f = p.inv_b[o + col];
+                    f = __ldcg(p.inv_b + o + col);
                     if (!p.tri) {
                         // representative removed at line 5 (written earlier in this launch: read at L2)
                         if (!(__ldcg(p.col_gate + o + col) < p.thr_bits)) f = 0.f;
@@ -378,10 +375,14 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
             tcgen05_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh.tmem_empty[acc]);
+            if (p.wait_norm_a && !norm_ok) {
+                if (!wait_counter(dep_ctr + 1, norm_total, lane, abort_flag, 9)) break;
+                norm_ok = true;
+            }
             if (row < pc.m) {
                 const bool skip = !p.tri && p.row_role[o + row] != 0;   // inherited reps are not candidates
                 if (!skip) {
-                    mx *= p.inv_a[o + row];
+                    mx *= __ldcg(p.inv_a + o + row);
                     if (mx > 0.f) atomicMax(p.out + o + row, __float_as_uint(mx));
                 }
             }
@@ -392,6 +393,10 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
                 if (lane == 0) atomicAdd(dep_ctr, 1u);
             }
         }
+    } else if (norms.X != nullptr) {
+        // ------------------------------------------------ row norms (warps 6 and up)
+        norm_rows(norms, blockIdx.x * NORM_WARPS + (warp - 6), gridDim.x * NORM_WARPS, lane,
+                  dep_ctr + 1, status);
     }
 
     tcgen05_fence_before();
@@ -415,7 +420,7 @@ bool gram_tc_available() { return encode_fn() != nullptr; }
 // tri and/or cross may be NULL.  With both, the cross epilogues wait inside the kernel for the
 // triangular segment (ctx->tile_ctr must be zero at launch) and the launch is cooperative.
 cudaError_t launch_gram_tc(ada_ctx* ctx, const GramProblem* tri, const GramProblem* cross,
-                           cudaStream_t s) {
+                           const NormJob* norms, cudaStream_t s) {
     if (!ctx->tc_attr_set) {
         cudaError_t e = cudaFuncSetAttribute(k_gram_tc, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              SMEM_BYTES);
@@ -442,6 +447,9 @@ cudaError_t launch_gram_tc(ada_ctx* ctx, const GramProblem* tri, const GramProbl
     }
     if (nseg == 0) return cudaSuccess;
     if (nseg == 1) { maps.a[1] = maps.a[0]; maps.b[1] = maps.b[0]; segs[1] = segs[0]; segs[1].B = 0; }
+    NormJob nj;
+    memset(&nj, 0, sizeof(nj));
+    if (norms != nullptr) nj = *norms;
     const bool fused = nseg == 2;
     prof_begin(ctx, fused ? K_GRAM_TC_CASCADE : (segs[0].tri ? K_GRAM_TC_TRI : K_GRAM_TC_CROSS), s);
     cudaLaunchConfig_t cfg;
@@ -454,8 +462,8 @@ cudaError_t launch_gram_tc(ada_ctx* ctx, const GramProblem* tri, const GramProbl
     attr[0].id = cudaLaunchAttributeCooperative;
     attr[0].val.cooperative = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = fused ? 1 : 0;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, k_gram_tc, maps, segs[0], segs[1], nseg, ctx->tile_ctr,
+    cfg.numAttrs = (fused && ctx->cooperative) ? 1 : 0;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, k_gram_tc, maps, segs[0], segs[1], nseg, nj, ctx->tile_ctr,
                                        ctx->status);
     prof_end(ctx, s);
     return e;

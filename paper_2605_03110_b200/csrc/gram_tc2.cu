@@ -160,7 +160,8 @@ struct GramMaps {
 // ---------------------------------------------------------------- the kernel
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramProblem seg0,
-           const __grid_constant__ GramProblem seg1, const int nseg, unsigned* __restrict__ dep_ctr,
+           const __grid_constant__ GramProblem seg1, const int nseg,
+          const __grid_constant__ NormJob norms, unsigned* __restrict__ dep_ctr,
            unsigned* __restrict__ status) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>(
@@ -289,13 +290,15 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
                 if (global_ns() - t0 > WAIT_LIMIT_NS / 2) { *abort_flag = 8; break; }
             }
         }
-    } else {
+    } else if (warp < 6) {
         // ------------------------------------------------ epilogue (warps 2..5, both CTAs)
         const int quad = warp & 3;
         float* cs = sh.col_scale[warp - 2];
         int* ct = sh.col_token[warp - 2];
         const unsigned dep_total = 8u * (unsigned)tiles0;
         bool dep_ok = !(nseg > 1 && tiles0 > 0);
+        bool norm_ok = norms.X == nullptr;           // row norms computed by this launch's norm warps
+        const unsigned norm_total = (unsigned)(gridDim.x * NORM_WARPS);
         // the accumulator goes back to the leader's barrier
         const unsigned empty_addr[2] = {map_to_cta(smem_u32(&sh.tmem_empty[0]), 0),
                                         map_to_cta(smem_u32(&sh.tmem_empty[1]), 0)};
@@ -308,21 +311,13 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
             const int64_t o = (int64_t)pc.b * p.cap;
             const int ncols = pc.ncols;
             if (sg == 1 && !dep_ok) {
-                int good = 1;
-                if (lane == 0) {
-                    const unsigned long long t0 = global_ns();
-                    unsigned seen;
-                    while (true) {
-                        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(dep_ctr) : "memory");
-                        if (seen >= dep_total) break;
-                        if (*abort_flag != 0) { good = 0; break; }
-                        if (global_ns() - t0 > WAIT_LIMIT_NS) { *abort_flag = 5; good = 0; break; }
-                        __nanosleep(64);
-                    }
-                }
-                good = __shfl_sync(0xffffffffu, good, 0);
-                if (!good) break;
+                // every triangular tile of this launch first (line 5 before line 7)
+                if (!wait_counter(dep_ctr, dep_total, lane, abort_flag, 5)) break;
                 dep_ok = true;
+            }
+            if (p.wait_norm_b && !norm_ok) {
+                if (!wait_counter(dep_ctr + 1, norm_total, lane, abort_flag, 9)) break;
+                norm_ok = true;
             }
             __syncwarp();
             for (int c = lane; c < ncols; c += 32) {
@@ -330,7 +325,7 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
                 float f = 0.f;
                 int tok = col;
                 if (col < pc.n) {
-                    f = p.inv_b[o + col];
+                    f = __ldcg(p.inv_b + o + col);
                     if (!p.tri) {
                         if (!(__ldcg(p.col_gate + o + col) < p.thr_bits)) f = 0.f;
                         if (p.causal) tok = p.col_token[o + col];
@@ -370,10 +365,14 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
             tcgen05_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_remote(empty_addr[acc]);
+            if (p.wait_norm_a && !norm_ok) {
+                if (!wait_counter(dep_ctr + 1, norm_total, lane, abort_flag, 9)) break;
+                norm_ok = true;
+            }
             if (row < pc.m) {
-                const bool skip = !p.tri && p.row_role[o + row] != 0;
+                const bool skip = !p.tri && p.row_role[o + row] != 0;   // inherited reps are not candidates
                 if (!skip) {
-                    mx *= p.inv_a[o + row];
+                    mx *= __ldcg(p.inv_a + o + row);
                     if (mx > 0.f) atomicMax(p.out + o + row, __float_as_uint(mx));
                 }
             }
@@ -383,6 +382,10 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
                 if (lane == 0) atomicAdd(dep_ctr, 1u);
             }
         }
+    } else if (norms.X != nullptr) {
+        // ------------------------------------------------ row norms (warps 6 and up)
+        norm_rows(norms, blockIdx.x * NORM_WARPS + (warp - 6), gridDim.x * NORM_WARPS, lane,
+                  dep_ctr + 1, status);
     }
 
     tcgen05_fence_before();
@@ -405,7 +408,7 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
 // Pair-CTA launch.  tri and/or cross may be NULL; with both the cross epilogues wait in-kernel
 // for the triangular segment (ctx->tile_ctr must be zero at launch).
 cudaError_t launch_gram_tc2(ada_ctx* ctx, const GramProblem* tri, const GramProblem* cross,
-                            cudaStream_t s) {
+                            const NormJob* norms, cudaStream_t s) {
     if (!ctx->tc2_attr_set) {
         cudaError_t e = cudaFuncSetAttribute(k_gram_tc2, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              SMEM_BYTES);
@@ -445,6 +448,9 @@ cudaError_t launch_gram_tc2(ada_ctx* ctx, const GramProblem* tri, const GramProb
     }
     if (nseg == 0) return cudaSuccess;
     if (nseg == 1) { maps.a[1] = maps.a[0]; maps.b[1] = maps.b[0]; segs[1] = segs[0]; segs[1].B = 0; }
+    NormJob nj;
+    memset(&nj, 0, sizeof(nj));
+    if (norms != nullptr) nj = *norms;
     const bool fused = nseg == 2;
     prof_begin(ctx, fused ? K_GRAM_TC_CASCADE : (segs[0].tri ? K_GRAM_TC_TRI : K_GRAM_TC_CROSS), s);
     cudaLaunchConfig_t cfg;
@@ -459,8 +465,8 @@ cudaError_t launch_gram_tc2(ada_ctx* ctx, const GramProblem* tri, const GramProb
     attr[1].id = cudaLaunchAttributeCooperative;
     attr[1].val.cooperative = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = fused ? 2 : 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, k_gram_tc2, maps, segs[0], segs[1], nseg, ctx->tile_ctr,
+    cfg.numAttrs = (fused && ctx->cooperative) ? 2 : 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, k_gram_tc2, maps, segs[0], segs[1], nseg, nj, ctx->tile_ctr,
                                        ctx->status);
     prof_end(ctx, s);
     return e;

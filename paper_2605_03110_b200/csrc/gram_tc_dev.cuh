@@ -20,7 +20,8 @@ static constexpr int UMMA_K = 16;
 static constexpr int A_BYTES = BM * BK * 2;                 // 16 KiB
 static constexpr int BOX_N = 64;                            // B rows per TMA box
 static constexpr int BOX_BYTES = BOX_N * BK * 2;            // 8 KiB
-static constexpr int NUM_THREADS = 192;
+static constexpr int NORM_WARPS = 8;
+static constexpr int NUM_THREADS = 192 + 32 * NORM_WARPS;   // producer, MMA, 4 epilogue warps, norm warps
 static constexpr int TMEM_COLS = 512;
 static constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // 2 s
 
@@ -200,6 +201,77 @@ static inline bool make_map(CUtensorMap* map, const void* base, int d, int rows,
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+
+// ---------------------------------------------------------------- in-launch row norms
+// bf16 pairs are the halves of 32-bit words; a bf16 is the upper half of an fp32
+static __device__ __forceinline__ float sumsq_bf16x8(const uint4& v) {
+    float s = 0.f;
+    const unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xffff0000u);
+        s = fmaf(lo, lo, s);
+        s = fmaf(hi, hi, s);
+    }
+    return s;
+}
+// Executed by the norm warps of every CTA: warp `w` of `nw` takes rows w, w+nw, ...; when a
+// warp has stored its last row it bumps the counter, so counter == nw means "all rows done".
+static __device__ __forceinline__ void norm_rows(const NormJob& job, int w, int nw, int lane,
+                                                 unsigned* counter, unsigned* status) {
+    const int nvec = job.d >> 3;
+    const __nv_bfloat16* X = reinterpret_cast<const __nv_bfloat16*>(job.X);
+    for (int64_t row = w; row < job.n_rows; row += nw) {
+        const uint4* src = reinterpret_cast<const uint4*>(X + row * job.ldx);
+        // eight independent 128-bit loads in flight per lane: these few warps have to cover
+        // the memory latency that a dedicated kernel would hide with occupancy
+        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+        int v = lane;
+        for (; v + 224 < nvec; v += 256) {
+            uint4 x[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) x[q] = __ldg(src + v + 32 * q);
+#pragma unroll
+            for (int q = 0; q < 8; q += 4) {
+                s0 += sumsq_bf16x8(x[q]); s1 += sumsq_bf16x8(x[q + 1]);
+                s2 += sumsq_bf16x8(x[q + 2]); s3 += sumsq_bf16x8(x[q + 3]);
+            }
+        }
+        for (; v < nvec; v += 32) s0 += sumsq_bf16x8(__ldg(src + v));
+        float ss = (s0 + s1) + (s2 + s3);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        float inv = 0.f;
+        if (!(ss <= 3.0e38f)) {
+            if (lane == 0) atomicOr(status, ST_NONFINITE);
+        } else if (ss > 0.f) {
+            inv = 1.0f / sqrtf(ss);
+        } else if (lane == 0) {
+            atomicAdd(status + 1, 1u);
+        }
+        if (lane == 0) job.inv_norm[row] = inv;
+    }
+    __threadfence();
+    __syncwarp();
+    if (lane == 0) atomicAdd(counter, 1u);
+}
+// Bounded, warp-uniform wait until a global counter reaches `target`.
+static __device__ __forceinline__ bool wait_counter(const unsigned* counter, unsigned target, int lane,
+                                                    volatile int* abort_flag, int where) {
+    int good = 1;
+    if (lane == 0) {
+        const unsigned long long t0 = global_ns();
+        unsigned seen;
+        while (true) {
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
+            if (seen >= target) break;
+            if (*abort_flag != 0) { good = 0; break; }
+            if (global_ns() - t0 > WAIT_LIMIT_NS) { *abort_flag = where; good = 0; break; }
+            __nanosleep(64);
+        }
+    }
+    return __shfl_sync(0xffffffffu, good, 0) != 0;
+}
 
 }  // namespace tc
 }  // namespace ada

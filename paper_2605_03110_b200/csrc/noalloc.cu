@@ -51,6 +51,7 @@ ada_status setup_device(int device, PerDevice** out) {
         c.maxd = 0;
         c.engine = ADA_ENGINE_AUTO;
         c.tc_attr_set = false;
+        c.cooperative = true;
         c.tc2_attr_set = false;
         c.tc2_pairs = 0;
         c.ws = nullptr;
@@ -118,7 +119,7 @@ extern "C" ada_status ada_select_full_noalloc(const void* X, int64_t T, int64_t 
     p.rows = (int)T; p.cap = (int)T; p.d = (int)d; p.B = 1;
     p.tri = 1;
     cudaError_t e;
-    if (dt == ADA_BF16 && gram_tc_available()) e = launch_gram_tc(ctx, &p, nullptr, s);
+    if (dt == ADA_BF16 && gram_tc_available()) e = launch_gram_tc(ctx, &p, nullptr, nullptr, s);
     else e = launch_gram_ffma(ctx, p, dt, s);
     if (e != cudaSuccess) return ADA_ERR_CUDA;
     if (launch_compact_full(ctx, 1, (int)T, thr, rep_idx, rep_cnt, gamma, s) != cudaSuccess)

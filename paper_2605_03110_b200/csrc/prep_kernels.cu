@@ -86,6 +86,7 @@ k_norm_gather(const T* __restrict__ X, int64_t n_rows, int Tseq, int d, int64_t 
               float* __restrict__ inv_rep, unsigned* __restrict__ status) {
     const int lane = threadIdx.x & 31;
     int64_t w = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (inv_norm == nullptr && Xhat == nullptr) w += n_rows;   // gather-only launch: list warps only
     constexpr int N = Vec16<T>::N;
     const int nvec = d / N;  // d*es is a multiple of 16 bytes
     if (w < n_rows) {
@@ -129,7 +130,18 @@ k_norm_gather(const T* __restrict__ X, int64_t n_rows, int Tseq, int d, int64_t 
     const uint4* src = reinterpret_cast<const uint4*>(X + ((int64_t)b * Tseq + idx) * ldx);
     uint4* dst = reinterpret_cast<uint4*>(Xrep + prow * (int64_t)d);
     float ss = 0.f;
-    for (int v = lane; v < nvec; v += 32) {
+    int v = lane;
+    for (; v + 224 < nvec; v += 256) {          // eight loads in flight per lane
+        uint4 x[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) x[q] = __ldg(src + v + 32 * q);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            ss += Vec16<T>::sumsq(x[q]);
+            dst[v + 32 * q] = x[q];
+        }
+    }
+    for (; v < nvec; v += 32) {
         const uint4 x = __ldg(src + v);
         ss += Vec16<T>::sumsq(x);
         dst[v] = x;
@@ -148,7 +160,8 @@ cudaError_t launch_norm_gather(ada_ctx* ctx, const void* X, int B, int T, int d,
                                float* inv_rep, cudaStream_t s) {
     const int64_t n_rows = (int64_t)B * T;
     const int warps = 8;
-    const int64_t n_warps = rep_in != nullptr ? 2 * n_rows : n_rows;
+    const bool gather_only = inv_norm == nullptr && Xhat == nullptr;
+    const int64_t n_warps = (rep_in != nullptr && !gather_only) ? 2 * n_rows : n_rows;
     const unsigned grid = (unsigned)((n_warps + warps - 1) / warps);
     prof_begin(ctx, K_NORM_GATHER, s);
     if (dt == ADA_F32) {
@@ -307,7 +320,8 @@ __global__ void __launch_bounds__(1024) k_compact(const CompactArgs a) {
             for (unsigned q = 0; q < gridDim.y; ++q)
                 for (unsigned j = 0; j < gridDim.x; ++j) a.agg[(int64_t)q * a.agg_stride + j] = 0ull;
             *a.done_ctr = 0u;
-            *a.dep_ctr = 0u;
+            a.dep_ctr[0] = 0u;
+            a.dep_ctr[1] = 0u;   // norm warps' counter of the Gram launch
         }
     }
 }
