@@ -186,18 +186,17 @@ def main():
     import torch
     import torch.distributed as dist
     from paper_2605_03110_b200 import binding as ada
+    from paper_2605_03110_b200 import replicas
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rep = replicas.from_env()
+    rank, world, local = rep.rank, rep.world, rep.local_rank
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+    replicas.init_process_group(rep, "nccl", dev)
     ada.lib()                                                   # fail loudly if not built
 
     # ---- inputs: every rank draws its own replica (weak scaling, no data-path collective) ----
-    host_layers = [lb.X for lb in wl.generate_layers(cfg, seed=rank)]
+    host_layers = [lb.X for lb in wl.generate_layers(cfg, seed=rep.seed)]
     tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
 
     def as_torch(X):
@@ -262,11 +261,7 @@ def main():
         e1.record(stream)
         barrier()
         clocks = sampler.finish()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = replicas.max_over_ranks(rep, e0.elapsed_time(e1), dev)
         return ms / steps, clocks
 
     # ---- headline: cascade pipeline, inputs resident in HBM ----
@@ -288,7 +283,7 @@ def main():
         stream = torch.cuda.current_stream()
         step_fn, indep_fn = g_casc.replay, g_ind.replay
     ms_step, clocks = timed(step_fn, args.steps, args.warmup)
-    value = world * B * T * L / (ms_step * 1e-3)
+    value = replicas.whole_job_throughput(rep, B * T * L, ms_step * 1e-3)
 
     # ---- independent selection (full Gram at every layer) for the cascade speedup ----
     ms_indep, _ = timed(indep_fn, max(3, args.steps // 2), 3)
@@ -389,15 +384,13 @@ def main():
             e2e_pipeline()
         barrier()
         n_e2e = max(3, args.steps // 2)
-        t0 = time.perf_counter()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)                       # the host calls run on this stream and wait for it
         for _ in range(n_e2e):
             e2e_pipeline()
-        torch.cuda.synchronize()
-        t_e2e = (time.perf_counter() - t0) / n_e2e
-        if world > 1:
-            t = torch.tensor([t_e2e], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            t_e2e = float(t.item())
+        e1.record(stream)
+        barrier()
+        t_e2e = replicas.max_over_ranks(rep, e0.elapsed_time(e1) * 1e-3 / n_e2e, dev)
         n_tok = B * T
         h2d = L * n_tok * d * es + (L - 1) * (n_tok * 4 + B * 4)
         d2h = (n_tok * 4 + B * 4) + (L - 1) * 3 * (n_tok * 4 + B * 4)

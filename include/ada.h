@@ -139,19 +139,21 @@ ada_status ada_cascade_step(ada_ctx* ctx, const void* X, int64_t B, int64_t T, i
                             int32_t* rem_cnt, float* gamma_rep, float* gamma_cross,
                             uint32_t flags, void* stream);
 
-/* Same operations with HOST buffers: inputs are copied to the device, the
- * device-pointer call above runs, results are copied back, and the call
- * returns after synchronising its own stream.  Counts are int32[B] on the
- * host.  The context must have been created with maxima covering the sizes. */
+/* Same operations with HOST buffers: inputs are copied to the device (staging
+ * buffers owned by the context, allocated on first use), the device-pointer
+ * call above runs, results are copied back, all on `stream`, and the call
+ * returns after synchronising that stream.  Counts are int32[B] on the host.
+ * Pinned host memory makes the copies asynchronous DMA transfers.  The context
+ * must have been created with maxima covering the sizes. */
 ada_status ada_select_full_host(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d,
                                 ada_dtype dt, double tau, int32_t* rep_idx, int32_t* rep_cnt,
-                                float* gamma);
+                                float* gamma, void* stream);
 ada_status ada_cascade_step_host(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d,
                                  ada_dtype dt, double tau, const int32_t* rep_in,
                                  const int32_t* rep_in_cnt, int32_t* rep_out,
                                  int32_t* rep_out_cnt, int32_t* add_idx, int32_t* add_cnt,
                                  int32_t* rem_idx, int32_t* rem_cnt, float* gamma_rep,
-                                 float* gamma_cross, uint32_t flags);
+                                 float* gamma_cross, uint32_t flags, void* stream);
 
 /*
  * Full selection for callers that cannot allocate device memory (the paper has no

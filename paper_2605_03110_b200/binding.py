@@ -57,10 +57,10 @@ def lib() -> C.CDLL:
         L.ada_cascade_step.argtypes = [vp, vp, i64, i64, i64, i64, C.c_int, C.c_double,
                                        i32p, i32p, i32p, i32p, i32p, i32p, i32p, i32p, fp, fp,
                                        C.c_uint32, vp]
-        L.ada_select_full_host.argtypes = [vp, vp, i64, i64, i64, C.c_int, C.c_double, i32p, i32p, fp]
+        L.ada_select_full_host.argtypes = [vp, vp, i64, i64, i64, C.c_int, C.c_double, i32p, i32p, fp, vp]
         L.ada_cascade_step_host.argtypes = [vp, vp, i64, i64, i64, C.c_int, C.c_double,
                                             i32p, i32p, i32p, i32p, i32p, i32p, i32p, i32p, fp, fp,
-                                            C.c_uint32]
+                                            C.c_uint32, vp]
         L.ada_select_full_noalloc.argtypes = [vp, i64, i64, i64, C.c_int, C.c_double, i32p, i32p,
                                               fp, vp]
         L.ada_gram_op_count.argtypes = [C.c_int, i64, i64, i64]
@@ -226,25 +226,27 @@ def ada_cascade_step(ctx: Context, X: torch.Tensor, tau: float, rep_in: torch.Te
 
 
 def ada_select_full_host(ctx: Context, X: torch.Tensor, tau: float, rep_idx: torch.Tensor,
-                         rep_cnt: torch.Tensor, gamma: Optional[torch.Tensor] = None) -> None:
-    """HOST tensors in and out (pinned memory recommended); synchronous."""
+                         rep_cnt: torch.Tensor, gamma: Optional[torch.Tensor] = None,
+                         stream=None) -> None:
+    """HOST tensors in and out (pinned memory recommended); returns after `stream` is idle."""
     X, B, T, d, ldx = _shape(X)
     assert not X.is_cuda and ldx == d
     _check(lib().ada_select_full_host(ctx.h, X.data_ptr(), B, T, d, dtype_of(X), float(tau),
-                                      rep_idx.data_ptr(), rep_cnt.data_ptr(), _ptr(gamma)),
-           "ada_select_full_host")
+                                      rep_idx.data_ptr(), rep_cnt.data_ptr(), _ptr(gamma),
+                                      _stream(stream)), "ada_select_full_host")
 
 
 def ada_cascade_step_host(ctx: Context, X: torch.Tensor, tau: float, rep_in, rep_in_cnt, rep_out,
                           rep_out_cnt, add_idx, add_cnt, rem_idx, rem_cnt, gamma_rep=None,
-                          gamma_cross=None, flags: int = 0) -> None:
+                          gamma_cross=None, flags: int = 0, stream=None) -> None:
     X, B, T, d, ldx = _shape(X)
     assert not X.is_cuda and ldx == d
     _check(lib().ada_cascade_step_host(ctx.h, X.data_ptr(), B, T, d, dtype_of(X), float(tau),
                                        rep_in.data_ptr(), rep_in_cnt.data_ptr(), rep_out.data_ptr(),
                                        rep_out_cnt.data_ptr(), add_idx.data_ptr(), add_cnt.data_ptr(),
                                        rem_idx.data_ptr(), rem_cnt.data_ptr(), _ptr(gamma_rep),
-                                       _ptr(gamma_cross), flags), "ada_cascade_step_host")
+                                       _ptr(gamma_cross), flags, _stream(stream)),
+           "ada_cascade_step_host")
 
 
 def ada_select_full_noalloc(X: torch.Tensor, tau: float, rep_idx: torch.Tensor,

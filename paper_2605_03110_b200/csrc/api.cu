@@ -376,8 +376,6 @@ static ada_status ensure_stage(ada_ctx* ctx) {
         return ADA_ERR_CUDA;
     }
     ctx->stage_bytes = bytes;
-    if (cudaStreamCreateWithFlags(&ctx->host_stream, cudaStreamNonBlocking) != cudaSuccess)
-        return ADA_ERR_CUDA;
     return ADA_OK;
 }
 
@@ -411,7 +409,7 @@ static Stage carve(ada_ctx* ctx) {
 
 ada_status ada_select_full_host(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d,
                                 ada_dtype dt, double tau, int32_t* rep_idx, int32_t* rep_cnt,
-                                float* gamma) {
+                                float* gamma, void* stream) {
     if (ctx == nullptr || X == nullptr || rep_idx == nullptr || rep_cnt == nullptr)
         return ADA_ERR_INVALID_ARG;
     if (B < 1 || T < 1 || d < 1) return ADA_ERR_INVALID_ARG;
@@ -420,7 +418,7 @@ ada_status ada_select_full_host(ada_ctx* ctx, const void* X, int64_t B, int64_t 
     ada_status st = ensure_stage(ctx);
     if (st != ADA_OK) return st;
     Stage sg = carve(ctx);
-    cudaStream_t s = ctx->host_stream;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t n_tok = (size_t)B * T;
     CU(cudaMemcpyAsync(sg.X, X, n_tok * d * ctx->es, cudaMemcpyHostToDevice, s));
     st = ada_select_full(ctx, sg.X, B, T, d, d, dt, tau, sg.l0, sg.c0, gamma ? sg.g0 : nullptr, s);
@@ -437,7 +435,7 @@ ada_status ada_cascade_step_host(ada_ctx* ctx, const void* X, int64_t B, int64_t
                                  const int32_t* rep_in_cnt, int32_t* rep_out,
                                  int32_t* rep_out_cnt, int32_t* add_idx, int32_t* add_cnt,
                                  int32_t* rem_idx, int32_t* rem_cnt, float* gamma_rep,
-                                 float* gamma_cross, uint32_t flags) {
+                                 float* gamma_cross, uint32_t flags, void* stream) {
     if (ctx == nullptr || X == nullptr || rep_in == nullptr || rep_in_cnt == nullptr ||
         rep_out == nullptr || rep_out_cnt == nullptr || add_idx == nullptr ||
         add_cnt == nullptr || rem_idx == nullptr || rem_cnt == nullptr)
@@ -448,7 +446,7 @@ ada_status ada_cascade_step_host(ada_ctx* ctx, const void* X, int64_t B, int64_t
     ada_status st = ensure_stage(ctx);
     if (st != ADA_OK) return st;
     Stage sg = carve(ctx);
-    cudaStream_t s = ctx->host_stream;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t n_tok = (size_t)B * T;
     CU(cudaMemcpyAsync(sg.X, X, n_tok * d * ctx->es, cudaMemcpyHostToDevice, s));
     CU(cudaMemcpyAsync(sg.l0, rep_in, n_tok * 4, cudaMemcpyHostToDevice, s));

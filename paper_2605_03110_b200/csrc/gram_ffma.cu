@@ -59,19 +59,28 @@ k_gram_ffma(const GramProblem p) {
     const T* a_ptr = A + (int64_t)(row0 + lr) * p.lda + lk;
     const T* b_ptr = Bm + (int64_t)(col0 + lr) * p.ldb + lk;
 
+    // software pipeline: the global loads of K block i+1 are in flight while block i is
+    // multiplied out of shared memory
+    float av[4] = {0.f, 0.f, 0.f, 0.f}, bv[4] = {0.f, 0.f, 0.f, 0.f};
+    if (lk < p.d) {                   // d is a multiple of 4: a group of 4 is all in or all out
+        if (a_ok) load4<T>(a_ptr, av);
+        if (b_ok) load4<T>(b_ptr, bv);
+    }
     for (int k0 = 0; k0 < p.d; k0 += BK) {
-        float av[4] = {0.f, 0.f, 0.f, 0.f}, bv[4] = {0.f, 0.f, 0.f, 0.f};
-        if (k0 + lk < p.d) {          // d is a multiple of 4: a group of 4 is all in or all out
-            if (a_ok) load4<T>(a_ptr + k0, av);
-            if (b_ok) load4<T>(b_ptr + k0, bv);
-        }
-        __syncthreads();
+        __syncthreads();              // the previous block has been consumed
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             As[lk + i][lr] = av[i];
             Bs[lk + i][lr] = bv[i];
         }
         __syncthreads();
+        const int kn = k0 + BK + lk;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) av[i] = bv[i] = 0.f;
+        if (kn < p.d) {
+            if (a_ok) load4<T>(a_ptr + k0 + BK, av);
+            if (b_ok) load4<T>(b_ptr + k0 + BK, bv);
+        }
 #pragma unroll
         for (int k = 0; k < BK; ++k) {
             const float4 a4 = *reinterpret_cast<const float4*>(&As[k][ty * 4]);
