@@ -157,6 +157,81 @@ def workload_dict(cfg):
 
 
 # ------------------------------------------------------------------------------------------
+def sweep(args):
+    """configs[4]: d = 4096, bf16, one layer transition X1 = X0 + 0.02 N(0, I); full selection on
+    X1 against one cascade step on X1 from R(X0), per T and r/T.  Times are CUDA-event means over
+    graph replays of ten calls each, with a 256 MiB write before every call so that it starts with a
+    cold L2; the time of the writes alone is measured the same way and subtracted."""
+    import torch
+    from paper_2605_03110_b200 import binding as ada
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    peaks = measured_peaks()
+    steps = max(5, min(args.steps, 20))
+
+    reps = 10
+    side = torch.cuda.Stream()
+
+    def graph_of(fn):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                for _ in range(reps):
+                    flush.zero_()
+                    fn(side)
+        return g
+
+    def time_graph(g):
+        for _ in range(2):
+            g.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / (steps * reps)         # microseconds per call + flush
+
+    t_flush = time_graph(graph_of(lambda st: None))
+
+    def timed_call(fn):
+        fn(None)                                                   # first-call set-up outside capture
+        torch.cuda.synchronize()
+        return time_graph(graph_of(fn)) - t_flush
+
+    print("| T | r/T | r | full us | cascade us | speedup | T/r (paper) | 1/(2q-q^2) | full TFLOP/s | "
+          "cascade: X once GB/s | cascade TFLOP/s |")
+    print("|---|---|---|---|---|---|---|---|---|---|---|")
+    for T in wl.SWEEP_T:
+        ctx = ada.ada_create(1, T, 4096, ada.ADA_BF16)
+        for q in wl.SWEEP_Q:
+            cfg = wl.sweep_config(T, q)
+            X0, X1 = [torch.from_numpy(lb.X.view(np.int16)).view(torch.bfloat16).to(dev)
+                      for lb in wl.generate_layers(cfg, seed=0)]
+            idx, cnt, _ = ada.ada_select_full(ctx, X0, cfg.tau, want_gamma=False)
+            r = int(cnt[0])
+            i2 = torch.empty_like(idx)
+            c2 = torch.empty_like(cnt)
+            out = ada.CascadeOut(1, T, dev, want_gamma=False)
+            t_full = timed_call(lambda st: ada.ada_select_full(ctx, X1, cfg.tau, i2, c2, want_gamma=False,
+                                                               stream=st))
+            t_casc = timed_call(lambda st: ada.ada_cascade_step(ctx, X1, cfg.tau, idx, cnt, out=out,
+                                                                stream=st))
+            d = 4096
+            f_full = d * T * (T - 1.0)
+            f_casc = d * r * (r - 1.0) + 2.0 * d * (T - r) * r
+            qq = r / T
+            print(f"| {T} | {q:g} | {r} | {t_full:.1f} | {t_casc:.1f} | {t_full / t_casc:.2f} | "
+                  f"{T / r:.1f} | {1.0 / (2 * qq - qq * qq):.2f} | {f_full / t_full / 1e6:.0f} | "
+                  f"{T * d * 2 / t_casc / 1e3:.0f} | {f_casc / t_casc / 1e6:.0f} |")
+            sys.stdout.flush()
+        ada.ada_destroy(ctx)
+    print(f"peaks ({peaks['src']}): HBM {peaks['hbm_gbs']} GB/s, bf16 {peaks['bf16_burst']} TFLOP/s burst / "
+          f"{peaks['bf16_sustained']} sustained")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -170,12 +245,18 @@ def main():
     ap.add_argument("--ref-warmup", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--sweep", action="store_true",
+                    help="crossover sweep (configs[4]): full selection vs one cascade step per (T, r/T); "
+                         "prints a table instead of the JSON line")
     ap.add_argument("--no-cooperative", action="store_true",
                     help="launch the fused cascade kernel as an ordinary grid (for profilers)")
     ap.add_argument("--no-graph", action="store_true",
                     help="launch every call from Python instead of replaying a CUDA graph of one step")
     args = ap.parse_args()
 
+    if args.sweep:
+        sweep(args)
+        return
     cfg = wl.CONFIGS[args.workload]
     if args.layers:
         cfg = wl.scaled(cfg, L=args.layers)
