@@ -196,6 +196,13 @@ uint64_t ada_gram_op_count(int cascade, int64_t T, int64_t d, int64_t r);
  * n_zero_norm_rows (optional, host) receives the number of zero rows seen. */
 ada_status ada_device_status(ada_ctx* ctx, void* stream, int64_t* n_zero_norm_rows);
 
+/* Self-test of the bounded-wait machinery: runs a one-warp kernel that waits, with a limit
+ * of `limit_ms` milliseconds, on a counter that nothing ever sets -- the same wait the Gram
+ * kernels use between CTAs.  The wait runs out, the kernel raises the TIMEOUT bit and returns
+ * normally; ada_device_status then reports ADA_ERR_TIMEOUT and the context stays usable.
+ * Nothing faults, traps or hangs. */
+ada_status ada_selftest_wait_timeout(ada_ctx* ctx, int limit_ms, void* stream);
+
 /* Per-kernel timing (for benchmarks): when enabled, every kernel launch of
  * this context is bracketed by CUDA events on the launching stream.
  * ada_profile_read synchronises those events, fills up to `cap` entries

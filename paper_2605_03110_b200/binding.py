@@ -25,7 +25,7 @@ SYMBOLS = [
     "ada_create", "ada_destroy", "ada_set_engine", "ada_normalize", "ada_select_full",
     "ada_cascade_step", "ada_select_full_host", "ada_cascade_step_host", "ada_gram_op_count",
     "ada_device_status", "ada_profile_enable", "ada_profile_read", "ada_status_string",
-    "ada_select_full_noalloc", "ada_set_cooperative",
+    "ada_select_full_noalloc", "ada_set_cooperative", "ada_selftest_wait_timeout",
 ]
 ADA_NOALLOC_MAX_T = 16384
 
@@ -51,6 +51,7 @@ def lib() -> C.CDLL:
         L.ada_destroy.argtypes = [vp]
         L.ada_set_engine.argtypes = [vp, C.c_int]
         L.ada_set_cooperative.argtypes = [vp, C.c_int]
+        L.ada_selftest_wait_timeout.argtypes = [vp, C.c_int, vp]
         L.ada_normalize.argtypes = [vp, vp, i64, i64, i64, i64, C.c_int, vp, fp, i32p, i32p, vp, vp]
         L.ada_select_full.argtypes = [vp, vp, i64, i64, i64, i64, C.c_int, C.c_double, i32p, i32p,
                                       fp, vp]
@@ -149,6 +150,12 @@ def ada_set_engine(ctx: Context, engine: int) -> None:
 
 def ada_set_cooperative(ctx: Context, on: bool) -> None:
     _check(lib().ada_set_cooperative(ctx.h, int(bool(on))), "ada_set_cooperative")
+
+
+def ada_selftest_wait_timeout(ctx: Context, limit_ms: int = 50, stream=None) -> None:
+    """Enqueue the bounded-wait self-test; ada_device_status then reports ADA_ERR_TIMEOUT."""
+    _check(lib().ada_selftest_wait_timeout(ctx.h, int(limit_ms), _stream(stream)),
+           "ada_selftest_wait_timeout")
 
 
 def ada_gram_op_count(cascade: bool, T: int, d: int, r: int = 0) -> int:

@@ -467,6 +467,13 @@ ada_status ada_cascade_step_host(ada_ctx* ctx, const void* X, int64_t B, int64_t
     return ADA_OK;
 }
 
+ada_status ada_selftest_wait_timeout(ada_ctx* ctx, int limit_ms, void* stream) {
+    if (ctx == nullptr || limit_ms < 1 || limit_ms > 2000) return ADA_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    CU(launch_selftest_wait(ctx, limit_ms, static_cast<cudaStream_t>(stream)));
+    return ADA_OK;
+}
+
 ada_status ada_profile_enable(ada_ctx* ctx, int on) {
     if (ctx == nullptr) return ADA_ERR_INVALID_ARG;
     ctx->prof.on = on != 0;

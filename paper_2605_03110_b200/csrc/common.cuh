@@ -144,6 +144,7 @@ cudaError_t launch_gram_ffma(ada_ctx* ctx, const GramProblem& p, ada_dtype dt, c
 cudaError_t launch_gram_tc(ada_ctx* ctx, const GramProblem* tri, const GramProblem* cross,
                            const NormJob* norms, cudaStream_t s);
 bool gram_tc_available();
+cudaError_t launch_selftest_wait(ada_ctx* ctx, int limit_ms, cudaStream_t s);
 
 // gram_tc2.cu (bf16, tcgen05.cta_group::2: two CTAs per 256-row tile)
 cudaError_t launch_gram_tc2(ada_ctx* ctx, const GramProblem* tri, const GramProblem* cross,

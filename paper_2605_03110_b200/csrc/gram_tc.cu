@@ -417,6 +417,28 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
 
 bool gram_tc_available() { return encode_fn() != nullptr; }
 
+namespace {
+// One warp waits on a counter that stays at zero; the limit expires and the status is raised.
+__global__ void k_selftest_wait(const unsigned* counter, unsigned long long limit_ns,
+                                unsigned* status) {
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) abort_flag = 0;
+    __syncwarp();
+    const bool ok = wait_counter(counter, 1u, threadIdx.x & 31, &abort_flag, 11, limit_ns);
+    if (!ok && threadIdx.x == 0) {
+        atomicOr(status, ST_TIMEOUT);
+        status[2] = (unsigned)abort_flag;
+    }
+}
+}  // namespace
+
+cudaError_t launch_selftest_wait(ada_ctx* ctx, int limit_ms, cudaStream_t s) {
+    // tile_ctr[2] is never written by any kernel
+    k_selftest_wait<<<1, 32, 0, s>>>(ctx->tile_ctr + 2, (unsigned long long)limit_ms * 1000000ull,
+                                     ctx->status);
+    return cudaGetLastError();
+}
+
 // tri and/or cross may be NULL.  With both, the cross epilogues wait inside the kernel for the
 // triangular segment (ctx->tile_ctr must be zero at launch) and the launch is cooperative.
 cudaError_t launch_gram_tc(ada_ctx* ctx, const GramProblem* tri, const GramProblem* cross,

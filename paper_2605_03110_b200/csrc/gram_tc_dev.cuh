@@ -257,7 +257,8 @@ static __device__ __forceinline__ void norm_rows(const NormJob& job, int w, int 
 }
 // Bounded, warp-uniform wait until a global counter reaches `target`.
 static __device__ __forceinline__ bool wait_counter(const unsigned* counter, unsigned target, int lane,
-                                                    volatile int* abort_flag, int where) {
+                                                    volatile int* abort_flag, int where,
+                                                    unsigned long long limit_ns = WAIT_LIMIT_NS) {
     int good = 1;
     if (lane == 0) {
         const unsigned long long t0 = global_ns();
@@ -266,7 +267,7 @@ static __device__ __forceinline__ bool wait_counter(const unsigned* counter, uns
             asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
             if (seen >= target) break;
             if (*abort_flag != 0) { good = 0; break; }
-            if (global_ns() - t0 > WAIT_LIMIT_NS) { *abort_flag = where; good = 0; break; }
+            if (global_ns() - t0 > limit_ns) { *abort_flag = where; good = 0; break; }
             __nanosleep(64);
         }
     }

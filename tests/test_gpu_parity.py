@@ -268,6 +268,20 @@ def test_error_paths(ada):
     ada.ada_destroy(ctx)
 
 
+def test_bounded_wait_runs_out_and_the_context_survives(ada):
+    """The in-kernel waits have a limit: a wait on a flag nothing sets ends with a status the
+    host can read (no trap, no hang), and the context keeps working afterwards."""
+    from parity import check_full
+    ctx = ada.ada_create(1, 256, 64, ada.ADA_BF16)
+    ada.ada_selftest_wait_timeout(ctx, limit_ms=50)
+    st, _ = ada.ada_device_status(ctx)
+    assert st == 7 and ada.status_string(st) == "ADA_ERR_TIMEOUT"
+    assert ada.ada_device_status(ctx)[0] == 0                   # reading clears it
+    band, reps = check_full(ctx, clustered(256, 64, 3, "bf16"), TAU)
+    assert len(reps[0]) > 0
+    ada.ada_destroy(ctx)
+
+
 def test_host_entry_points_match_device_ones(ada):
     from parity import lists, to_device
     cfg = wl.scaled(wl.CONFIGS[2], B=3, T=700, d=256, L=2)
