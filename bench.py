@@ -507,7 +507,8 @@ def main():
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16 x bf16 -> f32" if cfg.dtype == "bf16" else "f32",
+            "scaling": "weak", "vs_baseline": None, "dtype": ("bf16 x bf16 -> f32" if cfg.dtype == "bf16" else
+                      ("f32" if args.engine == 1 else "f32 as 3 bf16 terms (6 cross products) -> f32")),
             "data": "synthetic", "config": workload_dict(cfg), "clocks": clocks, "e2e": e2e,
             "gpu_launches": args.steps * sum(k["launches"] for k in kernels.values()),
             "roofline": roofline, "cpu_baseline": cpu_baseline,

@@ -63,11 +63,14 @@ typedef enum { ADA_F32 = 0, ADA_BF16 = 1 } ada_dtype;
 /* flags of ada_cascade_step */
 #define ADA_CROSS_CAUSAL 1u /* restrict Algorithm 1 line 8 to valid representatives s < t */
 
-/* Which Gram kernel family a context uses.  AUTO: tensor cores (tcgen05) for
- * ADA_BF16, fp32 FFMA for ADA_F32.  FFMA may be forced for bf16 input (a slow
- * cross-check of the tensor-core path); the tensor-core forms cannot be forced
- * for fp32.  TCGEN05 is the one-CTA kernel (128-row tiles), TCGEN05_PAIR the
- * two-CTA kernel (cta_group::2, 256-row tiles shared by the two SMs of a TPC). */
+/* Which Gram kernel family a context uses.  AUTO: tensor cores (tcgen05), one- or two-CTA
+ * form by problem size.  ADA_BF16 feeds the stored values to the MMA; ADA_F32 is split into
+ * three bf16 terms per value and contracted as the six leading cross terms (error at fp32
+ * rounding level, fp32 accumulation), at the price of a 6x longer contraction and a
+ * workspace of 48 bytes per element.  FFMA is the plain fp32 ALU kernel (any storage type;
+ * for ADA_BF16 a slow cross-check of the tensor-core path).  TCGEN05 forces the one-CTA
+ * kernel (128-row tiles), TCGEN05_PAIR the two-CTA kernel (cta_group::2, 256-row tiles
+ * shared by the two SMs of a TPC). */
 typedef enum {
     ADA_ENGINE_AUTO = 0,
     ADA_ENGINE_FFMA = 1,
@@ -79,7 +82,8 @@ typedef struct ada_ctx ada_ctx; /* opaque */
 
 /* Create a context on `device` able to serve up to maxB sequences of maxT
  * tokens of width maxd in storage type dt.  Allocates the workspace
- * (cudaMalloc; about maxB*maxT*(maxd*es + 32) bytes).  *out is NULL on error. */
+ * (cudaMalloc; about maxB*maxT*(maxd*es + 32) bytes, plus 48*maxB*maxT*maxd for ADA_F32).
+ * *out is NULL on error. */
 ada_status ada_create(ada_ctx** out, int device, int64_t maxB, int64_t maxT, int64_t maxd,
                       ada_dtype dt);
 ada_status ada_destroy(ada_ctx* ctx);

@@ -13,7 +13,7 @@ namespace {
 
 const char* const kKernelNames[K_COUNT] = {
     "norm_gather",     "gram_ffma_tri",    "gram_ffma_cross",
-    "gram_tc_tri",     "gram_tc_cross",    "gram_tc_cascade", "compact_full",
+    "gram_tc_tri",     "gram_tc_cross",    "gram_tc_cascade", "split_bf16x3",  "compact_full",
     "compact_cascade",
 };
 
@@ -51,6 +51,12 @@ bool use_tc(const ada_ctx* ctx, ada_dtype dt) {
     if (dt != ADA_BF16) return false;
     if (ctx->engine == ADA_ENGINE_FFMA) return false;
     return gram_tc_available();
+}
+
+// fp32 storage on the bf16 tensor cores through the three-term split
+bool use_split(const ada_ctx* ctx, ada_dtype dt) {
+    return dt == ADA_F32 && ctx->engine != ADA_ENGINE_FFMA && ctx->splitXA != nullptr &&
+           gram_tc_available();
 }
 
 // tensor-core launch of one or two segments, in the one-CTA or the pair-CTA form
@@ -163,6 +169,9 @@ ada_status ada_create(ada_ctx** out, int device, int64_t maxB, int64_t maxT, int
     const size_t o_inv = take(n_tok * 4), o_invr = take(n_tok * 4);
     const size_t o_reff = take((size_t)maxB * 4), o_stat = take(32);
     const size_t o_xrep = take(n_tok * (size_t)maxd * ctx->es + 1024);
+    const size_t split_bytes = dt == ADA_F32 ? n_tok * (size_t)maxd * 12 + 1024 : 0;
+    const size_t o_sxa = take(split_bytes), o_sxb = take(split_bytes), o_sra = take(split_bytes),
+                 o_srb = take(split_bytes);
     if (cudaMalloc(&ctx->ws, off) != cudaSuccess) {
         cudaGetLastError();
         delete ctx;
@@ -180,6 +189,10 @@ ada_status ada_create(ada_ctx** out, int device, int64_t maxB, int64_t maxT, int
     ctx->agg = reinterpret_cast<unsigned long long*>(ctx->ws + o_agg);
     ctx->agg_stride = agg_stride;
     ctx->Xrep = ctx->ws + o_xrep;
+    ctx->splitXA = split_bytes ? ctx->ws + o_sxa : nullptr;
+    ctx->splitXB = split_bytes ? ctx->ws + o_sxb : nullptr;
+    ctx->splitRA = split_bytes ? ctx->ws + o_sra : nullptr;
+    ctx->splitRB = split_bytes ? ctx->ws + o_srb : nullptr;
     if (cudaMemset(ctx->ws, 0, o_xrep) != cudaSuccess) {
         cudaFree(ctx->ws);
         delete ctx;
@@ -209,8 +222,7 @@ ada_status ada_set_engine(ada_ctx* ctx, ada_engine e) {
     if (e != ADA_ENGINE_AUTO && e != ADA_ENGINE_FFMA && e != ADA_ENGINE_TCGEN05 &&
         e != ADA_ENGINE_TCGEN05_PAIR)
         return ADA_ERR_INVALID_ARG;
-    if ((e == ADA_ENGINE_TCGEN05 || e == ADA_ENGINE_TCGEN05_PAIR) &&
-        (ctx->dt != ADA_BF16 || !gram_tc_available()))
+    if ((e == ADA_ENGINE_TCGEN05 || e == ADA_ENGINE_TCGEN05_PAIR) && !gram_tc_available())
         return ADA_ERR_UNSUPPORTED;
     ctx->engine = e;
     return ADA_OK;
@@ -253,8 +265,11 @@ ada_status ada_select_full(ada_ctx* ctx, const void* X, int64_t B, int64_t T, in
 
     // the gamma scratch is zero on entry (workspace invariant kept by the compaction kernels)
     // long-K tensor-core launches compute the row norms themselves, hidden behind the MMAs
+    const bool split = use_split(ctx, dt);
     const bool tc = use_tc(ctx, dt), fuse = tc && d >= 2048 && B * T >= 4096;
-    if (!fuse)
+    if (split)   // one pass: 1/||x|| and the bf16 terms of X
+        CU(launch_split(ctx, X, (int)B, (int)T, (int)d, ldx, false, s));
+    else if (!fuse)
         CU(launch_norm_gather(ctx, X, (int)B, (int)T, (int)d, ldx, dt, ctx->inv_norm, nullptr,
                               nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, s));
     NormJob nj;
@@ -270,7 +285,13 @@ ada_status ada_select_full(ada_ctx* ctx, const void* X, int64_t B, int64_t T, in
     p.rows = (int)T; p.cap = (int)T; p.d = (int)d; p.B = (int)B;
     p.tri = 1;
     p.wait_norm_a = p.wait_norm_b = fuse ? 1 : 0;
-    if (tc) CU(launch_tc(ctx, &p, nullptr, fuse ? &nj : nullptr, s));
+    if (split) {
+        p.A = ctx->splitXA; p.Bm = ctx->splitXB;
+        p.lda = p.ldb = 6 * d;
+        p.a_batch = p.b_batch = T * 6 * d;
+        p.d = (int)(6 * d);
+        CU(launch_tc(ctx, &p, nullptr, nullptr, s));
+    } else if (tc) CU(launch_tc(ctx, &p, nullptr, fuse ? &nj : nullptr, s));
     else CU(run_gram(ctx, p, dt, s));
     CU(launch_compact_full(ctx, (int)B, (int)T, thr, rep_idx, rep_cnt, gamma, s));
     return ADA_OK;
@@ -298,12 +319,16 @@ ada_status ada_cascade_step(ada_ctx* ctx, const void* X, int64_t B, int64_t T, i
     // lines 1-2: inverse norms of all rows; inherited list validated, scattered into the role
     // map and its rows gathered into Xrep
     // tensor cores: one launch does lines 3-8; for long K it also computes line 1's row norms
-    const bool fuse = use_tc(ctx, dt), fuse_norm = fuse && d >= 2048 && B * T >= 4096;
-    CU(launch_norm_gather(ctx, X, (int)B, (int)T, (int)d, ldx, dt, fuse_norm ? nullptr : ctx->inv_norm,
+    const bool split = use_split(ctx, dt);
+    const bool fuse = use_tc(ctx, dt) || split, fuse_norm = !split && fuse && d >= 2048 && B * T >= 4096;
+    CU(launch_norm_gather(ctx, X, (int)B, (int)T, (int)d, ldx, dt,
+                          (fuse_norm || split) ? nullptr : ctx->inv_norm,
                           nullptr, rep_in, rep_in_cnt, ctx->role, ctx->r_eff, ctx->Xrep,
                           ctx->inv_rep, s));
     NormJob nj;
     nj.X = X; nj.ldx = ldx; nj.n_rows = B * T; nj.d = (int)d; nj.inv_norm = ctx->inv_norm;
+    if (split)   // 1/||x|| of all rows; bf16 terms of X and of the gathered rows
+        CU(launch_split(ctx, X, (int)B, (int)T, (int)d, ldx, true, s));
     // lines 3-4: r x r Gram among inherited reps, max over earlier ones
     GramProblem p;
     memset(&p, 0, sizeof(p));
@@ -334,6 +359,13 @@ ada_status ada_cascade_step(ada_ctx* ctx, const void* X, int64_t B, int64_t T, i
     q.row_role = ctx->role;
     q.causal = (flags & ADA_CROSS_CAUSAL) ? 1 : 0;
     q.wait_norm_a = fuse_norm ? 1 : 0;
+    if (split) {
+        p.A = ctx->splitRA; p.Bm = ctx->splitRB;
+        q.A = ctx->splitXA; q.Bm = ctx->splitRB;
+        p.lda = p.ldb = q.lda = q.ldb = 6 * d;
+        p.a_batch = p.b_batch = q.a_batch = q.b_batch = T * 6 * d;
+        p.d = q.d = (int)(6 * d);
+    }
     if (fuse) CU(launch_tc(ctx, &p, &q, fuse_norm ? &nj : nullptr, s));
     else CU(run_gram(ctx, q, dt, s));
     // lines 5, 9, 10-11

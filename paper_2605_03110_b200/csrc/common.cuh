@@ -25,6 +25,7 @@ enum KernelId {
     K_GRAM_TC_TRI,
     K_GRAM_TC_CROSS,
     K_GRAM_TC_CASCADE,
+    K_SPLIT,
     K_COMPACT_FULL,
     K_COMPACT_CASCADE,
     K_COUNT
@@ -112,6 +113,9 @@ struct ada_ctx {
     unsigned* done_ctr;  // compaction blocks finished
     int agg_stride;
     void* Xrep;          // [maxB*maxT*maxd] gathered representative rows (raw values)
+    // fp32 contexts: three-term bf16 splits laid out for one contraction of length 6d
+    void *splitXA, *splitXB;   // [maxB*maxT][6 maxd] of X
+    void *splitRA, *splitRB;   // same, of the gathered representative rows
     // staging for the *_host entry points (allocated on first use)
     char* stage;
     size_t stage_bytes;
@@ -130,6 +134,8 @@ cudaError_t launch_norm_gather(ada_ctx* ctx, const void* X, int B, int T, int d,
                                ada_dtype dt, float* inv_norm, void* Xhat, const int32_t* rep_in,
                                const int32_t* rep_in_cnt, int32_t* role, int32_t* r_eff, void* Xrep,
                                float* inv_rep, cudaStream_t s);
+cudaError_t launch_split(ada_ctx* ctx, const void* X, int B, int T, int d, int64_t ldx, bool with_rep,
+                         cudaStream_t s);
 cudaError_t launch_compact_full(ada_ctx* ctx, int B, int T, float thr, int32_t* rep_idx,
                                 int32_t* rep_cnt, float* gamma, cudaStream_t s);
 cudaError_t launch_compact_cascade(ada_ctx* ctx, int B, int T, float thr, int32_t* rep_out,

@@ -178,6 +178,115 @@ cudaError_t launch_norm_gather(ada_ctx* ctx, const void* X, int B, int T, int d,
 }
 
 // ---------------------------------------------------------------------------
+// fp32 on the bf16 tensor cores: every fp32 value is split into three bf16 terms
+//   x = hi + mid + lo,  hi = bf16(x), mid = bf16(x - hi), lo = bf16(x - hi - mid)
+// (both differences are exact in fp32), and a dot product is evaluated as the six largest
+// of the nine cross terms, hi.hi + hi.mid + mid.hi + hi.lo + lo.hi + mid.mid, all of whose
+// bf16 x bf16 products are exact in the fp32 accumulator.  What is dropped is below
+// 2^-23 |x||y|, i.e. fp32 rounding level.  The six terms become ONE bf16 contraction of
+// length 6d by laying the terms side by side:
+//   A' = [hi | hi | mid | hi | lo | mid],   B' = [hi | mid | hi | lo | hi | mid].
+// This kernel writes A' and B' for the rows of X (job 0, which also yields 1/||x||) and for
+// the gathered representative rows (job 1, row count resident on the device).
+// ---------------------------------------------------------------------------
+struct SplitJob {
+    const float* X;          // rows to split
+    int64_t ldx;             // row stride of X in elements
+    int rows_per_seq;        // rows per sequence (capacity)
+    const int32_t* n_dev;    // [B] rows actually present per sequence, or NULL = all
+    __nv_bfloat16* A;        // [B*rows_per_seq][6d]
+    __nv_bfloat16* Bm;       // [B*rows_per_seq][6d]
+    float* inv_norm;         // optional
+};
+
+__device__ __forceinline__ void split3(float x, __nv_bfloat16& hi, __nv_bfloat16& mid, __nv_bfloat16& lo) {
+    hi = __float2bfloat16_rn(x);
+    const float r1 = x - __bfloat162float(hi);
+    mid = __float2bfloat16_rn(r1);
+    const float r2 = r1 - __bfloat162float(mid);
+    lo = __float2bfloat16_rn(r2);
+}
+
+__global__ void __launch_bounds__(256)
+k_split_bf16(const SplitJob j0, const SplitJob j1, int64_t n_rows, int d, unsigned* __restrict__ status) {
+    const int lane = threadIdx.x & 31;
+    int64_t w = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const bool second = w >= n_rows;
+    if (second) w -= n_rows;
+    const SplitJob& j = second ? j1 : j0;
+    if (j.X == nullptr || w >= n_rows) return;
+    if (j.n_dev != nullptr) {
+        const int b = (int)(w / j.rows_per_seq), i = (int)(w % j.rows_per_seq);
+        if (i >= j.n_dev[b]) return;
+    }
+    const float4* src = reinterpret_cast<const float4*>(j.X + w * j.ldx);
+    __nv_bfloat16* a = j.A + w * (int64_t)(6 * d);
+    __nv_bfloat16* bm = j.Bm + w * (int64_t)(6 * d);
+    float ss = 0.f;
+    for (int v = lane; v < (d >> 2); v += 32) {            // d is a multiple of 4
+        const float4 x = __ldg(src + v);
+        const float xs[4] = {x.x, x.y, x.z, x.w};
+        __nv_bfloat16 hi[4], mid[4], lo[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            ss = fmaf(xs[q], xs[q], ss);
+            split3(xs[q], hi[q], mid[q], lo[q]);
+        }
+        const uint2 H = *reinterpret_cast<const uint2*>(hi), M = *reinterpret_cast<const uint2*>(mid),
+                    L = *reinterpret_cast<const uint2*>(lo);
+        const int k = v * 4;
+        // A' = [hi | hi | mid | hi | lo | mid]
+        *reinterpret_cast<uint2*>(a + 0 * d + k) = H;
+        *reinterpret_cast<uint2*>(a + 1 * d + k) = H;
+        *reinterpret_cast<uint2*>(a + 2 * d + k) = M;
+        *reinterpret_cast<uint2*>(a + 3 * d + k) = H;
+        *reinterpret_cast<uint2*>(a + 4 * d + k) = L;
+        *reinterpret_cast<uint2*>(a + 5 * d + k) = M;
+        // B' = [hi | mid | hi | lo | hi | mid]
+        *reinterpret_cast<uint2*>(bm + 0 * d + k) = H;
+        *reinterpret_cast<uint2*>(bm + 1 * d + k) = M;
+        *reinterpret_cast<uint2*>(bm + 2 * d + k) = H;
+        *reinterpret_cast<uint2*>(bm + 3 * d + k) = L;
+        *reinterpret_cast<uint2*>(bm + 4 * d + k) = H;
+        *reinterpret_cast<uint2*>(bm + 5 * d + k) = M;
+    }
+    if (j.inv_norm != nullptr) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        float inv = 0.f;
+        if (!(ss <= 3.0e38f)) {
+            if (lane == 0) atomicOr(status, ST_NONFINITE);
+        } else if (ss > 0.f) {
+            inv = 1.0f / sqrtf(ss);
+        } else if (lane == 0) {
+            atomicAdd(status + 1, 1u);
+        }
+        if (lane == 0) j.inv_norm[w] = inv;
+    }
+}
+
+// X (B*T rows) -> ctx->splitXA/XB (+ inv_norm); with_rep: ctx->Xrep rows below r_eff -> splitRA/RB
+cudaError_t launch_split(ada_ctx* ctx, const void* X, int B, int T, int d, int64_t ldx, bool with_rep,
+                         cudaStream_t s) {
+    const int64_t n_rows = (int64_t)B * T;
+    SplitJob j0, j1;
+    j0.X = static_cast<const float*>(X); j0.ldx = ldx; j0.rows_per_seq = T; j0.n_dev = nullptr;
+    j0.A = static_cast<__nv_bfloat16*>(ctx->splitXA); j0.Bm = static_cast<__nv_bfloat16*>(ctx->splitXB);
+    j0.inv_norm = ctx->inv_norm;
+    j1 = j0;
+    j1.X = with_rep ? static_cast<const float*>(ctx->Xrep) : nullptr; j1.ldx = d; j1.n_dev = ctx->r_eff;
+    j1.A = static_cast<__nv_bfloat16*>(ctx->splitRA); j1.Bm = static_cast<__nv_bfloat16*>(ctx->splitRB);
+    j1.inv_norm = nullptr;
+    const int warps = 8;
+    const int64_t n_warps = with_rep ? 2 * n_rows : n_rows;
+    prof_begin(ctx, K_SPLIT, s);
+    k_split_bf16<<<(unsigned)((n_warps + warps - 1) / warps), warps * 32, 0, s>>>(j0, j1, n_rows, d,
+                                                                                  ctx->status);
+    prof_end(ctx, s);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------
 // Compaction (Definition 1's threshold; Algorithm 1 lines 5, 9, 10-11 and the lists of
 // Eq. 6).  Every 1024-thread block owns 1024 consecutive tokens of one sequence, one token
 // per thread, so all loads are coalesced and the whole sequence is in flight at once.

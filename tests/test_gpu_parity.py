@@ -30,8 +30,9 @@ def clustered(T, d, seed, dtype):
     return wl.f32_to_bf16_bits(X) if dtype == "bf16" else X
 
 
-# (storage, engine): AUTO, AUTO, forced FFMA, forced one-CTA tcgen05, forced pair-CTA tcgen05
-ENGINES = [("f32", 0), ("bf16", 0), ("bf16", 1), ("bf16", 2), ("bf16", 3)]
+# (storage, engine): 0 AUTO, 1 forced FFMA, 2 forced one-CTA tcgen05, 3 forced pair-CTA tcgen05
+# (fp32 storage reaches the tensor cores through the three-term bf16 split)
+ENGINES = [("f32", 0), ("f32", 1), ("f32", 3), ("bf16", 0), ("bf16", 1), ("bf16", 2), ("bf16", 3)]
 
 
 @pytest.mark.parametrize("dtype,engine", ENGINES)
@@ -95,8 +96,9 @@ def run_config_chain(ada, cfg, n_layers=None, causal=False, engine=0):
     return band_total
 
 
-def test_config1_gpt2_shaped_fp32(ada):
-    assert run_config_chain(ada, wl.CONFIGS[1]) == 0
+@pytest.mark.parametrize("engine", [0, 1])
+def test_config1_gpt2_shaped_fp32(ada, engine):
+    assert run_config_chain(ada, wl.CONFIGS[1], engine=engine) == 0
 
 
 @pytest.mark.parametrize("causal", [False, True])
