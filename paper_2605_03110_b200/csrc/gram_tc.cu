@@ -60,8 +60,17 @@ __device__ __forceinline__ int tri_tiles(int n, int tw) {
 // Stage geometry of the TMA ring for a tile of `ncols` columns: narrower tiles take fewer
 // bytes per K block, so more K blocks fit in flight and the loop stays ahead of the
 // load latency.
-__device__ __forceinline__ int stage_bytes(int ncols) {
+// bytes of one 64-element K block of a tile of `ncols` columns
+__device__ __forceinline__ int sub_bytes(int ncols) {
     return A_BYTES + ((ncols + BOX_N - 1) / BOX_N) * BOX_BYTES;
+}
+// K blocks per ring stage: two where three such stages still fit the ring (tiles up to 128
+// columns), so that the per-stage costs -- barrier round trips, fences, commit -- are paid
+// once per 128 K elements; one for wider tiles
+// (short contractions keep one: with a dozen K blocks the coarser pipeline costs more than
+// it saves)
+__device__ __forceinline__ int stage_ksub(int ncols, int d) {
+    return (d >= 2048 && 3 * 2 * sub_bytes(ncols) <= RING_BYTES) ? 2 : 1;
 }
 __device__ __forceinline__ int stage_count(int sbytes) {
     return min(MAX_STAGES, RING_BYTES / sbytes);
@@ -224,9 +233,11 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
                 const int sg = id < tiles0 ? 0 : 1;
                 const GramProblem& p = sg ? seg1 : seg0;
                 if (!decode_tile(p, sg ? par1 : par0, id - (sg ? tiles0 : 0), pc)) break;
-                const int num_kb = (p.d + BK - 1) / BK;
+                const int ksub = stage_ksub(pc.ncols, p.d);
+                const int num_kb = (p.d + BK * ksub - 1) / (BK * ksub);
                 const int nbox = (pc.ncols + BOX_N - 1) / BOX_N;
-                const int sb = stage_bytes(pc.ncols);
+                const int subb = sub_bytes(pc.ncols);
+                const int sb = ksub * subb;
                 if (sb != cur_sb) {
                     // new stage geometry: every stage of the old one must have been released
                     for (int q = 0; q < cur_nst && ok; ++q)
@@ -239,10 +250,14 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
                     if (!mbar_wait(&sh.empty[s], ((fills >> s) & 1u) ^ 1u, abort_flag, 1)) { ok = false; break; }
                     unsigned char* sa = smem + s * sb;
                     mbar_expect_tx(&sh.full[s], (unsigned)sb);
-                    tma_load_3d(&maps.a[sg], &sh.full[s], sa, kb * BK, pc.row0, pc.b);
-                    for (int j = 0; j < nbox; ++j)
-                        tma_load_3d(&maps.b[sg], &sh.full[s], sa + A_BYTES + j * BOX_BYTES, kb * BK,
-                                    pc.col0 + j * BOX_N, pc.b);
+                    for (int u = 0; u < ksub; ++u) {          // K blocks past d are zero-filled
+                        unsigned char* su = sa + u * subb;
+                        const int k0 = (kb * ksub + u) * BK;
+                        tma_load_3d(&maps.a[sg], &sh.full[s], su, k0, pc.row0, pc.b);
+                        for (int j = 0; j < nbox; ++j)
+                            tma_load_3d(&maps.b[sg], &sh.full[s], su + A_BYTES + j * BOX_BYTES, k0,
+                                        pc.col0 + j * BOX_N, pc.b);
+                    }
                     fills ^= 1u << s; used |= 1u << s; ever |= 1u << s;
                     s = (s + 1 == cur_nst) ? 0 : s + 1;
                 }
@@ -267,8 +282,10 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
                 const int sg = id < tiles0 ? 0 : 1;
                 const GramProblem& p = sg ? seg1 : seg0;
                 if (!decode_tile(p, sg ? par1 : par0, id - (sg ? tiles0 : 0), pc)) break;
-                const int num_kb = (p.d + BK - 1) / BK;
-                const int sb = stage_bytes(pc.ncols);
+                const int ksub = stage_ksub(pc.ncols, p.d);
+                const int num_kb = (p.d + BK * ksub - 1) / (BK * ksub);
+                const int subb = sub_bytes(pc.ncols);
+                const int sb = ksub * subb;
                 if (sb != cur_sb) { cur_sb = sb; cur_nst = stage_count(sb); s = 0; }
                 const unsigned acc = tile_it & 1u, acc_ph = (tile_it >> 1) & 1u;
                 if (!mbar_wait(&sh.tmem_empty[acc], acc_ph ^ 1u, abort_flag, 2)) { ok = false; break; }
@@ -278,13 +295,15 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(&sh.full[s], (uses >> s) & 1u, abort_flag, 3)) { ok = false; break; }
                     tcgen05_fence_after();
-                    const unsigned a_addr = smem_u32(smem + s * sb);
-                    const unsigned long long adesc = smem_desc_sw128(a_addr);
-                    const unsigned long long bdesc = smem_desc_sw128(a_addr + A_BYTES);
+                    for (int u = 0; u < ksub; ++u) {
+                        const unsigned a_addr = smem_u32(smem + s * sb + u * subb);
+                        const unsigned long long adesc = smem_desc_sw128(a_addr);
+                        const unsigned long long bdesc = smem_desc_sw128(a_addr + A_BYTES);
 #pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; ++k) {
-                        // advancing K by 16 bf16 = 32 bytes = 2 descriptor address units
-                        umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+                        for (int k = 0; k < BK / UMMA_K; ++k) {
+                            // advancing K by 16 bf16 = 32 bytes = 2 descriptor address units
+                            umma_bf16(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | u | k) != 0);
+                        }
                     }
                     umma_commit(&sh.empty[s]);          // stage reusable once these MMAs retire
                     uses ^= 1u << s;

@@ -26,6 +26,11 @@ using namespace tc;
 namespace {
 
 constexpr int PM = 2 * BM;     // rows of a pair tile
+// A ring stage holds KSUB consecutive 64-element K blocks (each its own 128-byte-swizzled
+// sub-tile), so that the per-stage costs -- barrier round trips, fences, commit -- are paid
+// once per 128 K elements and the MMA issue stays ahead of the tensor pipe.
+constexpr int KSUB = 2;
+constexpr int BKS = BK * KSUB; // K elements per stage
 
 // ---------------------------------------------------------------- PTX, pair forms
 __device__ __forceinline__ unsigned cluster_rank() {
@@ -146,9 +151,11 @@ __device__ __forceinline__ bool decode_tile(const GramProblem& p, int id, Piece&
     return false;
 }
 // per-CTA stage: 128 rows of A and ncols/2 rows of B (in 64-row boxes)
-__device__ __forceinline__ int stage_bytes_pair(int ncols) {
+// bytes of one 64-element K block of a stage, and of the whole stage
+__device__ __forceinline__ int sub_bytes_pair(int ncols) {
     return A_BYTES + (((ncols >> 1) + BOX_N - 1) / BOX_N) * BOX_BYTES;
 }
+__device__ __forceinline__ int stage_bytes_pair(int ncols) { return KSUB * sub_bytes_pair(ncols); }
 __device__ __forceinline__ int stage_count(int sbytes) {
     return min(MAX_STAGES, RING_BYTES / sbytes);
 }
@@ -215,7 +222,7 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
                 const int sg = id < tiles0 ? 0 : 1;
                 const GramProblem& p = sg ? seg1 : seg0;
                 if (!decode_tile(p, id - (sg ? tiles0 : 0), pc)) break;
-                const int num_kb = (p.d + BK - 1) / BK;
+                const int num_kb = (p.d + BKS - 1) / BKS;
                 const int half = pc.ncols >> 1;
                 const int nbox = (half + BOX_N - 1) / BOX_N;
                 const int sb = stage_bytes_pair(pc.ncols);
@@ -233,10 +240,16 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
                     unsigned char* sa = smem + s * sb;
                     // the leader's barrier counts the bytes of both CTAs
                     if (rank == 0) mbar_expect_tx(&sh.full[s], 2u * (unsigned)sb);
-                    tma_load_3d_pair(&maps.a[sg], &sh.full[s], sa, kb * BK, a_row, pc.b);
-                    for (int j = 0; j < nbox; ++j)
-                        tma_load_3d_pair(&maps.b[sg], &sh.full[s], sa + A_BYTES + j * BOX_BYTES, kb * BK,
-                                         b_row + j * BOX_N, pc.b);
+                    // K blocks past d are zero-filled by the TMA unit
+#pragma unroll
+                    for (int u = 0; u < KSUB; ++u) {
+                        unsigned char* su = sa + u * (sb / KSUB);
+                        const int k0 = kb * BKS + u * BK;
+                        tma_load_3d_pair(&maps.a[sg], &sh.full[s], su, k0, a_row, pc.b);
+                        for (int j = 0; j < nbox; ++j)
+                            tma_load_3d_pair(&maps.b[sg], &sh.full[s], su + A_BYTES + j * BOX_BYTES, k0,
+                                             b_row + j * BOX_N, pc.b);
+                    }
                     fills ^= 1u << s; used |= 1u << s; ever |= 1u << s;
                     s = (s + 1 == cur_nst) ? 0 : s + 1;
                 }
@@ -261,7 +274,7 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
                 const int sg = id < tiles0 ? 0 : 1;
                 const GramProblem& p = sg ? seg1 : seg0;
                 if (!decode_tile(p, id - (sg ? tiles0 : 0), pc)) break;
-                const int num_kb = (p.d + BK - 1) / BK;
+                const int num_kb = (p.d + BKS - 1) / BKS;
                 const int sb = stage_bytes_pair(pc.ncols);
                 if (sb != cur_sb) { cur_sb = sb; cur_nst = stage_count(sb); s = 0; }
                 const unsigned acc = tile_it & 1u, acc_ph = (tile_it >> 1) & 1u;
@@ -272,12 +285,15 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(&sh.full[s], (uses >> s) & 1u, abort_flag, 3)) { ok = false; break; }
                     tcgen05_fence_after();
-                    const unsigned a_addr = smem_u32(smem + s * sb);
-                    const unsigned long long adesc = smem_desc_sw128(a_addr);
-                    const unsigned long long bdesc = smem_desc_sw128(a_addr + A_BYTES);
 #pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; ++k)
-                        umma_bf16_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+                    for (int u = 0; u < KSUB; ++u) {
+                        const unsigned a_addr = smem_u32(smem + s * sb + u * (sb / KSUB));
+                        const unsigned long long adesc = smem_desc_sw128(a_addr);
+                        const unsigned long long bdesc = smem_desc_sw128(a_addr + A_BYTES);
+#pragma unroll
+                        for (int k = 0; k < BK / UMMA_K; ++k)
+                            umma_bf16_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | u | k) != 0);
+                    }
                     umma_commit_pair_both(&sh.empty[s]);   // both producers may refill this stage
                     uses ^= 1u << s;
                     s = (s + 1 == cur_nst) ? 0 : s + 1;
