@@ -223,10 +223,20 @@ static __device__ __forceinline__ void norm_rows(const NormJob& job, int w, int 
     const __nv_bfloat16* X = reinterpret_cast<const __nv_bfloat16*>(job.X);
     for (int64_t row = w; row < job.n_rows; row += nw) {
         const uint4* src = reinterpret_cast<const uint4*>(X + row * job.ldx);
-        // eight independent 128-bit loads in flight per lane: these few warps have to cover
-        // the memory latency that a dedicated kernel would hide with occupancy
+        // sixteen (then eight) independent 128-bit loads in flight per lane: these few warps
+        // have to cover the memory latency that a dedicated kernel would hide with occupancy
         float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
         int v = lane;
+        for (; v + 480 < nvec; v += 512) {
+            uint4 x[16];
+#pragma unroll
+            for (int q = 0; q < 16; ++q) x[q] = __ldg(src + v + 32 * q);
+#pragma unroll
+            for (int q = 0; q < 16; q += 4) {
+                s0 += sumsq_bf16x8(x[q]); s1 += sumsq_bf16x8(x[q + 1]);
+                s2 += sumsq_bf16x8(x[q + 2]); s3 += sumsq_bf16x8(x[q + 3]);
+            }
+        }
         for (; v + 224 < nvec; v += 256) {
             uint4 x[8];
 #pragma unroll
