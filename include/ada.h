@@ -143,6 +143,23 @@ ada_status ada_cascade_step(ada_ctx* ctx, const void* X, int64_t B, int64_t T, i
                             int32_t* rem_cnt, float* gamma_rep, float* gamma_cross,
                             uint32_t flags, void* stream);
 
+/*
+ * Nearest-representative map (Section 2.3: the attention output of a redundant token is
+ * taken from the representative s* in R maximising |G_ts*|).  For every token t of X and a
+ * representative set R given as an ascending list (e.g. the output of ada_select_full or
+ * ada_cascade_step on the same X):
+ *   nearest_idx[t] = argmax_{s in R} |G_ts|, the lowest index on ties; a representative maps
+ *                    to itself; -1 when R is empty
+ *   nearest_gamma[t] (optional) = that maximum |G_ts*| (1 for a representative, 0 for zero rows)
+ * One T x r cross-Gram on the tensor cores with an argmax epilogue (both storage types;
+ * fp32 through the three-term split), whatever engine the context is set to; the Gram is
+ * not stored.  Sizes B*T for both outputs.
+ */
+ada_status ada_nearest_rep(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d,
+                           int64_t ldx, ada_dtype dt, const int32_t* rep_idx,
+                           const int32_t* rep_cnt, int32_t* nearest_idx, float* nearest_gamma,
+                           void* stream);
+
 /* Same operations with HOST buffers: inputs are copied to the device (staging
  * buffers owned by the context, allocated on first use), the device-pointer
  * call above runs, results are copied back, all on `stream`, and the call

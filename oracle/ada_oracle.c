@@ -213,6 +213,38 @@ int ada_oracle_cascade(const double* X, int64_t T, int64_t d, double tau,
     return 0;
 }
 
+/* Section 2.3: the attention output of a redundant token is taken from its nearest
+ * representative, s* = argmax_{s in R} |G_ts|.  For every token t: nearest[t] = s*
+ * (lowest index on exact ties), gamma_near[t] = |G_{t s*}|; a representative is its own
+ * nearest representative (gamma_near = |G_tt|: 1, or 0 for a zero row); an empty R gives -1. */
+int ada_oracle_nearest(const double* X, int64_t T, int64_t d, const int32_t* rep, int64_t r,
+                       int32_t* nearest, double* gamma_near) {
+    double* Xhat = (double*)malloc(sizeof(double) * (size_t)T * (size_t)d);
+    uint8_t* is_rep = (uint8_t*)calloc((size_t)T, 1);
+    if (!Xhat || !is_rep) return -1;
+    ada_oracle_normalize(X, T, d, Xhat, NULL);
+    for (int64_t i = 0; i < r; ++i) is_rep[rep[i]] = 1;
+#pragma omp parallel for schedule(dynamic, 4)
+    for (int64_t t = 0; t < T; ++t) {
+        const double* xt = Xhat + t * d;
+        if (is_rep[t]) {
+            nearest[t] = (int32_t)t;
+            gamma_near[t] = fabs(dot(xt, xt, d));
+            continue;
+        }
+        int32_t best = -1;
+        double g = -1.0;
+        for (int64_t i = 0; i < r; ++i) {           /* ascending s: strict > keeps the lowest index */
+            double c = fabs(dot(Xhat + (int64_t)rep[i] * d, xt, d));
+            if (c > g) { g = c; best = rep[i]; }
+        }
+        nearest[t] = best;
+        gamma_near[t] = best >= 0 ? g : 0.0;
+    }
+    free(Xhat); free(is_rep);
+    return 0;
+}
+
 /* Eq. (4)/(5): Gram operation counts.  full: T^2 d.  cascade: r^2 d + (T-r) r d
  * with r the inherited count. */
 uint64_t ada_oracle_op_count(int cascade, int64_t T, int64_t d, int64_t r) {

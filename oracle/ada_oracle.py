@@ -44,6 +44,8 @@ def _load():
         lib.ada_oracle_cascade.argtypes = [dp, i64, i64, C.c_double, ip, i64, C.c_int, bp,
                                            ip, i64, dp, dp, ip, ip, ip, C.POINTER(i64)]
         lib.ada_oracle_cascade.restype = C.c_int
+        lib.ada_oracle_nearest.argtypes = [dp, i64, i64, ip, i64, ip, dp]
+        lib.ada_oracle_nearest.restype = C.c_int
         lib.ada_oracle_op_count.argtypes = [C.c_int, i64, i64, i64]
         lib.ada_oracle_op_count.restype = C.c_uint64
         lib.ada_oracle_jaccard.argtypes = [ip, i64, ip, i64]
@@ -149,6 +151,18 @@ def cascade_step(X, tau: float, rep_in, causal: bool = False,
     if rc != 0:
         raise MemoryError
     return CascadeResult(rep[:n[0]].copy(), add[:n[1]].copy(), rem[:n[2]].copy(), gr[:r].copy(), gc)
+
+
+def nearest(X, rep):
+    """Section 2.3: nearest representative of every token.  Returns (nearest int32[T], gamma[T])."""
+    X = _x(X)
+    T, d = X.shape
+    rep = np.ascontiguousarray(rep, dtype=np.int32)
+    out = np.empty(T, dtype=np.int32)
+    g = np.empty(T, dtype=np.float64)
+    if _load().ada_oracle_nearest(_dp(X), T, d, _ip(rep), rep.size, _ip(out), _dp(g)) != 0:
+        raise MemoryError
+    return out, g
 
 
 def op_count(cascade: bool, T: int, d: int, r: int = 0) -> int:

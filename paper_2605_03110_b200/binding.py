@@ -25,7 +25,7 @@ SYMBOLS = [
     "ada_create", "ada_destroy", "ada_set_engine", "ada_normalize", "ada_select_full",
     "ada_cascade_step", "ada_select_full_host", "ada_cascade_step_host", "ada_gram_op_count",
     "ada_device_status", "ada_profile_enable", "ada_profile_read", "ada_status_string",
-    "ada_select_full_noalloc", "ada_set_cooperative", "ada_selftest_wait_timeout",
+    "ada_select_full_noalloc", "ada_set_cooperative", "ada_selftest_wait_timeout", "ada_nearest_rep",
 ]
 ADA_NOALLOC_MAX_T = 16384
 
@@ -58,6 +58,7 @@ def lib() -> C.CDLL:
         L.ada_cascade_step.argtypes = [vp, vp, i64, i64, i64, i64, C.c_int, C.c_double,
                                        i32p, i32p, i32p, i32p, i32p, i32p, i32p, i32p, fp, fp,
                                        C.c_uint32, vp]
+        L.ada_nearest_rep.argtypes = [vp, vp, i64, i64, i64, i64, C.c_int, i32p, i32p, i32p, fp, vp]
         L.ada_select_full_host.argtypes = [vp, vp, i64, i64, i64, C.c_int, C.c_double, i32p, i32p, fp, vp]
         L.ada_cascade_step_host.argtypes = [vp, vp, i64, i64, i64, C.c_int, C.c_double,
                                             i32p, i32p, i32p, i32p, i32p, i32p, i32p, i32p, fp, fp,
@@ -230,6 +231,18 @@ def ada_cascade_step(ctx: Context, X: torch.Tensor, tau: float, rep_in: torch.Te
                                   _ptr(out.gamma_cross), flags, _stream(stream)),
            "ada_cascade_step")
     return out
+
+
+def ada_nearest_rep(ctx: Context, X: torch.Tensor, rep_idx: torch.Tensor, rep_cnt: torch.Tensor,
+                    want_gamma=True, stream=None):
+    """Section 2.3.  Returns (nearest_idx[B,T] int32, nearest_gamma[B,T] or None)."""
+    X, B, T, d, ldx = _shape(X)
+    near = torch.empty((B, T), dtype=torch.int32, device=X.device)
+    g = torch.empty((B, T), dtype=torch.float32, device=X.device) if want_gamma else None
+    _check(lib().ada_nearest_rep(ctx.h, X.data_ptr(), B, T, d, ldx, dtype_of(X), rep_idx.data_ptr(),
+                                 rep_cnt.data_ptr(), near.data_ptr(), _ptr(g), _stream(stream)),
+           "ada_nearest_rep")
+    return near, g
 
 
 def ada_select_full_host(ctx: Context, X: torch.Tensor, tau: float, rep_idx: torch.Tensor,

@@ -14,7 +14,7 @@ namespace {
 const char* const kKernelNames[K_COUNT] = {
     "norm_gather",     "gram_ffma_tri",    "gram_ffma_cross",
     "gram_tc_tri",     "gram_tc_cross",    "gram_tc_cascade", "split_bf16x3",  "compact_full",
-    "compact_cascade",
+    "compact_cascade", "nearest_finish",
 };
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -166,6 +166,7 @@ ada_status ada_create(ada_ctx** out, int device, int64_t maxB, int64_t maxT, int
     const size_t o_ctr = take(32);
     const int agg_stride = (int)((maxT + 1023) / 1024);
     const size_t o_done = take(32), o_agg = take((size_t)maxB * agg_stride * 8);
+    const size_t o_near = take(n_tok * 8);
     const size_t o_inv = take(n_tok * 4), o_invr = take(n_tok * 4);
     const size_t o_reff = take((size_t)maxB * 4), o_stat = take(32);
     const size_t o_xrep = take(n_tok * (size_t)maxd * ctx->es + 1024);
@@ -188,6 +189,7 @@ ada_status ada_create(ada_ctx** out, int device, int64_t maxB, int64_t maxT, int
     ctx->done_ctr = reinterpret_cast<unsigned*>(ctx->ws + o_done);
     ctx->agg = reinterpret_cast<unsigned long long*>(ctx->ws + o_agg);
     ctx->agg_stride = agg_stride;
+    ctx->near_key = reinterpret_cast<unsigned long long*>(ctx->ws + o_near);
     ctx->Xrep = ctx->ws + o_xrep;
     ctx->splitXA = split_bytes ? ctx->ws + o_sxa : nullptr;
     ctx->splitXB = split_bytes ? ctx->ws + o_sxb : nullptr;
@@ -371,6 +373,47 @@ ada_status ada_cascade_step(ada_ctx* ctx, const void* X, int64_t B, int64_t T, i
     // lines 5, 9, 10-11
     CU(launch_compact_cascade(ctx, (int)B, (int)T, thr, rep_out, rep_out_cnt, add_idx, add_cnt,
                               rem_idx, rem_cnt, gamma_rep, gamma_cross, s));
+    return ADA_OK;
+}
+
+ada_status ada_nearest_rep(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d,
+                           int64_t ldx, ada_dtype dt, const int32_t* rep_idx,
+                           const int32_t* rep_cnt, int32_t* nearest_idx, float* nearest_gamma,
+                           void* stream) {
+    ada_status st = check_common(ctx, X, B, T, d, ldx, dt);
+    if (st != ADA_OK) return st;
+    if (rep_idx == nullptr || rep_cnt == nullptr || nearest_idx == nullptr) return ADA_ERR_INVALID_ARG;
+    const bool split = dt == ADA_F32;
+    if (!gram_tc_available() || (split && ctx->splitXA == nullptr)) return ADA_ERR_UNSUPPORTED;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // role map and keys are zero on entry (workspace invariant); the finish kernel clears them
+    CU(launch_norm_gather(ctx, X, (int)B, (int)T, (int)d, ldx, dt, split ? nullptr : ctx->inv_norm,
+                          nullptr, rep_idx, rep_cnt, ctx->role, ctx->r_eff, ctx->Xrep, ctx->inv_rep, s));
+    if (split) CU(launch_split(ctx, X, (int)B, (int)T, (int)d, ldx, true, s));
+    GramProblem q;
+    memset(&q, 0, sizeof(q));
+    q.A = X; q.Bm = ctx->Xrep;
+    q.lda = ldx; q.ldb = d;
+    q.a_batch = T * ldx; q.b_batch = T * d;
+    if (split) {
+        q.A = ctx->splitXA; q.Bm = ctx->splitRB;
+        q.lda = q.ldb = 6 * d;
+        q.a_batch = q.b_batch = T * 6 * d;
+    }
+    q.inv_a = ctx->inv_norm; q.inv_b = ctx->inv_rep;
+    q.out = ctx->g_tok;
+    q.out_arg = ctx->near_key;
+    q.n_dev = ctx->r_eff; q.n_host = 0;
+    q.rows = (int)T; q.cap = (int)T; q.d = (int)(split ? 6 * d : d); q.B = (int)B;
+    q.tri = 0;
+    q.col_gate = ctx->g_rep;          // all zero: every column passes the gate
+    q.thr_bits = 0xFFFFFFFFu;
+    q.col_token = rep_idx;
+    q.row_role = ctx->role;           // representatives are resolved by the finish kernel
+    q.causal = 0;
+    CU(launch_gram_tc(ctx, nullptr, &q, nullptr, s));
+    CU(launch_nearest_finish(ctx, (int)B, (int)T, rep_idx, nearest_idx, nearest_gamma, s));
     return ADA_OK;
 }
 

@@ -28,6 +28,7 @@ enum KernelId {
     K_SPLIT,
     K_COMPACT_FULL,
     K_COMPACT_CASCADE,
+    K_NEAREST_FINISH,
     K_COUNT
 };
 
@@ -65,6 +66,9 @@ struct GramProblem {
     // set when inv_a / inv_b are produced inside the same launch (NormJob): the epilogue
     // waits for the norm warps before it reads them
     int wait_norm_a, wait_norm_b;
+    // nearest-representative mode (cross only): instead of `out`, combine per row the packed
+    // key (value bits << 32 | ~column) with a 64-bit atomicMax: largest value, lowest column
+    unsigned long long* out_arg;
 };
 
 // Row norms computed inside a tensor-core Gram launch by four extra warps per CTA
@@ -112,6 +116,7 @@ struct ada_ctx {
     unsigned long long* agg;  // [maxB][agg_stride] block counts published by the compaction
     unsigned* done_ctr;  // compaction blocks finished
     int agg_stride;
+    unsigned long long* near_key;  // [maxB*maxT] packed (value, ~column) of the nearest representative
     void* Xrep;          // [maxB*maxT*maxd] gathered representative rows (raw values)
     // fp32 contexts: three-term bf16 splits laid out for one contraction of length 6d
     void *splitXA, *splitXB;   // [maxB*maxT][6 maxd] of X
@@ -136,6 +141,8 @@ cudaError_t launch_norm_gather(ada_ctx* ctx, const void* X, int B, int T, int d,
                                float* inv_rep, cudaStream_t s);
 cudaError_t launch_split(ada_ctx* ctx, const void* X, int B, int T, int d, int64_t ldx, bool with_rep,
                          cudaStream_t s);
+cudaError_t launch_nearest_finish(ada_ctx* ctx, int B, int T, const int32_t* rep_idx,
+                                  int32_t* nearest_idx, float* nearest_gamma, cudaStream_t s);
 cudaError_t launch_compact_full(ada_ctx* ctx, int B, int T, float thr, int32_t* rep_idx,
                                 int32_t* rep_cnt, float* gamma, cudaStream_t s);
 cudaError_t launch_compact_cascade(ada_ctx* ctx, int B, int T, float thr, int32_t* rep_out,

@@ -370,10 +370,18 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
             const int row = pc.row0 + quad * 32 + lane;
             const bool need_cmp = p.tri ? (pc.col0 + ncols > pc.row0) : (p.causal != 0);
             float mx = 0.f;
+            int arg = 0;                                  // nearest-representative mode: column of mx
+            const bool want_arg = p.out_arg != nullptr;
             for (int c0 = 0; c0 < ncols32; c0 += 32) {
                 float v[32];
                 tmem_ld32(tmem_base + ((unsigned)(quad * 32) << 16) + acc * BN + c0, v);
-                if (!need_cmp) {
+                if (want_arg) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {        // ascending columns, strict '>': lowest index on ties
+                        const float x = fabsf(v[j]) * cs[c0 + j];
+                        if (x > mx) { mx = x; arg = c0 + j; }
+                    }
+                } else if (!need_cmp) {
 #pragma unroll
                     for (int j = 0; j < 32; j += 4) {
                         const float4 f = *reinterpret_cast<const float4*>(cs + c0 + j);
@@ -402,7 +410,14 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
                 const bool skip = !p.tri && p.row_role[o + row] != 0;   // inherited reps are not candidates
                 if (!skip) {
                     mx *= __ldcg(p.inv_a + o + row);
-                    if (mx > 0.f) atomicMax(p.out + o + row, __float_as_uint(mx));
+                    if (want_arg) {
+                        const unsigned long long key =
+                            ((unsigned long long)__float_as_uint(mx) << 32) |
+                            (unsigned long long)(0xFFFFFFFFu - (unsigned)(pc.col0 + arg));
+                        if (mx > 0.f) atomicMax(p.out_arg + o + row, key);
+                    } else if (mx > 0.f) {
+                        atomicMax(p.out + o + row, __float_as_uint(mx));
+                    }
                 }
             }
             if (sg == 0 && nseg > 1) {

@@ -72,6 +72,7 @@ ada_status setup_device(int device, PerDevice** out) {
         c.role = nullptr;
         c.r_eff = nullptr;
         c.Xrep = nullptr;
+        c.near_key = nullptr;
         c.splitXA = c.splitXB = c.splitRA = c.splitRB = nullptr;
         pd.ready = true;
     }

@@ -435,6 +435,52 @@ __global__ void __launch_bounds__(1024) k_compact(const CompactArgs a) {
     }
 }
 
+// Nearest-representative map (Section 2.3): turns the packed keys of the argmax Gram launch
+// into token indices.  A representative is its own nearest representative; a token whose
+// correlations are all zero gets the first representative (lowest index among equals); an
+// empty set gives -1.  Clears the keys and the role map it reads.
+__global__ void __launch_bounds__(256)
+k_nearest_finish(unsigned long long* __restrict__ near_key, int32_t* __restrict__ role,
+                 const int32_t* __restrict__ r_eff, const float* __restrict__ inv_norm,
+                 const int32_t* __restrict__ rep_idx, int T, int32_t* __restrict__ nearest_idx,
+                 float* __restrict__ nearest_gamma) {
+    const int b = blockIdx.y, t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= T) return;
+    const int64_t o = (int64_t)b * T;
+    const unsigned long long key = near_key[o + t];
+    const int p = role[o + t];
+    near_key[o + t] = 0ull;
+    role[o + t] = 0;
+    int idx;
+    float g;
+    if (p > 0) {
+        idx = t;
+        g = inv_norm[o + t] > 0.f ? 1.f : 0.f;
+    } else if (r_eff[b] <= 0) {
+        idx = -1;
+        g = 0.f;
+    } else if (key == 0ull) {
+        idx = rep_idx[o];
+        g = 0.f;
+    } else {
+        const unsigned pos = 0xFFFFFFFFu - (unsigned)(key & 0xFFFFFFFFull);
+        idx = rep_idx[o + pos];
+        g = __uint_as_float((unsigned)(key >> 32));
+    }
+    nearest_idx[o + t] = idx;
+    if (nearest_gamma != nullptr) nearest_gamma[o + t] = g;
+}
+
+cudaError_t launch_nearest_finish(ada_ctx* ctx, int B, int T, const int32_t* rep_idx,
+                                  int32_t* nearest_idx, float* nearest_gamma, cudaStream_t s) {
+    prof_begin(ctx, K_NEAREST_FINISH, s);
+    k_nearest_finish<<<dim3((T + 255) / 256, B), 256, 0, s>>>(ctx->near_key, ctx->role, ctx->r_eff,
+                                                               ctx->inv_norm, rep_idx, T, nearest_idx,
+                                                               nearest_gamma);
+    prof_end(ctx, s);
+    return cudaGetLastError();
+}
+
 static cudaError_t launch_compact(ada_ctx* ctx, int kid, const CompactArgs& a, int B, cudaStream_t s) {
     const int nblk = (a.T + 1023) / 1024;
     if (nblk > a.agg_stride) return cudaErrorInvalidValue;

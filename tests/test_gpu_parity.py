@@ -270,6 +270,74 @@ def test_error_paths(ada):
     ada.ada_destroy(ctx)
 
 
+def check_nearest(ada, ctx, Xnp, rep_lists, tol):
+    """ada_nearest_rep vs the oracle: same index, except where the oracle's runner-up is within
+    the tolerance of its maximum (then any representative that close is accepted)."""
+    from parity import to_device
+    B, T, _ = Xnp.shape
+    rin = np.zeros((B, T), dtype=np.int32)
+    rcnt = np.zeros(B, dtype=np.int32)
+    for b, r in enumerate(rep_lists):
+        rin[b, :len(r)] = r
+        rcnt[b] = len(r)
+    near, g = ada.ada_nearest_rep(ctx, to_device(Xnp), torch.from_numpy(rin).cuda(),
+                                  torch.from_numpy(rcnt).cuda())
+    assert ada.ada_device_status(ctx)[0] == 0
+    near, g = near.cpu().numpy(), g.cpu().numpy()
+    n_close = 0
+    for b in range(B):
+        X64 = wl.as_f64(Xnp[b])
+        ref, gref = oracle.nearest(X64, rep_lists[b])
+        assert np.max(np.abs(g[b] - gref), initial=0.0) <= tol
+        diff = np.nonzero(near[b] != ref)[0]
+        if diff.size:
+            Xh, _ = oracle.normalize(X64)
+            for t in diff:
+                assert near[b][t] in set(rep_lists[b])
+                assert abs(float(Xh[t] @ Xh[near[b][t]])) >= gref[t] - tol, (b, int(t))
+                n_close += 1
+    return n_close
+
+
+@pytest.mark.parametrize("dtype,T,d", [("bf16", 1, 8), ("bf16", 300, 72), ("bf16", 1500, 512),
+                                       ("f32", 129, 8), ("f32", 700, 256)])
+def test_nearest_representative_small(ada, dtype, T, d):
+    tol = 2e-3 if dtype == "bf16" else 1e-5
+    ctx = ada.ada_create(1, T, d, ada.ADA_BF16 if dtype == "bf16" else ada.ADA_F32)
+    X = clustered(T, d, 77 + T, dtype)
+    full, _ = oracle.select_full(wl.as_f64(X[0]), TAU)
+    for R in (full.tolist(), [], [T - 1], list(range(T)), list(range(0, T, 3))):
+        check_nearest(ada, ctx, X, [R], tol)
+    ada.ada_destroy(ctx)
+
+
+def test_nearest_representative_on_configs(ada):
+    """After full selection and after a cascade step, batched and at d = 4096."""
+    from parity import lists, to_device
+    for cfg, n_layers in ((wl.CONFIGS[2], 2), (wl.CONFIGS[3], 2)):
+        ctx = ada.ada_create(cfg.B, cfg.T, cfg.d, ada.ADA_BF16)
+        idx = cnt = None
+        for lb in wl.generate_layers(cfg, seed=0, n_layers=n_layers):
+            Xd = to_device(lb.X)
+            if lb.layer == 0:
+                idx, cnt, _ = ada.ada_select_full(ctx, Xd, cfg.tau)
+            else:
+                out = ada.ada_cascade_step(ctx, Xd, cfg.tau, idx, cnt)
+                idx, cnt = out.rep_out, out.rep_out_cnt
+            reps = [r.tolist() for r in lists(idx, cnt)]
+            check_nearest(ada, ctx, lb.X, reps, 2e-3)
+            near, _ = ada.ada_nearest_rep(ctx, Xd, idx, cnt)
+            near = near.cpu().numpy()
+            for b in range(cfg.B):          # label-level: the nearest representative shares the label
+                nonrep = np.setdiff1d(np.arange(cfg.T), reps[b])
+                assert np.all(lb.labels[b][near[b][nonrep]] == lb.labels[b][nonrep])
+        # the workspace is clean again: a following selection is unaffected
+        again = ada.ada_select_full(ctx, Xd, cfg.tau)
+        ref = [oracle.select_full(wl.as_f64(lb.X[b]), cfg.tau)[0].tolist() for b in range(cfg.B)]
+        assert [r.tolist() for r in lists(again[0], again[1])] == ref
+        ada.ada_destroy(ctx)
+
+
 def test_bounded_wait_runs_out_and_the_context_survives(ada):
     """The in-kernel waits have a limit: a wait on a flag nothing sets ends with a status the
     host can read (no trap, no hang), and the context keeps working afterwards."""

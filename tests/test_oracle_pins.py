@@ -380,3 +380,36 @@ def test_forced_valid_and_row_sampling():
     part = oracle.cascade_step(X, SMALL.tau, Rp, only_rows=nonrep)
     assert np.allclose(part.gamma_cross[nonrep], ref.gamma_cross[nonrep], atol=0)
     assert part.add.tolist() == [t for t in ref.add.tolist() if t in set(nonrep.tolist())]
+
+
+# ---------------------------------------------------------------- nearest representative (Section 2.3)
+def test_nearest_on_example_a_and_brute_force():
+    X = rows_at_angles(EX_A_DEG, EX_A_NORM)
+    near, g = oracle.nearest(X, [0, 4])                 # reps at 0 and 90 degrees
+    assert near.tolist() == [0, 0, 0, 4, 4, 0]          # 20,40 -> 0; 60 -> 90 (cos 30 > cos 60); 180 -> 0
+    assert np.allclose(g, [1.0, acos(20), acos(40), acos(30), 1.0, 1.0], atol=1e-12)
+    rng = np.random.default_rng(9)
+    Y = rng.standard_normal((60, 7))
+    R = sorted(rng.choice(60, 11, replace=False).tolist())
+    near, g = oracle.nearest(Y, R)
+    Yh = Y / np.linalg.norm(Y, axis=1, keepdims=True)
+    G = np.abs(Yh @ Yh[R].T)
+    for t in range(60):
+        if t in R:
+            assert near[t] == t and abs(g[t] - 1.0) < 1e-12
+        else:
+            assert near[t] == R[int(np.argmax(G[t]))] and abs(g[t] - G[t].max()) < 1e-12
+    assert oracle.nearest(Y, [])[0].tolist() == [-1] * 60
+
+
+def test_nearest_ties_go_to_the_lowest_index_and_labels_agree():
+    X = np.zeros((4, 3))
+    X[0] = [1, 0, 0]; X[1] = [1, 0, 0]; X[2] = [0, 1, 0]; X[3] = [2, 0, 0]
+    near, _ = oracle.nearest(X, [0, 1, 2])
+    assert near[3] == 0                                  # exact tie between reps 0 and 1
+    st = chain(SMALL)[3]
+    near, g = oracle.nearest(st["X"], st["R"])
+    lab = st["labels"]
+    nonrep = np.setdiff1d(np.arange(lab.size), st["R"])
+    # a redundant token's nearest representative carries its prototype label
+    assert np.all(lab[near[nonrep]] == lab[nonrep]) and np.all(g[nonrep] > 0.9)
