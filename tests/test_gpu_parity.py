@@ -338,6 +338,36 @@ def test_nearest_representative_on_configs(ada):
         ada.ada_destroy(ctx)
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_padded_row_stride(ada, dtype):
+    """ldx > d: X is a column slice of a wider buffer (TMA strides, vector loads, split kernel)."""
+    from parity import lists
+    T, d, ldx = 333, 200, 264
+    X = clustered(T, d, 5, dtype)[0]
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    wide = torch.full((1, T, ldx), 7.0, dtype=tdt, device="cuda")          # padding must be ignored
+    if dtype == "bf16":
+        wide[0, :, :d] = torch.from_numpy(X.view(np.int16)).view(torch.bfloat16).cuda()
+    else:
+        wide[0, :, :d] = torch.from_numpy(X).cuda()
+    Xv = wide[:, :, :d]
+    assert Xv.stride(1) == ldx
+    ctx = ada.ada_create(1, T, d, ada.ADA_BF16 if dtype == "bf16" else ada.ADA_F32)
+    idx, cnt, gamma = ada.ada_select_full(ctx, Xv, TAU)
+    ref_rep, ref_g = oracle.select_full(wl.as_f64(X), TAU)
+    tol = 2e-3 if dtype == "bf16" else 1e-5
+    assert np.max(np.abs(gamma.cpu().numpy()[0] - ref_g)) <= tol
+    assert lists(idx, cnt)[0].tolist() == ref_rep.tolist()
+    out = ada.ada_cascade_step(ctx, Xv, TAU, idx, cnt)
+    ref = oracle.cascade_step(wl.as_f64(X), TAU, ref_rep)
+    assert lists(out.rep_out, out.rep_out_cnt)[0].tolist() == ref.rep.tolist()
+    assert np.max(np.abs(out.gamma_cross.cpu().numpy()[0] - ref.gamma_cross)) <= tol
+    near, _ = ada.ada_nearest_rep(ctx, Xv, out.rep_out, out.rep_out_cnt)
+    assert near.cpu().numpy()[0].tolist() == oracle.nearest(wl.as_f64(X), ref.rep)[0].tolist()
+    assert ada.ada_device_status(ctx)[0] == 0
+    ada.ada_destroy(ctx)
+
+
 def test_bounded_wait_runs_out_and_the_context_survives(ada):
     """The in-kernel waits have a limit: a wait on a flag nothing sets ends with a status the
     host can read (no trap, no hang), and the context keeps working afterwards."""
