@@ -248,6 +248,8 @@ def main():
     ap.add_argument("--sweep", action="store_true",
                     help="crossover sweep (configs[4]): full selection vs one cascade step per (T, r/T); "
                          "prints a table instead of the JSON line")
+    ap.add_argument("--causal", action="store_true",
+                    help="cascade steps with ADA_CROSS_CAUSAL (line 8 restricted to s < t)")
     ap.add_argument("--no-cooperative", action="store_true",
                     help="launch the fused cascade kernel as an ordinary grid (for profilers)")
     ap.add_argument("--no-graph", action="store_true",
@@ -303,6 +305,7 @@ def main():
     if args.no_cooperative:
         ada.ada_set_cooperative(ctx, False)
     stream = torch.cuda.current_stream()
+    cflags = ada.ADA_CROSS_CAUSAL if args.causal else 0
 
     i32 = dict(dtype=torch.int32, device=dev)
     idx = [torch.empty((B, T), **i32) for _ in range(2)]
@@ -319,7 +322,7 @@ def main():
         for l in range(1, L):
             nxt = 1 - cur
             ada.ada_cascade_step(ctx, dev_layers[l], cfg.tau, outs[cur].rep_out, outs[cur].rep_out_cnt,
-                                 out=outs[nxt], stream=stream)
+                                 out=outs[nxt], flags=cflags, stream=stream)
             cur = nxt
             if record:
                 r_hist[l, 0].copy_(outs[cur].rep_out_cnt)
@@ -445,7 +448,7 @@ def main():
     casc_sets.append([outs[0].rep_out[b, :int(outs[0].rep_out_cnt[b])].cpu().numpy() for b in range(B)])
     for l in range(1, L):
         ada.ada_cascade_step(ctx, dev_layers[l], cfg.tau, outs[cur].rep_out, outs[cur].rep_out_cnt,
-                             out=outs[1 - cur])
+                             out=outs[1 - cur], flags=cflags)
         cur = 1 - cur
         casc_sets.append([outs[cur].rep_out[b, :int(outs[cur].rep_out_cnt[b])].cpu().numpy()
                           for b in range(B)])
@@ -472,7 +475,7 @@ def main():
             c = 0
             for l in range(1, L):
                 ada.ada_cascade_step_host(ctx, pin[l], cfg.tau, h_idx[c], h_cnt[c], h_idx[1 - c],
-                                          h_cnt[1 - c], h_add, h_addc, h_rem, h_remc)
+                                          h_cnt[1 - c], h_add, h_addc, h_rem, h_remc, flags=cflags)
                 c = 1 - c
 
         for _ in range(2):
@@ -505,7 +508,8 @@ def main():
         for l in range(n_lay):
             if l > 0:
                 t1 = time.perf_counter()
-                R = [oracle.cascade_step(wl.as_f64(host_layers[l][b]), cfg.tau, R[b]).rep
+                R = [oracle.cascade_step(wl.as_f64(host_layers[l][b]), cfg.tau, R[b],
+                                         causal=args.causal).rep
                      for b in range(B)]
                 t_c.append(time.perf_counter() - t1)
             mism += sum(R[b].tolist() != casc_sets[l][b].tolist() for b in range(B))
@@ -539,6 +543,7 @@ def main():
                      "jaccard_cascade_vs_full_last": j_cvf[-1]},
             "parity_sample": parity_sample, "zero_norm_rows": n_zero,
             "engine": "ffma" if args.engine == 1 else "auto", "cuda_graph": not args.no_graph,
+            "cross_check": "causal (s < t)" if args.causal else "as printed in Algorithm 1 (all valid representatives)",
         }
         print(json.dumps(line))
     ada.ada_destroy(ctx)

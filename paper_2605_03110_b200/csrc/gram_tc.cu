@@ -159,6 +159,14 @@ __device__ __forceinline__ bool decode_tile(const GramProblem& p, int par, int i
 }
 
 // ---------------------------------------------------------------- the kernel
+// Under ADA_CROSS_CAUSAL a cross tile whose first (lowest) column token is not below the
+// tile's last row has no admissible (row, column) pair: every role skips it, so neither
+// its loads nor its MMAs are issued.  Column tokens ascend with the column index.
+__device__ __forceinline__ bool dead_tile(const GramProblem& p, const Piece& pc) {
+    if (p.tri || !p.causal || p.col_token == nullptr) return false;
+    return p.col_token[(int64_t)pc.b * p.cap + pc.col0] >= pc.row0 + BM;
+}
+
 struct GramMaps {
     CUtensorMap a[2], b[2];       // per segment: left operand (128-row boxes), right operand (64-row boxes)
 };
@@ -233,6 +241,7 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
                 const int sg = id < tiles0 ? 0 : 1;
                 const GramProblem& p = sg ? seg1 : seg0;
                 if (!decode_tile(p, sg ? par1 : par0, id - (sg ? tiles0 : 0), pc)) break;
+                if (dead_tile(p, pc)) continue;   // causal cross tile with no admissible pair
                 const int ksub = stage_ksub(pc.ncols, p.d);
                 const int num_kb = (p.d + BK * ksub - 1) / (BK * ksub);
                 const int nbox = (pc.ncols + BOX_N - 1) / BOX_N;
@@ -278,16 +287,18 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
             unsigned uses = 0, tile_it = 0;   // bit s of `uses`: parity of the number of uses of stage s
             int cur_sb = 0, cur_nst = 0, s = 0;
             bool ok = true;
-            for (int id = blockIdx.x; ok && id < total; id += gridDim.x, ++tile_it) {
+            for (int id = blockIdx.x; ok && id < total; id += gridDim.x) {
                 const int sg = id < tiles0 ? 0 : 1;
                 const GramProblem& p = sg ? seg1 : seg0;
                 if (!decode_tile(p, sg ? par1 : par0, id - (sg ? tiles0 : 0), pc)) break;
+                if (dead_tile(p, pc)) continue;   // causal cross tile with no admissible pair
                 const int ksub = stage_ksub(pc.ncols, p.d);
                 const int num_kb = (p.d + BK * ksub - 1) / (BK * ksub);
                 const int subb = sub_bytes(pc.ncols);
                 const int sb = ksub * subb;
                 if (sb != cur_sb) { cur_sb = sb; cur_nst = stage_count(sb); s = 0; }
                 const unsigned acc = tile_it & 1u, acc_ph = (tile_it >> 1) & 1u;
+                ++tile_it;
                 if (!mbar_wait(&sh.tmem_empty[acc], acc_ph ^ 1u, abort_flag, 2)) { ok = false; break; }
                 tcgen05_fence_after();
                 const unsigned idesc = instr_desc(pc.ncols);
@@ -328,11 +339,13 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
         bool norm_ok = norms.X == nullptr;           // row norms computed by this launch's norm warps
         const unsigned norm_total = (unsigned)(gridDim.x * NORM_WARPS);      // cross epilogues must see segment 0 finished
         unsigned tile_it = 0;
-        for (int id = blockIdx.x; id < total; id += gridDim.x, ++tile_it) {
+        for (int id = blockIdx.x; id < total; id += gridDim.x) {
             const int sg = id < tiles0 ? 0 : 1;
             const GramProblem& p = sg ? seg1 : seg0;
             if (!decode_tile(p, sg ? par1 : par0, id - (sg ? tiles0 : 0), pc)) break;
+                if (dead_tile(p, pc)) continue;   // causal cross tile with no admissible pair
             const unsigned acc = tile_it & 1u, acc_ph = (tile_it >> 1) & 1u;
+                ++tile_it;
             const int64_t o = (int64_t)pc.b * p.cap;
             const int ncols = pc.ncols;
             const int ncols32 = (ncols + 31) & ~31;   // TMEM is read 32 columns at a time

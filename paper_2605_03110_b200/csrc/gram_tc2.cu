@@ -160,6 +160,14 @@ __device__ __forceinline__ int stage_count(int sbytes) {
     return min(MAX_STAGES, RING_BYTES / sbytes);
 }
 
+// Under ADA_CROSS_CAUSAL a cross tile whose first (lowest) column token is not below the
+// tile's last row has no admissible (row, column) pair: every role skips it, so neither
+// its loads nor its MMAs are issued.  Column tokens ascend with the column index.
+__device__ __forceinline__ bool dead_tile(const GramProblem& p, const Piece& pc) {
+    if (p.tri || !p.causal || p.col_token == nullptr) return false;
+    return p.col_token[(int64_t)pc.b * p.cap + pc.col0] >= pc.row0 + PM;
+}
+
 struct GramMaps {
     CUtensorMap a[2], b[2];
 };
@@ -222,6 +230,7 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
                 const int sg = id < tiles0 ? 0 : 1;
                 const GramProblem& p = sg ? seg1 : seg0;
                 if (!decode_tile(p, id - (sg ? tiles0 : 0), pc)) break;
+                if (dead_tile(p, pc)) continue;   // causal cross tile with no admissible pair
                 const int num_kb = (p.d + BKS - 1) / BKS;
                 const int half = pc.ncols >> 1;
                 const int nbox = (half + BOX_N - 1) / BOX_N;
@@ -270,14 +279,16 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
             unsigned uses = 0, tile_it = 0;
             int cur_sb = 0, cur_nst = 0, s = 0;
             bool ok = true;
-            for (int id = pair; ok && id < total; id += npairs, ++tile_it) {
+            for (int id = pair; ok && id < total; id += npairs) {
                 const int sg = id < tiles0 ? 0 : 1;
                 const GramProblem& p = sg ? seg1 : seg0;
                 if (!decode_tile(p, id - (sg ? tiles0 : 0), pc)) break;
+                if (dead_tile(p, pc)) continue;   // causal cross tile with no admissible pair
                 const int num_kb = (p.d + BKS - 1) / BKS;
                 const int sb = stage_bytes_pair(pc.ncols);
                 if (sb != cur_sb) { cur_sb = sb; cur_nst = stage_count(sb); s = 0; }
                 const unsigned acc = tile_it & 1u, acc_ph = (tile_it >> 1) & 1u;
+                ++tile_it;
                 if (!mbar_wait(&sh.tmem_empty[acc], acc_ph ^ 1u, abort_flag, 2)) { ok = false; break; }
                 tcgen05_fence_after();
                 const unsigned idesc = instr_desc_pair(pc.ncols);
@@ -319,11 +330,13 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
         const unsigned empty_addr[2] = {map_to_cta(smem_u32(&sh.tmem_empty[0]), 0),
                                         map_to_cta(smem_u32(&sh.tmem_empty[1]), 0)};
         unsigned tile_it = 0;
-        for (int id = pair; id < total; id += npairs, ++tile_it) {
+        for (int id = pair; id < total; id += npairs) {
             const int sg = id < tiles0 ? 0 : 1;
             const GramProblem& p = sg ? seg1 : seg0;
             if (!decode_tile(p, id - (sg ? tiles0 : 0), pc)) break;
+                if (dead_tile(p, pc)) continue;   // causal cross tile with no admissible pair
             const unsigned acc = tile_it & 1u, acc_ph = (tile_it >> 1) & 1u;
+                ++tile_it;
             const int64_t o = (int64_t)pc.b * p.cap;
             const int ncols = pc.ncols;
             if (sg == 1 && !dep_ok) {
