@@ -35,9 +35,9 @@ UNIT = "tokens*layers/s"
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant
 # kernel, from the ncu captures summarised under profiles/ (None until captured).
 NCU_TRAFFIC_BYTES = {
-    # fused cascade launch on configs[3]: mean of the captured layers 1 (77.6 MB) and 30 (106.1 MB),
+    # fused cascade launch on configs[3]: mean of the captured layers 1 (76.9 MB) and 30 (108.4 MB),
     # profiles/gram_tc2_cascade_cfg4.md
-    ("gram_tc_cascade", 4): 91.85e6,
+    ("gram_tc_cascade", 4): 92.65e6,
 }
 
 
