@@ -32,6 +32,10 @@
  *     NaN/Inf in X, an expired bounded wait) set bits in the context's device
  *     status word, leave the call's outputs in bounds but meaningless, and are
  *     reported by ada_device_status.
+ *   - The first call that reaches a given kernel on a context performs one-time host-side
+ *     set-up (function attributes, an occupancy query); make one call of each kind before
+ *     capturing calls into a CUDA graph.  After that the device-pointer calls are plain
+ *     stream-ordered launches with no host synchronisation.
  *   - Arithmetic: squared norms and Gram accumulation in fp32.  ADA_BF16
  *     multiplies the stored bf16 values on the tensor cores (products exact in
  *     fp32) and applies 1/(|x_s| |x_t|) in the epilogue; a normalised bf16 copy

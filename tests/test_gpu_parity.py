@@ -338,6 +338,45 @@ def test_nearest_representative_on_configs(ada):
         ada.ada_destroy(ctx)
 
 
+@pytest.mark.parametrize("cfg_id,n_layers,causal", [(1, 12, False), (2, 12, True), (3, 28, False),
+                                                    (3, 28, True), (4, 10, False)])
+def test_full_length_free_running_chains_match_label_prediction(ada, cfg_id, n_layers, causal):
+    """The production pattern at full size and depth: every layer's output set feeds the next
+    call on the device, nothing is read back in between; the sets, additions and removals of
+    every layer must equal the label-level replay of Definition 1 / Algorithm 1 (which uses
+    no Gram at all)."""
+    from parity import lists, to_device
+    cfg = wl.CONFIGS[cfg_id]
+    ctx = ada.ada_create(cfg.B, cfg.T, cfg.d, ada.ADA_F32 if cfg.dtype == "f32" else ada.ADA_BF16)
+    flags = ada.ADA_CROSS_CAUSAL if causal else 0
+    idx = cnt = None
+    expect = [None] * cfg.B
+    outs = []
+    for lb in wl.generate_layers(cfg, seed=0, n_layers=n_layers):
+        Xd = to_device(lb.X)
+        if lb.layer == 0:
+            idx, cnt, _ = ada.ada_select_full(ctx, Xd, cfg.tau, want_gamma=False)
+            for b in range(cfg.B):
+                expect[b] = (full_from_labels(lb.labels[b]), None, None)
+            outs.append((idx.clone(), cnt.clone(), None))
+        else:
+            out = ada.ada_cascade_step(ctx, Xd, cfg.tau, idx, cnt, flags=flags, want_gamma=False)
+            idx, cnt = out.rep_out, out.rep_out_cnt
+            for b in range(cfg.B):
+                expect[b] = cascade_from_labels(lb.labels[b], expect[b][0], causal)
+            outs.append((idx.clone(), cnt.clone(),
+                         (out.add_idx.clone(), out.add_cnt.clone(), out.rem_idx.clone(), out.rem_cnt.clone())))
+        got = lists(*outs[-1][:2])
+        for b in range(cfg.B):
+            assert got[b].tolist() == expect[b][0].tolist(), (lb.layer, b)
+            if lb.layer > 0:
+                a_i, a_c, m_i, m_c = outs[-1][2]
+                assert lists(a_i, a_c)[b].tolist() == expect[b][1].tolist()
+                assert lists(m_i, m_c)[b].tolist() == expect[b][2].tolist()
+    assert ada.ada_device_status(ctx)[0] == 0
+    ada.ada_destroy(ctx)
+
+
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
 def test_padded_row_stride(ada, dtype):
     """ldx > d: X is a column slice of a wider buffer (TMA strides, vector loads, split kernel)."""
