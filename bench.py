@@ -520,6 +520,19 @@ def main():
                                   f"t(full, layer 0) + {L - 1} x mean t(cascade step)",
                         "t_full_s": t_full, "t_cascade_step_s": float(np.mean(t_c)) if t_c else None}
         parity_sample = {"layers_checked": n_lay, "set_mismatches": mism}
+        if cfg.cfg_id == 1:      # the small fp32 configuration: also one host thread
+            nthr = oracle.num_threads()
+            oracle.set_threads(1)
+            t0 = time.perf_counter()
+            R1 = [oracle.select_full(wl.as_f64(host_layers[0][b]), cfg.tau)[0] for b in range(B)]
+            t_f1 = time.perf_counter() - t0
+            t1 = time.perf_counter()
+            if n_lay > 1:
+                [oracle.cascade_step(wl.as_f64(host_layers[1][b]), cfg.tau, R1[b], causal=args.causal)
+                 for b in range(B)]
+            t_c1 = time.perf_counter() - t1 if n_lay > 1 else t_f1
+            oracle.set_threads(nthr)
+            cpu_baseline["one_thread_value"] = B * T * L / (t_f1 + (L - 1) * t_c1)
 
     if rank == 0:
         line = {

@@ -255,6 +255,20 @@ def test_error_paths(ada):
     with pytest.raises(ada.AdaError) as e:                      # d*es not a multiple of 16
         ada.ada_select_full(ctx, torch.randn(1, 64, 30, device="cuda"), TAU)
     assert e.value.status == 2
+    flat = torch.randn(64 * 32 + 8, device="cuda")              # X not 16-byte aligned
+    with pytest.raises(ada.AdaError) as e:
+        ada.ada_select_full(ctx, flat[1:1 + 64 * 32].view(1, 64, 32), TAU)
+    assert e.value.status == 2
+    idx = torch.zeros((1, 64), dtype=torch.int32, device="cuda")
+    cnt = torch.ones(1, dtype=torch.int32, device="cuda")
+    with pytest.raises(ada.AdaError) as e:                      # rep_out must not alias rep_in
+        out = ada.CascadeOut(1, 64, "cuda", False)
+        out.rep_out = idx
+        ada.ada_cascade_step(ctx, X, TAU, idx, cnt, out=out)
+    assert e.value.status == 1
+    with pytest.raises(ada.AdaError) as e:                      # unknown flag bit
+        ada.ada_cascade_step(ctx, X, TAU, idx, cnt, flags=4)
+    assert e.value.status == 1
     # device-detected: unsorted inherited list, count out of range, NaN
     bad = torch.tensor([[3, 2] + [0] * 62], dtype=torch.int32, device="cuda")
     ada.ada_cascade_step(ctx, X, TAU, bad, torch.tensor([2], dtype=torch.int32, device="cuda"))
