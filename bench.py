@@ -232,6 +232,88 @@ def sweep(args):
           f"{peaks['bf16_sustained']} sustained")
 
 
+def heads_bench(args, cfg):
+    """Per-head selection (Section 8.5) on the layers of `cfg` read as (T, h, d/h): the whole
+    L-layer cascade pipeline with one representative set per head, beside the shared-set pipeline
+    on the same tensors.  CUDA-graph replay of one step, CUDA events, inputs resident in HBM.
+    Prints a table instead of the JSON line."""
+    import torch
+    from paper_2605_03110_b200 import binding as ada
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    h = args.heads
+    assert cfg.B == 1 and cfg.dtype == "bf16" and cfg.d % h == 0
+    T, d, L, d_h = cfg.T, cfg.d, cfg.L, cfg.d // h
+    layers = [torch.from_numpy(lb.X[0].view(np.int16)).view(torch.bfloat16).to(dev)
+              for lb in wl.generate_layers(cfg, seed=0)]
+    side = torch.cuda.Stream()
+    peaks = measured_peaks()
+
+    def pipeline(kind):
+        nb = h if kind == "heads" else 1
+        ctx = ada.ada_create(nb, T, d_h if kind == "heads" else d, ada.ADA_BF16)
+        outs = [ada.CascadeOut(nb, T, dev, want_gamma=False) for _ in range(2)]
+        view = (lambda X: X.view(T, h, d_h)) if kind == "heads" else (lambda X: X.view(1, T, d))
+        full = ada.ada_select_full_heads if kind == "heads" else ada.ada_select_full
+        step = ada.ada_cascade_step_heads if kind == "heads" else ada.ada_cascade_step
+
+        def run(st, n_layers=L):
+            full(ctx, view(layers[0]), cfg.tau, outs[0].rep_out, outs[0].rep_out_cnt, want_gamma=False,
+                 stream=st)
+            cur = 0
+            for l in range(1, n_layers):
+                step(ctx, view(layers[l]), cfg.tau, outs[cur].rep_out, outs[cur].rep_out_cnt,
+                     out=outs[1 - cur], stream=st)
+                cur = 1 - cur
+            return outs[cur]
+
+        def graph_time(fn):
+            fn(None)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(g, stream=side):
+                    fn(side)
+            for _ in range(max(3, args.warmup)):
+                g.replay()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(args.steps):
+                g.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / args.steps
+
+        ms_pipe = graph_time(run)
+        ms_full = graph_time(lambda st: run(st, 1))
+        last = run(None)
+        torch.cuda.synchronize()
+        r = last.rep_out_cnt.cpu().numpy()
+        st_, _ = ada.ada_device_status(ctx)
+        assert st_ == 0
+        ada.ada_destroy(ctx)
+        return ms_pipe, ms_full, r
+
+    rows = []
+    for kind in ("shared", "heads"):
+        ms_pipe, ms_full, r = pipeline(kind)
+        ms_step = (ms_pipe - ms_full) / (L - 1)
+        rows.append((kind, ms_pipe, ms_full, ms_step, r))
+    x_bytes = T * d * 2
+    print(f"workload configs[{cfg.cfg_id - 1}] {cfg.name}: T={T} d={d} L={L} bf16, heads h={h} d_h={d_h}; "
+          f"{args.steps} graph replays after {max(3, args.warmup)} warm-up")
+    print("| sets | step (L layers) ms | tokens*layers/s | full selection us | cascade step us | "
+          "cascade step: X once GB/s | r at the last layer |")
+    print("|---|---|---|---|---|---|---|")
+    for kind, ms_pipe, ms_full, ms_step, r in rows:
+        rr = f"{int(r[0])}" if kind == "shared" else f"{int(r.min())}..{int(r.max())} (mean {r.mean():.0f})"
+        print(f"| {'one per head' if kind == 'heads' else 'one shared'} | {ms_pipe:.3f} | "
+              f"{T * L / (ms_pipe * 1e-3):.3e} | {ms_full * 1e3:.1f} | {ms_step * 1e3:.1f} | "
+              f"{x_bytes / (ms_step * 1e-3) / 1e9:.0f} | {rr} |")
+    print(f"peaks ({peaks['src']}): HBM {peaks['hbm_gbs']} GB/s")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -254,8 +336,15 @@ def main():
                     help="launch the fused cascade kernel as an ordinary grid (for profilers)")
     ap.add_argument("--no-graph", action="store_true",
                     help="launch every call from Python instead of replaying a CUDA graph of one step")
+    ap.add_argument("--heads", type=int, default=0,
+                    help="per-head selection (one set per head, d_h = d / HEADS) beside the shared-set "
+                         "pipeline on --workload 3 or 4; prints a table instead of the JSON line")
     args = ap.parse_args()
 
+    if args.heads:
+        cfg = wl.CONFIGS[args.workload]
+        heads_bench(args, wl.scaled(cfg, L=args.layers) if args.layers else cfg)
+        return
     if args.sweep:
         sweep(args)
         return

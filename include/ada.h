@@ -148,6 +148,28 @@ ada_status ada_cascade_step(ada_ctx* ctx, const void* X, int64_t B, int64_t T, i
                             uint32_t flags, void* stream);
 
 /*
+ * Per-head selection (Section 8.5: one representative set per attention head, h separate
+ * validations per layer at h * T * r_h * d_h operations).  X is ONE sequence of T tokens whose
+ * row holds the h heads side by side: head j of token t is the d_h elements starting at
+ * X[t * ldx + j * d_h] (ldx >= h * d_h; d_h * element size a multiple of 16 bytes), the layout
+ * a projection writes.  The h heads are h independent problems of width d_h, each computed
+ * exactly as ada_select_full / ada_cascade_step compute a sequence, in one launch sequence and
+ * without a transposed copy of X.  Every per-sequence array of those calls is per head here:
+ * lists and gamma arrays have h * T entries (head j at offset j * T), counts have h.  The
+ * context must have been created with maxB >= h, maxT >= T, maxd >= d_h.  Errors, ownership
+ * and stream semantics are those of the calls they mirror.
+ */
+ada_status ada_select_full_heads(ada_ctx* ctx, const void* X, int64_t T, int64_t h, int64_t d_h,
+                                 int64_t ldx, ada_dtype dt, double tau, int32_t* rep_idx,
+                                 int32_t* rep_cnt, float* gamma, void* stream);
+ada_status ada_cascade_step_heads(ada_ctx* ctx, const void* X, int64_t T, int64_t h, int64_t d_h,
+                                  int64_t ldx, ada_dtype dt, double tau, const int32_t* rep_in,
+                                  const int32_t* rep_in_cnt, int32_t* rep_out,
+                                  int32_t* rep_out_cnt, int32_t* add_idx, int32_t* add_cnt,
+                                  int32_t* rem_idx, int32_t* rem_cnt, float* gamma_rep,
+                                  float* gamma_cross, uint32_t flags, void* stream);
+
+/*
  * Nearest-representative map (Section 2.3: the attention output of a redundant token is
  * taken from the representative s* in R maximising |G_ts*|).  For every token t of X and a
  * representative set R given as an ascending list (e.g. the output of ada_select_full or

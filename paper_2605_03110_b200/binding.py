@@ -26,6 +26,7 @@ SYMBOLS = [
     "ada_cascade_step", "ada_select_full_host", "ada_cascade_step_host", "ada_gram_op_count",
     "ada_device_status", "ada_profile_enable", "ada_profile_read", "ada_status_string",
     "ada_select_full_noalloc", "ada_set_cooperative", "ada_selftest_wait_timeout", "ada_nearest_rep",
+    "ada_select_full_heads", "ada_cascade_step_heads",
 ]
 ADA_NOALLOC_MAX_T = 16384
 
@@ -58,6 +59,8 @@ def lib() -> C.CDLL:
         L.ada_cascade_step.argtypes = [vp, vp, i64, i64, i64, i64, C.c_int, C.c_double,
                                        i32p, i32p, i32p, i32p, i32p, i32p, i32p, i32p, fp, fp,
                                        C.c_uint32, vp]
+        L.ada_select_full_heads.argtypes = L.ada_select_full.argtypes
+        L.ada_cascade_step_heads.argtypes = L.ada_cascade_step.argtypes
         L.ada_nearest_rep.argtypes = [vp, vp, i64, i64, i64, i64, C.c_int, i32p, i32p, i32p, fp, vp]
         L.ada_select_full_host.argtypes = [vp, vp, i64, i64, i64, C.c_int, C.c_double, i32p, i32p, fp, vp]
         L.ada_cascade_step_host.argtypes = [vp, vp, i64, i64, i64, C.c_int, C.c_double,
@@ -230,6 +233,48 @@ def ada_cascade_step(ctx: Context, X: torch.Tensor, tau: float, rep_in: torch.Te
                                   out.rem_cnt.data_ptr(), _ptr(out.gamma_rep),
                                   _ptr(out.gamma_cross), flags, _stream(stream)),
            "ada_cascade_step")
+    return out
+
+
+def _shape_heads(X: torch.Tensor):
+    if X.dim() != 3 or X.stride(2) != 1 or X.stride(1) != X.shape[2]:
+        raise ValueError("X must be T x h x d_h with the heads of a token side by side")
+    T, h, d_h = X.shape
+    return T, h, d_h, X.stride(0)
+
+
+def ada_select_full_heads(ctx: Context, X: torch.Tensor, tau: float, rep_idx=None, rep_cnt=None,
+                          gamma=None, want_gamma=True, stream=None):
+    """Section 8.5: Definition 1 per head of X (T, h, d_h).  Returns (rep_idx[h,T], rep_cnt[h],
+    gamma[h,T] or None)."""
+    T, h, d_h, ldx = _shape_heads(X)
+    dev = X.device
+    if rep_idx is None:
+        rep_idx = torch.empty((h, T), dtype=torch.int32, device=dev)
+    if rep_cnt is None:
+        rep_cnt = torch.empty((h,), dtype=torch.int32, device=dev)
+    if gamma is None and want_gamma:
+        gamma = torch.empty((h, T), dtype=torch.float32, device=dev)
+    _check(lib().ada_select_full_heads(ctx.h, X.data_ptr(), T, h, d_h, ldx, dtype_of(X), float(tau),
+                                       rep_idx.data_ptr(), rep_cnt.data_ptr(), _ptr(gamma),
+                                       _stream(stream)), "ada_select_full_heads")
+    return rep_idx, rep_cnt, gamma
+
+
+def ada_cascade_step_heads(ctx: Context, X: torch.Tensor, tau: float, rep_in: torch.Tensor,
+                           rep_in_cnt: torch.Tensor, out: Optional[CascadeOut] = None,
+                           flags: int = 0, want_gamma=True, stream=None) -> CascadeOut:
+    """Section 8.5: Algorithm 1 per head of X (T, h, d_h); lists are [h, T], counts [h]."""
+    T, h, d_h, ldx = _shape_heads(X)
+    if out is None:
+        out = CascadeOut(h, T, X.device, want_gamma)
+    _check(lib().ada_cascade_step_heads(ctx.h, X.data_ptr(), T, h, d_h, ldx, dtype_of(X),
+                                        float(tau), rep_in.data_ptr(), rep_in_cnt.data_ptr(),
+                                        out.rep_out.data_ptr(), out.rep_out_cnt.data_ptr(),
+                                        out.add_idx.data_ptr(), out.add_cnt.data_ptr(),
+                                        out.rem_idx.data_ptr(), out.rem_cnt.data_ptr(),
+                                        _ptr(out.gamma_rep), _ptr(out.gamma_cross), flags,
+                                        _stream(stream)), "ada_cascade_step_heads")
     return out
 
 

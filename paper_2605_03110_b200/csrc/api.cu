@@ -249,17 +249,16 @@ ada_status ada_normalize(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int6
         return ADA_ERR_UNSUPPORTED;
     DeviceGuard guard(ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    CU(launch_norm_gather(ctx, X, (int)B, (int)T, (int)d, ldx, dt, inv_norm, Xhat,
+    CU(launch_norm_gather(ctx, X, (int)B, (int)T, (int)d, ldx, T * ldx, dt, inv_norm, Xhat,
                           gather ? rep_idx : nullptr, rep_cnt, nullptr, nullptr, Xrep, ctx->inv_rep,
                           s));
     return ADA_OK;
 }
 
-ada_status ada_select_full(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d,
-                           int64_t ldx, ada_dtype dt, double tau, int32_t* rep_idx,
-                           int32_t* rep_cnt, float* gamma, void* stream) {
-    ada_status st = check_common(ctx, X, B, T, d, ldx, dt);
-    if (st != ADA_OK) return st;
+// Definition 1 for B independent problems; row (b, t) of X starts at element b * xb + t * ldx
+static ada_status select_full_impl(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d,
+                                   int64_t ldx, int64_t xb, ada_dtype dt, double tau,
+                                   int32_t* rep_idx, int32_t* rep_cnt, float* gamma, void* stream) {
     if (rep_idx == nullptr || rep_cnt == nullptr || !tau_ok(tau)) return ADA_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -268,11 +267,11 @@ ada_status ada_select_full(ada_ctx* ctx, const void* X, int64_t B, int64_t T, in
     // the gamma scratch is zero on entry (workspace invariant kept by the compaction kernels)
     // long-K tensor-core launches compute the row norms themselves, hidden behind the MMAs
     const bool split = use_split(ctx, dt);
-    const bool tc = use_tc(ctx, dt), fuse = tc && d >= 2048 && B * T >= 4096;
+    const bool tc = use_tc(ctx, dt), fuse = tc && d >= 2048 && B * T >= 4096 && xb == T * ldx;
     if (split)   // one pass: 1/||x|| and the bf16 terms of X
-        CU(launch_split(ctx, X, (int)B, (int)T, (int)d, ldx, false, s));
+        CU(launch_split(ctx, X, (int)B, (int)T, (int)d, ldx, xb, false, s));
     else if (!fuse)
-        CU(launch_norm_gather(ctx, X, (int)B, (int)T, (int)d, ldx, dt, ctx->inv_norm, nullptr,
+        CU(launch_norm_gather(ctx, X, (int)B, (int)T, (int)d, ldx, xb, dt, ctx->inv_norm, nullptr,
                               nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, s));
     NormJob nj;
     nj.X = X; nj.ldx = ldx; nj.n_rows = B * T; nj.d = (int)d; nj.inv_norm = ctx->inv_norm;
@@ -280,7 +279,7 @@ ada_status ada_select_full(ada_ctx* ctx, const void* X, int64_t B, int64_t T, in
     memset(&p, 0, sizeof(p));
     p.A = X; p.Bm = X;
     p.lda = ldx; p.ldb = ldx;
-    p.a_batch = T * ldx; p.b_batch = T * ldx;
+    p.a_batch = xb; p.b_batch = xb;
     p.inv_a = ctx->inv_norm; p.inv_b = ctx->inv_norm;
     p.out = ctx->g_tok;
     p.n_dev = nullptr; p.n_host = (int)T;
@@ -299,14 +298,37 @@ ada_status ada_select_full(ada_ctx* ctx, const void* X, int64_t B, int64_t T, in
     return ADA_OK;
 }
 
-ada_status ada_cascade_step(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d,
-                            int64_t ldx, ada_dtype dt, double tau, const int32_t* rep_in,
-                            const int32_t* rep_in_cnt, int32_t* rep_out, int32_t* rep_out_cnt,
-                            int32_t* add_idx, int32_t* add_cnt, int32_t* rem_idx,
-                            int32_t* rem_cnt, float* gamma_rep, float* gamma_cross,
-                            uint32_t flags, void* stream) {
+ada_status ada_select_full(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d,
+                           int64_t ldx, ada_dtype dt, double tau, int32_t* rep_idx,
+                           int32_t* rep_cnt, float* gamma, void* stream) {
     ada_status st = check_common(ctx, X, B, T, d, ldx, dt);
     if (st != ADA_OK) return st;
+    return select_full_impl(ctx, X, B, T, d, ldx, T * ldx, dt, tau, rep_idx, rep_cnt, gamma, stream);
+}
+
+// heads interleaved inside each token's row: head j of token t starts at t * ldx + j * d_h
+static ada_status check_heads(ada_ctx* ctx, const void* X, int64_t T, int64_t h, int64_t d_h,
+                              int64_t ldx, ada_dtype dt) {
+    ada_status st = check_common(ctx, X, h, T, d_h, ldx, dt);
+    if (st != ADA_OK) return st;
+    return ldx < h * d_h ? ADA_ERR_INVALID_ARG : ADA_OK;
+}
+
+ada_status ada_select_full_heads(ada_ctx* ctx, const void* X, int64_t T, int64_t h, int64_t d_h,
+                                 int64_t ldx, ada_dtype dt, double tau, int32_t* rep_idx,
+                                 int32_t* rep_cnt, float* gamma, void* stream) {
+    ada_status st = check_heads(ctx, X, T, h, d_h, ldx, dt);
+    if (st != ADA_OK) return st;
+    return select_full_impl(ctx, X, h, T, d_h, ldx, d_h, dt, tau, rep_idx, rep_cnt, gamma, stream);
+}
+
+// Algorithm 1 for B independent problems; row (b, t) of X starts at element b * xb + t * ldx
+static ada_status cascade_impl(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d,
+                               int64_t ldx, int64_t xb, ada_dtype dt, double tau,
+                               const int32_t* rep_in, const int32_t* rep_in_cnt, int32_t* rep_out,
+                               int32_t* rep_out_cnt, int32_t* add_idx, int32_t* add_cnt,
+                               int32_t* rem_idx, int32_t* rem_cnt, float* gamma_rep,
+                               float* gamma_cross, uint32_t flags, void* stream) {
     if (rep_in == nullptr || rep_in_cnt == nullptr || rep_out == nullptr ||
         rep_out_cnt == nullptr || add_idx == nullptr || add_cnt == nullptr ||
         rem_idx == nullptr || rem_cnt == nullptr || !tau_ok(tau))
@@ -322,15 +344,16 @@ ada_status ada_cascade_step(ada_ctx* ctx, const void* X, int64_t B, int64_t T, i
     // map and its rows gathered into Xrep
     // tensor cores: one launch does lines 3-8; for long K it also computes line 1's row norms
     const bool split = use_split(ctx, dt);
-    const bool fuse = use_tc(ctx, dt) || split, fuse_norm = !split && fuse && d >= 2048 && B * T >= 4096;
-    CU(launch_norm_gather(ctx, X, (int)B, (int)T, (int)d, ldx, dt,
+    const bool fuse = use_tc(ctx, dt) || split,
+               fuse_norm = !split && fuse && d >= 2048 && B * T >= 4096 && xb == T * ldx;
+    CU(launch_norm_gather(ctx, X, (int)B, (int)T, (int)d, ldx, xb, dt,
                           (fuse_norm || split) ? nullptr : ctx->inv_norm,
                           nullptr, rep_in, rep_in_cnt, ctx->role, ctx->r_eff, ctx->Xrep,
                           ctx->inv_rep, s));
     NormJob nj;
     nj.X = X; nj.ldx = ldx; nj.n_rows = B * T; nj.d = (int)d; nj.inv_norm = ctx->inv_norm;
     if (split)   // 1/||x|| of all rows; bf16 terms of X and of the gathered rows
-        CU(launch_split(ctx, X, (int)B, (int)T, (int)d, ldx, true, s));
+        CU(launch_split(ctx, X, (int)B, (int)T, (int)d, ldx, xb, true, s));
     // lines 3-4: r x r Gram among inherited reps, max over earlier ones
     GramProblem p;
     memset(&p, 0, sizeof(p));
@@ -348,7 +371,7 @@ ada_status ada_cascade_step(ada_ctx* ctx, const void* X, int64_t B, int64_t T, i
     memset(&q, 0, sizeof(q));
     q.A = X; q.Bm = ctx->Xrep;
     q.lda = ldx; q.ldb = d;
-    q.a_batch = T * ldx; q.b_batch = T * d;
+    q.a_batch = xb; q.b_batch = T * d;
     q.inv_a = ctx->inv_norm; q.inv_b = ctx->inv_rep;
     q.out = ctx->g_tok;
     q.n_dev = ctx->r_eff; q.n_host = 0;
@@ -376,6 +399,32 @@ ada_status ada_cascade_step(ada_ctx* ctx, const void* X, int64_t B, int64_t T, i
     return ADA_OK;
 }
 
+ada_status ada_cascade_step(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d,
+                            int64_t ldx, ada_dtype dt, double tau, const int32_t* rep_in,
+                            const int32_t* rep_in_cnt, int32_t* rep_out, int32_t* rep_out_cnt,
+                            int32_t* add_idx, int32_t* add_cnt, int32_t* rem_idx,
+                            int32_t* rem_cnt, float* gamma_rep, float* gamma_cross,
+                            uint32_t flags, void* stream) {
+    ada_status st = check_common(ctx, X, B, T, d, ldx, dt);
+    if (st != ADA_OK) return st;
+    return cascade_impl(ctx, X, B, T, d, ldx, T * ldx, dt, tau, rep_in, rep_in_cnt, rep_out,
+                        rep_out_cnt, add_idx, add_cnt, rem_idx, rem_cnt, gamma_rep, gamma_cross,
+                        flags, stream);
+}
+
+ada_status ada_cascade_step_heads(ada_ctx* ctx, const void* X, int64_t T, int64_t h, int64_t d_h,
+                                  int64_t ldx, ada_dtype dt, double tau, const int32_t* rep_in,
+                                  const int32_t* rep_in_cnt, int32_t* rep_out,
+                                  int32_t* rep_out_cnt, int32_t* add_idx, int32_t* add_cnt,
+                                  int32_t* rem_idx, int32_t* rem_cnt, float* gamma_rep,
+                                  float* gamma_cross, uint32_t flags, void* stream) {
+    ada_status st = check_heads(ctx, X, T, h, d_h, ldx, dt);
+    if (st != ADA_OK) return st;
+    return cascade_impl(ctx, X, h, T, d_h, ldx, d_h, dt, tau, rep_in, rep_in_cnt, rep_out,
+                        rep_out_cnt, add_idx, add_cnt, rem_idx, rem_cnt, gamma_rep, gamma_cross,
+                        flags, stream);
+}
+
 ada_status ada_nearest_rep(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d,
                            int64_t ldx, ada_dtype dt, const int32_t* rep_idx,
                            const int32_t* rep_cnt, int32_t* nearest_idx, float* nearest_gamma,
@@ -388,9 +437,9 @@ ada_status ada_nearest_rep(ada_ctx* ctx, const void* X, int64_t B, int64_t T, in
     DeviceGuard guard(ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // role map and keys are zero on entry (workspace invariant); the finish kernel clears them
-    CU(launch_norm_gather(ctx, X, (int)B, (int)T, (int)d, ldx, dt, split ? nullptr : ctx->inv_norm,
+    CU(launch_norm_gather(ctx, X, (int)B, (int)T, (int)d, ldx, T * ldx, dt, split ? nullptr : ctx->inv_norm,
                           nullptr, rep_idx, rep_cnt, ctx->role, ctx->r_eff, ctx->Xrep, ctx->inv_rep, s));
-    if (split) CU(launch_split(ctx, X, (int)B, (int)T, (int)d, ldx, true, s));
+    if (split) CU(launch_split(ctx, X, (int)B, (int)T, (int)d, ldx, T * ldx, true, s));
     GramProblem q;
     memset(&q, 0, sizeof(q));
     q.A = X; q.Bm = ctx->Xrep;

@@ -136,11 +136,11 @@ void prof_end(ada_ctx* ctx, cudaStream_t s);
 
 // prep_kernels.cu
 cudaError_t launch_norm_gather(ada_ctx* ctx, const void* X, int B, int T, int d, int64_t ldx,
-                               ada_dtype dt, float* inv_norm, void* Xhat, const int32_t* rep_in,
+                               int64_t xb, ada_dtype dt, float* inv_norm, void* Xhat, const int32_t* rep_in,
                                const int32_t* rep_in_cnt, int32_t* role, int32_t* r_eff, void* Xrep,
                                float* inv_rep, cudaStream_t s);
-cudaError_t launch_split(ada_ctx* ctx, const void* X, int B, int T, int d, int64_t ldx, bool with_rep,
-                         cudaStream_t s);
+cudaError_t launch_split(ada_ctx* ctx, const void* X, int B, int T, int d, int64_t ldx, int64_t xb,
+                         bool with_rep, cudaStream_t s);
 cudaError_t launch_nearest_finish(ada_ctx* ctx, int B, int T, const int32_t* rep_idx,
                                   int32_t* nearest_idx, float* nearest_gamma, cudaStream_t s);
 cudaError_t launch_compact_full(ada_ctx* ctx, int B, int T, float thr, int32_t* rep_idx,

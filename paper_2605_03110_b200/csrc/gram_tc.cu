@@ -106,19 +106,30 @@ __device__ __forceinline__ int seg_tiles(const GramProblem& p, int par) {
     }
     return total;
 }
+// The tile ids a CTA takes from one segment ascend, so the search for a tile's sequence
+// resumes at the sequence of the previous tile: `b` is that sequence, `base` the id of its
+// first tile.  (With dozens of short sequences -- heads -- a search from sequence 0 for every
+// tile would cost more than the tile's main loop.)
+struct TileCursor {
+    int b, base;
+};
 // tile `id` of segment p -> piece; false when id is past the segment's last tile
-__device__ __forceinline__ bool decode_tile(const GramProblem& p, int par, int id, Piece& t) {
+__device__ __forceinline__ bool decode_tile(const GramProblem& p, int par, int id, Piece& t,
+                                            TileCursor& cur) {
     const int tw = par;
-    for (int b = 0; b < p.B; ++b) {
+    for (; cur.b < p.B; ++cur.b) {
+        const int b = cur.b;
         const int n = seq_n(p, b);
-        if (n <= 0) continue;
-        int cnt, nct = 0, w = 0;
-        if (p.tri) cnt = tri_tiles(n, tw);
-        else {
-            cross_cols(n, par, nct, w);
-            cnt = ((p.rows + BM - 1) / BM) * nct;
+        int cnt = 0, nct = 0, w = 0;
+        if (n > 0) {
+            if (p.tri) cnt = tri_tiles(n, tw);
+            else {
+                cross_cols(n, par, nct, w);
+                cnt = ((p.rows + BM - 1) / BM) * nct;
+            }
         }
-        if (id >= cnt) { id -= cnt; continue; }
+        if (id - cur.base >= cnt) { cur.base += cnt; continue; }
+        id -= cur.base;
         t.b = b;
         t.n = n;
         int nc;
@@ -167,6 +178,36 @@ __device__ __forceinline__ bool dead_tile(const GramProblem& p, const Piece& pc)
     return p.col_token[(int64_t)pc.b * p.cap + pc.col0] >= pc.row0 + BM;
 }
 
+// The first TAB tiles of every CTA are decoded once, by TAB threads in parallel while the
+// kernel starts, into a table in shared memory: with a short contraction a tile's main loop
+// is a few hundred cycles, less than the serial integer work of decoding it three times
+// (producer, MMA issuer, epilogue).  Entry: x = row0 | ncols/16 << 24 | dead << 31, y = col0,
+// z = n (0: no tile), w = sequence.  Tiles past the table are decoded on the fly.
+constexpr int TAB = 80;
+struct SharedTc : Shared {
+    uint4 tile_tab[TAB];
+};
+constexpr int SMEM_TC_BYTES = RING_BYTES + (int)sizeof(SharedTc) + 1024;
+static_assert(SMEM_TC_BYTES <= 227 * 1024, "shared memory budget");
+
+// 0: no such tile, 1: tile in pc, 2: tile in pc but nothing to do (dead_tile)
+__device__ __forceinline__ int next_tile(const uint4* tab, int it, const GramProblem& p, int par,
+                                         int local_id, Piece& pc, TileCursor& cur) {
+    if (it < TAB) {
+        const uint4 e = tab[it];
+        if (e.z == 0u) return 0;
+        pc.row0 = (int)(e.x & 0xFFFFFFu);
+        pc.ncols = (int)((e.x >> 24) & 31u) * 16;
+        pc.col0 = (int)e.y;
+        pc.n = (int)e.z;
+        pc.b = (int)e.w;
+        pc.m = p.tri ? pc.n : p.rows;
+        return (e.x >> 31) ? 2 : 1;
+    }
+    if (!decode_tile(p, par, local_id, pc, cur)) return 0;
+    return dead_tile(p, pc) ? 2 : 1;
+}
+
 struct GramMaps {
     CUtensorMap a[2], b[2];       // per segment: left operand (128-row boxes), right operand (64-row boxes)
 };
@@ -179,7 +220,7 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-    Shared& sh = *reinterpret_cast<Shared*>(smem + RING_BYTES);
+    SharedTc& sh = *reinterpret_cast<SharedTc*>(smem + RING_BYTES);
     volatile int* abort_flag = &sh.abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -228,6 +269,21 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
     const unsigned tmem_base = sh.tmem_base;
     const int tiles0 = sh.tiles0, total = sh.tiles0 + sh.tiles1, par0 = sh.par0, par1 = sh.par1;
     Piece pc;
+    if (threadIdx.x < TAB) {
+        const int id = blockIdx.x + (int)threadIdx.x * (int)gridDim.x;
+        uint4 e = make_uint4(0u, 0u, 0u, 0u);
+        if (id < total) {
+            const int sg = id < tiles0 ? 0 : 1;
+            const GramProblem& p = sg ? seg1 : seg0;
+            TileCursor c0 = {0, 0};
+            if (decode_tile(p, sg ? par1 : par0, id - (sg ? tiles0 : 0), pc, c0))
+                e = make_uint4((unsigned)pc.row0 | ((unsigned)(pc.ncols >> 4) << 24) |
+                                   (dead_tile(p, pc) ? 0x80000000u : 0u),
+                               (unsigned)pc.col0, (unsigned)pc.n, (unsigned)pc.b);
+        }
+        sh.tile_tab[threadIdx.x] = e;
+    }
+    __syncthreads();
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
@@ -237,11 +293,17 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
             unsigned ever = 0;       // stages ever filled
             int cur_sb = 0, cur_nst = 0, s = 0;
             bool ok = true;
-            for (int id = blockIdx.x; ok && id < total; id += gridDim.x) {
+            TileCursor cur = {0, 0};
+            int cur_sg = 0;
+            int it = 0;
+            for (int id = blockIdx.x; ok && id < total; id += gridDim.x, ++it) {
                 const int sg = id < tiles0 ? 0 : 1;
                 const GramProblem& p = sg ? seg1 : seg0;
-                if (!decode_tile(p, sg ? par1 : par0, id - (sg ? tiles0 : 0), pc)) break;
-                if (dead_tile(p, pc)) continue;   // causal cross tile with no admissible pair
+                if (sg != cur_sg) { cur.b = 0; cur.base = 0; cur_sg = sg; }
+                const int got_tile = next_tile(sh.tile_tab, it, p, sg ? par1 : par0,
+                                               id - (sg ? tiles0 : 0), pc, cur);
+                if (got_tile == 0) break;
+                if (got_tile == 2) continue;      // causal cross tile with no admissible pair
                 const int ksub = stage_ksub(pc.ncols, p.d);
                 const int num_kb = (p.d + BK * ksub - 1) / (BK * ksub);
                 const int nbox = (pc.ncols + BOX_N - 1) / BOX_N;
@@ -287,11 +349,17 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
             unsigned uses = 0, tile_it = 0;   // bit s of `uses`: parity of the number of uses of stage s
             int cur_sb = 0, cur_nst = 0, s = 0;
             bool ok = true;
-            for (int id = blockIdx.x; ok && id < total; id += gridDim.x) {
+            TileCursor cur = {0, 0};
+            int cur_sg = 0;
+            int it = 0;
+            for (int id = blockIdx.x; ok && id < total; id += gridDim.x, ++it) {
                 const int sg = id < tiles0 ? 0 : 1;
                 const GramProblem& p = sg ? seg1 : seg0;
-                if (!decode_tile(p, sg ? par1 : par0, id - (sg ? tiles0 : 0), pc)) break;
-                if (dead_tile(p, pc)) continue;   // causal cross tile with no admissible pair
+                if (sg != cur_sg) { cur.b = 0; cur.base = 0; cur_sg = sg; }
+                const int got_tile = next_tile(sh.tile_tab, it, p, sg ? par1 : par0,
+                                               id - (sg ? tiles0 : 0), pc, cur);
+                if (got_tile == 0) break;
+                if (got_tile == 2) continue;      // causal cross tile with no admissible pair
                 const int ksub = stage_ksub(pc.ncols, p.d);
                 const int num_kb = (p.d + BK * ksub - 1) / (BK * ksub);
                 const int subb = sub_bytes(pc.ncols);
@@ -339,11 +407,17 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
         bool norm_ok = norms.X == nullptr;           // row norms computed by this launch's norm warps
         const unsigned norm_total = (unsigned)(gridDim.x * NORM_WARPS);      // cross epilogues must see segment 0 finished
         unsigned tile_it = 0;
-        for (int id = blockIdx.x; id < total; id += gridDim.x) {
+        TileCursor cur = {0, 0};
+            int cur_sg = 0;
+        int it = 0;
+        for (int id = blockIdx.x; id < total; id += gridDim.x, ++it) {
             const int sg = id < tiles0 ? 0 : 1;
             const GramProblem& p = sg ? seg1 : seg0;
-            if (!decode_tile(p, sg ? par1 : par0, id - (sg ? tiles0 : 0), pc)) break;
-                if (dead_tile(p, pc)) continue;   // causal cross tile with no admissible pair
+            if (sg != cur_sg) { cur.b = 0; cur.base = 0; cur_sg = sg; }
+            const int got_tile = next_tile(sh.tile_tab, it, p, sg ? par1 : par0,
+                                           id - (sg ? tiles0 : 0), pc, cur);
+            if (got_tile == 0) break;
+            if (got_tile == 2) continue;          // causal cross tile with no admissible pair
             const unsigned acc = tile_it & 1u, acc_ph = (tile_it >> 1) & 1u;
                 ++tile_it;
             const int64_t o = (int64_t)pc.b * p.cap;
@@ -360,57 +434,97 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
             }
             // stage this tile's column factors (0 for inadmissible columns); warp-private copy
             __syncwarp();
-            for (int c = lane; c < ncols32; c += 32) {
-                const int col = pc.col0 + c;
-                float f = 0.f;
-                int tok = col;
-                if (c < ncols && col < pc.n) {
-                    f = __ldcg(p.inv_b + o + col);
-                    if (!p.tri) {
-                        // representative removed at line 5 (written earlier in this launch: read at L2)
-                        if (!(__ldcg(p.col_gate + o + col) < p.thr_bits)) f = 0.f;
-                        if (p.causal) tok = p.col_token[o + col];
+            {
+                // all of the tile's global loads are issued before the first is used: with a
+                // short contraction the epilogue is the critical path, and eight dependent
+                // round trips to L2 would be most of it
+                float fb[BN / 32];
+                unsigned gate[BN / 32] = {};
+                int tk[BN / 32] = {};
+                // (columns past the tile are clamped to its last one and discarded afterwards,
+                // so that no load hangs on a data-dependent branch)
+                const int last = pc.n - 1;
+#pragma unroll
+                for (int q = 0; q < BN / 32; ++q)
+                    fb[q] = __ldcg(p.inv_b + o + min(pc.col0 + lane + 32 * q, last));
+                if (!p.tri) {
+                    // representative removed at line 5 (written earlier in this launch: read at L2)
+#pragma unroll
+                    for (int q = 0; q < BN / 32; ++q)
+                        gate[q] = __ldcg(p.col_gate + o + min(pc.col0 + lane + 32 * q, last));
+                }
+                if (!p.tri && p.causal) {
+#pragma unroll
+                    for (int q = 0; q < BN / 32; ++q)
+                        tk[q] = p.col_token[o + min(pc.col0 + lane + 32 * q, last)];
+                }
+#pragma unroll
+                for (int q = 0; q < BN / 32; ++q) {
+                    const int c = lane + 32 * q, col = pc.col0 + c;
+                    const bool live = c < ncols && col < pc.n;
+                    if (c < ncols32) {
+                        cs[c] = (live && (p.tri || gate[q] < p.thr_bits)) ? fb[q] : 0.f;
+                        ct[c] = (live && !p.tri && p.causal) ? tk[q] : col;
                     }
                 }
-                cs[c] = f;
-                ct[c] = tok;
             }
             __syncwarp();
+            // this thread's row: its role and inverse norm are fetched while the MMAs finish
+            const int row = pc.row0 + quad * 32 + lane;
+            const bool row_live = row < pc.m;
+            const bool skip = row_live && !p.tri && p.row_role[o + row] != 0;   // inherited reps are not candidates
+            const bool inv_early = !(p.wait_norm_a && !norm_ok);
+            float inv_row = (row_live && inv_early) ? __ldcg(p.inv_a + o + row) : 0.f;
             // warp-uniform outcome of the bounded wait
             const bool got = mbar_wait(&sh.tmem_full[acc], acc_ph, abort_flag, 4);
             if (!__all_sync(0xffffffffu, got)) break;
             tcgen05_fence_after();
-            const int row = pc.row0 + quad * 32 + lane;
             const bool need_cmp = p.tri ? (pc.col0 + ncols > pc.row0) : (p.causal != 0);
-            float mx = 0.f;
-            int arg = 0;                                  // nearest-representative mode: column of mx
+            float mx4[2] = {0.f, 0.f};                    // independent partial maxima
+            int arg = 0;                                  // nearest-representative mode: column of the maximum
             const bool want_arg = p.out_arg != nullptr;
-            for (int c0 = 0; c0 < ncols32; c0 += 32) {
-                float v[32];
-                tmem_ld32(tmem_base + ((unsigned)(quad * 32) << 16) + acc * BN + c0, v);
-                if (want_arg) {
+            const unsigned tbase = tmem_base + ((unsigned)(quad * 32) << 16) + acc * BN;
+            if (want_arg) {
+                for (int c0 = 0; c0 < ncols32; c0 += 32) {
+                    float v[32];
+                    tmem_ld32(tbase + c0, v);
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {        // ascending columns, strict '>': lowest index on ties
                         const float x = fabsf(v[j]) * cs[c0 + j];
-                        if (x > mx) { mx = x; arg = c0 + j; }
-                    }
-                } else if (!need_cmp) {
-#pragma unroll
-                    for (int j = 0; j < 32; j += 4) {
-                        const float4 f = *reinterpret_cast<const float4*>(cs + c0 + j);
-                        mx = fmaxf(mx, fabsf(v[j]) * f.x);
-                        mx = fmaxf(mx, fabsf(v[j + 1]) * f.y);
-                        mx = fmaxf(mx, fabsf(v[j + 2]) * f.z);
-                        mx = fmaxf(mx, fabsf(v[j + 3]) * f.w);
-                    }
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const float x = fabsf(v[j]) * cs[c0 + j];
-                        if (ct[c0 + j] < row) mx = fmaxf(mx, x);
+                        if (x > mx4[0]) { mx4[0] = x; arg = c0 + j; }
                     }
                 }
+            } else {
+                auto consume = [&](const unsigned (&r)[32], int c0) {
+                    if (!need_cmp) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            const float4 f = *reinterpret_cast<const float4*>(cs + c0 + j);
+                            mx4[0] = fmaxf(mx4[0], fabsf(__uint_as_float(r[j])) * f.x);
+                            mx4[1] = fmaxf(mx4[1], fabsf(__uint_as_float(r[j + 1])) * f.y);
+                            mx4[0] = fmaxf(mx4[0], fabsf(__uint_as_float(r[j + 2])) * f.z);
+                            mx4[1] = fmaxf(mx4[1], fabsf(__uint_as_float(r[j + 3])) * f.w);
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            const float4 f = *reinterpret_cast<const float4*>(cs + c0 + j);
+                            const int4 t = *reinterpret_cast<const int4*>(ct + c0 + j);
+                            if (t.x < row) mx4[0] = fmaxf(mx4[0], fabsf(__uint_as_float(r[j])) * f.x);
+                            if (t.y < row) mx4[1] = fmaxf(mx4[1], fabsf(__uint_as_float(r[j + 1])) * f.y);
+                            if (t.z < row) mx4[0] = fmaxf(mx4[0], fabsf(__uint_as_float(r[j + 2])) * f.z);
+                            if (t.w < row) mx4[1] = fmaxf(mx4[1], fabsf(__uint_as_float(r[j + 3])) * f.w);
+                        }
+                    }
+                };
+                for (int c0 = 0; c0 < ncols32; c0 += 32) {
+                    unsigned ra[32];
+                    tmem_ld32_issue(tbase + c0, ra);
+                    tmem_ld_wait(ra);
+                    consume(ra, c0);
+                }
             }
+            float mx = fmaxf(mx4[0], mx4[1]);
             // accumulator consumed: hand it back to the MMA warp
             tcgen05_fence_before();
             __syncwarp();
@@ -419,10 +533,10 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
                 if (!wait_counter(dep_ctr + 1, norm_total, lane, abort_flag, 9)) break;
                 norm_ok = true;
             }
-            if (row < pc.m) {
-                const bool skip = !p.tri && p.row_role[o + row] != 0;   // inherited reps are not candidates
+            if (row_live) {
                 if (!skip) {
-                    mx *= __ldcg(p.inv_a + o + row);
+                    if (!inv_early) inv_row = __ldcg(p.inv_a + o + row);
+                    mx *= inv_row;
                     if (want_arg) {
                         const unsigned long long key =
                             ((unsigned long long)__float_as_uint(mx) << 32) |
@@ -492,7 +606,7 @@ cudaError_t launch_gram_tc(ada_ctx* ctx, const GramProblem* tri, const GramProbl
                            const NormJob* norms, cudaStream_t s) {
     if (!ctx->tc_attr_set) {
         cudaError_t e = cudaFuncSetAttribute(k_gram_tc, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             SMEM_BYTES);
+                                             SMEM_TC_BYTES);
         if (e != cudaSuccess) return e;
         ctx->tc_attr_set = true;
     }
@@ -525,7 +639,7 @@ cudaError_t launch_gram_tc(ada_ctx* ctx, const GramProblem* tri, const GramProbl
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3(ctx->sm_count);
     cfg.blockDim = dim3(NUM_THREADS);
-    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.dynamicSmemBytes = SMEM_TC_BYTES;
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeCooperative;

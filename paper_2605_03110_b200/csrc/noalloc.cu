@@ -107,7 +107,7 @@ extern "C" ada_status ada_select_full_noalloc(const void* X, int64_t T, int64_t 
     // that must start at zero -- the gamma bit patterns and the status/counter words.
     if (cudaMemsetAsync(ctx->g_tok, 0, (size_t)T * 4, s) != cudaSuccess) return ADA_ERR_CUDA;
     if (cudaMemsetAsync(ctx->status, 0, kTailBytes, s) != cudaSuccess) return ADA_ERR_CUDA;
-    if (launch_norm_gather(ctx, X, 1, (int)T, (int)d, ldx, dt, ctx->inv_norm, nullptr, nullptr,
+    if (launch_norm_gather(ctx, X, 1, (int)T, (int)d, ldx, T * ldx, dt, ctx->inv_norm, nullptr, nullptr,
                            nullptr, nullptr, nullptr, nullptr, nullptr, s) != cudaSuccess)
         return ADA_ERR_CUDA;
     GramProblem p;

@@ -79,7 +79,7 @@ __device__ __forceinline__ float warp_row_sumsq(const uint4* __restrict__ src, i
 // no dependency between them and no separate scatter pass.
 template <typename T>
 __global__ void __launch_bounds__(256)
-k_norm_gather(const T* __restrict__ X, int64_t n_rows, int Tseq, int d, int64_t ldx,
+k_norm_gather(const T* __restrict__ X, int64_t n_rows, int Tseq, int d, int64_t ldx, int64_t xb,
               float* __restrict__ inv_norm, T* __restrict__ Xhat,
               const int32_t* __restrict__ rep_in, const int32_t* __restrict__ rep_in_cnt,
               int32_t* __restrict__ role, int32_t* __restrict__ r_eff, T* __restrict__ Xrep,
@@ -91,7 +91,9 @@ k_norm_gather(const T* __restrict__ X, int64_t n_rows, int Tseq, int d, int64_t 
     const int nvec = d / N;  // d*es is a multiple of 16 bytes
     if (w < n_rows) {
         const int64_t row = w;
-        const uint4* src = reinterpret_cast<const uint4*>(X + row * ldx);
+        // row (b, t) of X starts at b * xb + t * ldx (xb = Tseq * ldx for stacked sequences,
+        // the head width for heads interleaved inside one row)
+        const uint4* src = reinterpret_cast<const uint4*>(X + (row / Tseq) * xb + (row % Tseq) * ldx);
         const float ss = warp_row_sumsq<T>(src, nvec, lane);
         float inv = 0.f;
         if (!(ss <= 3.0e38f)) {  // NaN or overflow to Inf
@@ -127,7 +129,7 @@ k_norm_gather(const T* __restrict__ X, int64_t n_rows, int Tseq, int d, int64_t 
         return;
     }
     const int64_t prow = (int64_t)b * Tseq + i;
-    const uint4* src = reinterpret_cast<const uint4*>(X + ((int64_t)b * Tseq + idx) * ldx);
+    const uint4* src = reinterpret_cast<const uint4*>(X + (int64_t)b * xb + (int64_t)idx * ldx);
     uint4* dst = reinterpret_cast<uint4*>(Xrep + prow * (int64_t)d);
     float ss = 0.f;
     int v = lane;
@@ -155,7 +157,7 @@ k_norm_gather(const T* __restrict__ X, int64_t n_rows, int Tseq, int d, int64_t 
 }
 
 cudaError_t launch_norm_gather(ada_ctx* ctx, const void* X, int B, int T, int d, int64_t ldx,
-                               ada_dtype dt, float* inv_norm, void* Xhat, const int32_t* rep_in,
+                               int64_t xb, ada_dtype dt, float* inv_norm, void* Xhat, const int32_t* rep_in,
                                const int32_t* rep_in_cnt, int32_t* role, int32_t* r_eff, void* Xrep,
                                float* inv_rep, cudaStream_t s) {
     const int64_t n_rows = (int64_t)B * T;
@@ -166,11 +168,11 @@ cudaError_t launch_norm_gather(ada_ctx* ctx, const void* X, int B, int T, int d,
     prof_begin(ctx, K_NORM_GATHER, s);
     if (dt == ADA_F32) {
         k_norm_gather<float><<<grid, warps * 32, 0, s>>>(
-            (const float*)X, n_rows, T, d, ldx, inv_norm, (float*)Xhat, rep_in, rep_in_cnt, role,
+            (const float*)X, n_rows, T, d, ldx, xb, inv_norm, (float*)Xhat, rep_in, rep_in_cnt, role,
             r_eff, (float*)Xrep, inv_rep, ctx->status);
     } else {
         k_norm_gather<__nv_bfloat16><<<grid, warps * 32, 0, s>>>(
-            (const __nv_bfloat16*)X, n_rows, T, d, ldx, inv_norm, (__nv_bfloat16*)Xhat, rep_in,
+            (const __nv_bfloat16*)X, n_rows, T, d, ldx, xb, inv_norm, (__nv_bfloat16*)Xhat, rep_in,
             rep_in_cnt, role, r_eff, (__nv_bfloat16*)Xrep, inv_rep, ctx->status);
     }
     prof_end(ctx, s);
@@ -192,6 +194,7 @@ cudaError_t launch_norm_gather(ada_ctx* ctx, const void* X, int B, int T, int d,
 struct SplitJob {
     const float* X;          // rows to split
     int64_t ldx;             // row stride of X in elements
+    int64_t xb;              // sequence stride of X in elements
     int rows_per_seq;        // rows per sequence (capacity)
     const int32_t* n_dev;    // [B] rows actually present per sequence, or NULL = all
     __nv_bfloat16* A;        // [B*rows_per_seq][6d]
@@ -219,7 +222,8 @@ k_split_bf16(const SplitJob j0, const SplitJob j1, int64_t n_rows, int d, unsign
         const int b = (int)(w / j.rows_per_seq), i = (int)(w % j.rows_per_seq);
         if (i >= j.n_dev[b]) return;
     }
-    const float4* src = reinterpret_cast<const float4*>(j.X + w * j.ldx);
+    const float4* src = reinterpret_cast<const float4*>(j.X + (w / j.rows_per_seq) * j.xb +
+                                                        (w % j.rows_per_seq) * j.ldx);
     __nv_bfloat16* a = j.A + w * (int64_t)(6 * d);
     __nv_bfloat16* bm = j.Bm + w * (int64_t)(6 * d);
     float ss = 0.f;
@@ -266,15 +270,15 @@ k_split_bf16(const SplitJob j0, const SplitJob j1, int64_t n_rows, int d, unsign
 }
 
 // X (B*T rows) -> ctx->splitXA/XB (+ inv_norm); with_rep: ctx->Xrep rows below r_eff -> splitRA/RB
-cudaError_t launch_split(ada_ctx* ctx, const void* X, int B, int T, int d, int64_t ldx, bool with_rep,
-                         cudaStream_t s) {
+cudaError_t launch_split(ada_ctx* ctx, const void* X, int B, int T, int d, int64_t ldx, int64_t xb,
+                         bool with_rep, cudaStream_t s) {
     const int64_t n_rows = (int64_t)B * T;
     SplitJob j0, j1;
-    j0.X = static_cast<const float*>(X); j0.ldx = ldx; j0.rows_per_seq = T; j0.n_dev = nullptr;
+    j0.X = static_cast<const float*>(X); j0.ldx = ldx; j0.xb = xb; j0.rows_per_seq = T; j0.n_dev = nullptr;
     j0.A = static_cast<__nv_bfloat16*>(ctx->splitXA); j0.Bm = static_cast<__nv_bfloat16*>(ctx->splitXB);
     j0.inv_norm = ctx->inv_norm;
     j1 = j0;
-    j1.X = with_rep ? static_cast<const float*>(ctx->Xrep) : nullptr; j1.ldx = d; j1.n_dev = ctx->r_eff;
+    j1.X = with_rep ? static_cast<const float*>(ctx->Xrep) : nullptr; j1.ldx = d; j1.xb = (int64_t)T * d; j1.n_dev = ctx->r_eff;
     j1.A = static_cast<__nv_bfloat16*>(ctx->splitRA); j1.Bm = static_cast<__nv_bfloat16*>(ctx->splitRB);
     j1.inv_norm = nullptr;
     const int warps = 8;

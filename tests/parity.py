@@ -39,12 +39,18 @@ def check_set(got, gamma_ref, candidates, thr, tol):
     return band
 
 
-def check_full(ctx, Xnp, tau, stream=None):
-    """ada_select_full vs the oracle on every sequence.  Returns band count."""
+def check_full(ctx, Xnp, tau, stream=None, heads=False):
+    """ada_select_full vs the oracle on every sequence.  Returns band count.
+    heads: Xnp is (T, h, d_h); the device gets it as it is (ada_select_full_heads), the oracle
+    gets each head as a sequence of its own."""
     tol = TOL[dtype_name(Xnp)]
     thr = 1.0 - tau * tau
     Xd = to_device(Xnp)
-    rep_idx, rep_cnt, gamma = ada.ada_select_full(ctx, Xd, tau)
+    if heads:
+        rep_idx, rep_cnt, gamma = ada.ada_select_full_heads(ctx, Xd, tau)
+        Xnp = np.ascontiguousarray(Xnp.transpose(1, 0, 2))
+    else:
+        rep_idx, rep_cnt, gamma = ada.ada_select_full(ctx, Xd, tau)
     st, _ = ada.ada_device_status(ctx)
     assert st == 0, ada.status_string(st)
     reps = lists(rep_idx, rep_cnt)
@@ -61,20 +67,22 @@ def check_full(ctx, Xnp, tau, stream=None):
     return band, reps
 
 
-def check_cascade(ctx, Xnp, tau, rep_in_lists, causal=False):
-    """ada_cascade_step vs the oracle, same inherited sets on both sides."""
+def check_cascade(ctx, Xnp, tau, rep_in_lists, causal=False, heads=False):
+    """ada_cascade_step vs the oracle, same inherited sets on both sides (heads: as check_full)."""
     tol = TOL[dtype_name(Xnp)]
     thr = 1.0 - tau * tau
-    B, T, _ = Xnp.shape
     Xd = to_device(Xnp)
+    if heads:
+        Xnp = np.ascontiguousarray(Xnp.transpose(1, 0, 2))
+    B, T, _ = Xnp.shape
     rin = np.zeros((B, T), dtype=np.int32)
     rcnt = np.zeros(B, dtype=np.int32)
     for b, r in enumerate(rep_in_lists):
         rin[b, :len(r)] = r
         rcnt[b] = len(r)
-    out = ada.ada_cascade_step(ctx, Xd, tau, torch.from_numpy(rin).cuda(),
-                               torch.from_numpy(rcnt).cuda(),
-                               flags=ada.ADA_CROSS_CAUSAL if causal else 0)
+    step = ada.ada_cascade_step_heads if heads else ada.ada_cascade_step
+    out = step(ctx, Xd, tau, torch.from_numpy(rin).cuda(), torch.from_numpy(rcnt).cuda(),
+               flags=ada.ADA_CROSS_CAUSAL if causal else 0)
     st, _ = ada.ada_device_status(ctx)
     assert st == 0, ada.status_string(st)
     rep, add, rem = lists(out.rep_out, out.rep_out_cnt), lists(out.add_idx, out.add_cnt), \
