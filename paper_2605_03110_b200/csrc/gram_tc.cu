@@ -34,6 +34,22 @@ using namespace tc;
 
 namespace {
 
+// The kernel comes in two shapes.  The long-contraction shape (14 warps, the last eight for the
+// optional row norms) lives off its main loop: one epilogue set, a 216 KiB ring whose stage size
+// follows each tile's width.  The short-contraction shape (d <= 512, e.g. one attention head)
+// lives off its epilogue, because a 128 x 256 fp32 accumulator takes about 2300 cycles to read
+// out of TMEM, more than such a tile's main loop: 10 warps, two epilogue sets that take
+// alternate tiles (one accumulator each, so that one set's bookkeeping -- tile lookup, column
+// factors, barrier, atomics -- overlaps the other's TMEM reads), a ring geometry fixed per
+// segment (no drain between tiles of different width), one 256-row TMA box for a full-width
+// right operand, and a 208 KiB ring to make room for the second set's column factors.
+template <bool SHORTK>
+struct Shape {
+    static constexpr int RING = SHORTK ? 208 * 1024 : RING_BYTES;
+    static constexpr int EPI_WARPS = SHORTK ? 8 : 4;
+    static constexpr int THREADS = SHORTK ? 64 + 32 * 8 : NUM_THREADS;
+};
+
 // ---------------------------------------------------------------- work schedule
 // A launch covers up to two problems ("segments"): a triangular one (Definition 1 on X, or
 // Algorithm 1 lines 3-4 on the gathered representatives) and a cross one (lines 7-8).
@@ -69,11 +85,11 @@ __device__ __forceinline__ int sub_bytes(int ncols) {
 // once per 128 K elements; one for wider tiles
 // (short contractions keep one: with a dozen K blocks the coarser pipeline costs more than
 // it saves)
-__device__ __forceinline__ int stage_ksub(int ncols, int d) {
-    return (d >= 2048 && 3 * 2 * sub_bytes(ncols) <= RING_BYTES) ? 2 : 1;
+__device__ __forceinline__ int stage_ksub(int ncols, int d, int ring) {
+    return (d >= 2048 && 3 * 2 * sub_bytes(ncols) <= ring) ? 2 : 1;
 }
-__device__ __forceinline__ int stage_count(int sbytes) {
-    return min(MAX_STAGES, RING_BYTES / sbytes);
+__device__ __forceinline__ int stage_count(int sbytes, int ring) {
+    return min(MAX_STAGES, ring / sbytes);
 }
 // cross: columns are cut into nct equal tiles of width w (multiple of 16, <= 256).  `want` is
 // the number of column tiles per row tile that would give every CTA one tile: a problem
@@ -84,28 +100,7 @@ __device__ __forceinline__ void cross_cols(int n, int want, int& nct, int& w) {
     nct = min(max(want, lo), hi);
     w = nct > 0 ? ((((n + nct - 1) / nct) + 15) & ~15) : 0;
 }
-// column tiles per row tile that fill the grid once (cross segment)
-__device__ __forceinline__ int cross_want(const GramProblem& p, int G) {
-    int row_tiles = 0;
-    for (int b = 0; b < p.B; ++b)
-        if (seq_n(p, b) > 0) row_tiles += (p.rows + BM - 1) / BM;
-    return row_tiles > 0 ? max(1, G / row_tiles) : 1;
-}
-// `par`: column tile width (triangular segment) or wanted column tiles per row tile (cross)
-__device__ __forceinline__ int seg_tiles(const GramProblem& p, int par) {
-    int total = 0;
-    for (int b = 0; b < p.B; ++b) {
-        const int n = seq_n(p, b);
-        if (n <= 0) continue;
-        if (p.tri) total += tri_tiles(n, par);
-        else {
-            int nct, w;
-            cross_cols(n, par, nct, w);
-            total += ((p.rows + BM - 1) / BM) * nct;
-        }
-    }
-    return total;
-}
+// `par` below: column tile width (triangular segment) or wanted column tiles per row tile (cross)
 // The tile ids a CTA takes from one segment ascend, so the search for a tile's sequence
 // resumes at the sequence of the previous tile: `b` is that sequence, `base` the id of its
 // first tile.  (With dozens of short sequences -- heads -- a search from sequence 0 for every
@@ -184,11 +179,28 @@ __device__ __forceinline__ bool dead_tile(const GramProblem& p, const Piece& pc)
 // (producer, MMA issuer, epilogue).  Entry: x = row0 | ncols/16 << 24 | dead << 31, y = col0,
 // z = n (0: no tile), w = sequence.  Tiles past the table are decoded on the fly.
 constexpr int TAB = 80;
-struct SharedTc : Shared {
+template <bool SHORTK>
+struct alignas(16) SharedTc {
+    unsigned long long full[MAX_STAGES];
+    unsigned long long empty[MAX_STAGES];
+    unsigned long long tmem_full[2];
+    unsigned long long tmem_empty[2];
+    unsigned long long drain;
+    unsigned tmem_base;
+    int abort_flag;
+    int tiles0, tiles1, par0, par1;
+    int wide0, wide1;           // widest tile of each segment (fixes the segment's ring geometry)
     uint4 tile_tab[TAB];
+    // per epilogue warp, so that staging needs no barrier across warps
+    alignas(16) float col_scale[Shape<SHORTK>::EPI_WARPS][BN];
+    alignas(16) int col_token[Shape<SHORTK>::EPI_WARPS][BN];
 };
-constexpr int SMEM_TC_BYTES = RING_BYTES + (int)sizeof(SharedTc) + 1024;
-static_assert(SMEM_TC_BYTES <= 227 * 1024, "shared memory budget");
+template <bool SHORTK>
+constexpr int smem_tc_bytes() {
+    return Shape<SHORTK>::RING + (int)sizeof(SharedTc<SHORTK>) + 1024;   // +1024: alignment slack
+}
+static_assert(smem_tc_bytes<false>() <= 227 * 1024 && smem_tc_bytes<true>() <= 227 * 1024,
+              "shared memory budget");
 
 // 0: no such tile, 1: tile in pc, 2: tile in pc but nothing to do (dead_tile)
 __device__ __forceinline__ int next_tile(const uint4* tab, int it, const GramProblem& p, int par,
@@ -209,10 +221,12 @@ __device__ __forceinline__ int next_tile(const uint4* tab, int it, const GramPro
 }
 
 struct GramMaps {
-    CUtensorMap a[2], b[2];       // per segment: left operand (128-row boxes), right operand (64-row boxes)
+    // per segment: left operand (128-row boxes), right operand in 64-row and in 256-row boxes
+    CUtensorMap a[2], b[2], bw[2];
 };
 
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+template <bool SHORTK>
+__global__ void __launch_bounds__(Shape<SHORTK>::THREADS, 1)
 k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramProblem seg0,
           const __grid_constant__ GramProblem seg1, const int nseg,
           const __grid_constant__ NormJob norms, unsigned* __restrict__ dep_ctr,
@@ -220,7 +234,8 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-    SharedTc& sh = *reinterpret_cast<SharedTc*>(smem + RING_BYTES);
+    constexpr int RING = Shape<SHORTK>::RING;
+    SharedTc<SHORTK>& sh = *reinterpret_cast<SharedTc<SHORTK>*>(smem + RING);
     volatile int* abort_flag = &sh.abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -239,22 +254,84 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (threadIdx.x == 64) {
+    if (warp == 2) {
+        // Work plan.  Everything per sequence -- its length, its tile counts -- is computed by
+        // the lanes in parallel and reduced with shuffles: the lengths live in global memory, and
+        // one thread walking dozens of sequences (heads) would hold the whole CTA back.
+        const int G = (int)gridDim.x;
+        int s256 = 0, s128 = 0, s64 = 0, rt0 = 0, rt1 = 0;
+        for (int b = lane; b < seg0.B; b += 32) {
+            const int n = seq_n(seg0, b);
+            if (n <= 0) continue;
+            if (seg0.tri) {
+                s256 += tri_tiles(n, BN);
+                s128 += tri_tiles(n, BM);
+                s64 += tri_tiles(n, BM / 2);
+            } else {
+                rt0 += (seg0.rows + BM - 1) / BM;
+            }
+        }
+        if (nseg > 1 && !seg1.tri)
+            for (int b = lane; b < seg1.B; b += 32)
+                if (seq_n(seg1, b) > 0) rt1 += (seg1.rows + BM - 1) / BM;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            s256 += __shfl_xor_sync(0xffffffffu, s256, o);
+            s128 += __shfl_xor_sync(0xffffffffu, s128, o);
+            s64 += __shfl_xor_sync(0xffffffffu, s64, o);
+            rt0 += __shfl_xor_sync(0xffffffffu, rt0, o);
+            rt1 += __shfl_xor_sync(0xffffffffu, rt1, o);
+        }
         // a triangular problem too small to give every CTA a 256-wide tile is cut 128 or 64 wide
-        int tw = BN;
-        int t0 = seg_tiles(seg0, tw);
         // (narrower tiles move fewer bytes per K block and finish sooner) as long as that
-        // still fits in one round of the grid
-        if (seg0.tri && 2 * t0 < (int)gridDim.x) { tw = BM; t0 = seg_tiles(seg0, tw); }
-        if (seg0.tri && 2 * t0 < (int)gridDim.x) { tw = BM / 2; t0 = seg_tiles(seg0, tw); }
-        if (!seg0.tri) { tw = cross_want(seg0, gridDim.x); t0 = seg_tiles(seg0, tw); }
-        sh.par0 = tw;
-        sh.tiles0 = t0;
-        sh.par1 = 1;
-        sh.tiles1 = 0;
-        if (nseg > 1) {
-            sh.par1 = seg1.tri ? BN : cross_want(seg1, gridDim.x);
-            sh.tiles1 = seg_tiles(seg1, sh.par1);
+        // still fits in one round of the grid; a cross problem gets as many column tiles per
+        // row tile as fill the grid once
+        int par0 = BN, t0 = s256;
+        if (seg0.tri && 2 * t0 < G) { par0 = BM; t0 = s128; }
+        if (seg0.tri && 2 * t0 < G) { par0 = BM / 2; t0 = s64; }
+        if (!seg0.tri) par0 = rt0 > 0 ? max(1, G / rt0) : 1;
+        const int par1 = (nseg > 1 && !seg1.tri) ? (rt1 > 0 ? max(1, G / rt1) : 1) : BN;
+        int c0 = 0, c1 = 0, w0 = 16, w1 = 16;
+        for (int b = lane; b < seg0.B; b += 32) {
+            const int n = seq_n(seg0, b);
+            if (n <= 0) continue;
+            if (seg0.tri) {
+                w0 = max(w0, min(par0, (n + 15) & ~15));
+            } else {
+                int nct, w;
+                cross_cols(n, par0, nct, w);
+                c0 += ((seg0.rows + BM - 1) / BM) * nct;
+                w0 = max(w0, w);
+            }
+        }
+        if (nseg > 1)
+            for (int b = lane; b < seg1.B; b += 32) {
+                const int n = seq_n(seg1, b);
+                if (n <= 0) continue;
+                if (seg1.tri) {
+                    c1 += tri_tiles(n, BN);
+                    w1 = max(w1, min(BN, (n + 15) & ~15));
+                } else {
+                    int nct, w;
+                    cross_cols(n, par1, nct, w);
+                    c1 += ((seg1.rows + BM - 1) / BM) * nct;
+                    w1 = max(w1, w);
+                }
+            }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            c0 += __shfl_xor_sync(0xffffffffu, c0, o);
+            c1 += __shfl_xor_sync(0xffffffffu, c1, o);
+            w0 = max(w0, __shfl_xor_sync(0xffffffffu, w0, o));
+            w1 = max(w1, __shfl_xor_sync(0xffffffffu, w1, o));
+        }
+        if (lane == 0) {
+            sh.par0 = par0;
+            sh.tiles0 = seg0.tri ? t0 : c0;
+            sh.wide0 = min(w0, BN);
+            sh.par1 = nseg > 1 ? par1 : 1;
+            sh.tiles1 = nseg > 1 ? c1 : 0;
+            sh.wide1 = min(w1, BN);
         }
     }
     if (warp == 1) {
@@ -268,6 +345,7 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
     tcgen05_fence_after();
     const unsigned tmem_base = sh.tmem_base;
     const int tiles0 = sh.tiles0, total = sh.tiles0 + sh.tiles1, par0 = sh.par0, par1 = sh.par1;
+    const int wide0 = sh.wide0, wide1 = sh.wide1;
     Piece pc;
     if (threadIdx.x < TAB) {
         const int id = blockIdx.x + (int)threadIdx.x * (int)gridDim.x;
@@ -304,30 +382,38 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
                                                id - (sg ? tiles0 : 0), pc, cur);
                 if (got_tile == 0) break;
                 if (got_tile == 2) continue;      // causal cross tile with no admissible pair
-                const int ksub = stage_ksub(pc.ncols, p.d);
+                // ring geometry is fixed per segment by its widest tile, so that a narrower
+                // (diagonal or last) tile needs no drain of the ring: it fills less of its stage
+                const int wide = SHORTK ? (sg ? wide1 : wide0) : pc.ncols;
+                const int ksub = stage_ksub(wide, p.d, RING);
                 const int num_kb = (p.d + BK * ksub - 1) / (BK * ksub);
                 const int nbox = (pc.ncols + BOX_N - 1) / BOX_N;
-                const int subb = sub_bytes(pc.ncols);
+                const int subb = sub_bytes(wide);
                 const int sb = ksub * subb;
+                const unsigned tx = (unsigned)(ksub * sub_bytes(pc.ncols));
                 if (sb != cur_sb) {
                     // new stage geometry: every stage of the old one must have been released
                     for (int q = 0; q < cur_nst && ok; ++q)
                         if ((used >> q) & 1u)
                             ok = mbar_wait(&sh.empty[q], ((fills >> q) & 1u) ^ 1u, abort_flag, 6);
                     if (!ok) break;
-                    cur_sb = sb; cur_nst = stage_count(sb); s = 0; used = 0;
+                    cur_sb = sb; cur_nst = stage_count(sb, RING); s = 0; used = 0;
                 }
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(&sh.empty[s], ((fills >> s) & 1u) ^ 1u, abort_flag, 1)) { ok = false; break; }
                     unsigned char* sa = smem + s * sb;
-                    mbar_expect_tx(&sh.full[s], (unsigned)sb);
+                    mbar_expect_tx(&sh.full[s], tx);
                     for (int u = 0; u < ksub; ++u) {          // K blocks past d are zero-filled
                         unsigned char* su = sa + u * subb;
                         const int k0 = (kb * ksub + u) * BK;
                         tma_load_3d(&maps.a[sg], &sh.full[s], su, k0, pc.row0, pc.b);
-                        for (int j = 0; j < nbox; ++j)
-                            tma_load_3d(&maps.b[sg], &sh.full[s], su + A_BYTES + j * BOX_BYTES, k0,
-                                        pc.col0 + j * BOX_N, pc.b);
+                        if (SHORTK && nbox == BN / BOX_N) {   // full-width tile: one 256-row box
+                            tma_load_3d(&maps.bw[sg], &sh.full[s], su + A_BYTES, k0, pc.col0, pc.b);
+                        } else {
+                            for (int j = 0; j < nbox; ++j)
+                                tma_load_3d(&maps.b[sg], &sh.full[s], su + A_BYTES + j * BOX_BYTES, k0,
+                                            pc.col0 + j * BOX_N, pc.b);
+                        }
                     }
                     fills ^= 1u << s; used |= 1u << s; ever |= 1u << s;
                     s = (s + 1 == cur_nst) ? 0 : s + 1;
@@ -360,11 +446,12 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
                                                id - (sg ? tiles0 : 0), pc, cur);
                 if (got_tile == 0) break;
                 if (got_tile == 2) continue;      // causal cross tile with no admissible pair
-                const int ksub = stage_ksub(pc.ncols, p.d);
+                const int wide = SHORTK ? (sg ? wide1 : wide0) : pc.ncols;
+                const int ksub = stage_ksub(wide, p.d, RING);
                 const int num_kb = (p.d + BK * ksub - 1) / (BK * ksub);
-                const int subb = sub_bytes(pc.ncols);
+                const int subb = sub_bytes(wide);
                 const int sb = ksub * subb;
-                if (sb != cur_sb) { cur_sb = sb; cur_nst = stage_count(sb); s = 0; }
+                if (sb != cur_sb) { cur_sb = sb; cur_nst = stage_count(sb, RING); s = 0; }
                 const unsigned acc = tile_it & 1u, acc_ph = (tile_it >> 1) & 1u;
                 ++tile_it;
                 if (!mbar_wait(&sh.tmem_empty[acc], acc_ph ^ 1u, abort_flag, 2)) { ok = false; break; }
@@ -397,9 +484,10 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
                 if (global_ns() - t0 > WAIT_LIMIT_NS / 2) { *abort_flag = 8; break; }
             }
         }
-    } else if (warp < 6) {
-        // ------------------------------------------------ epilogue (warps 2..5)
+    } else if (warp < 2 + Shape<SHORTK>::EPI_WARPS) {
+        // ------------------------------------------------ epilogue (warps 2..5, and 6..9 without norm warps)
         const int quad = warp & 3;                    // TMEM lane quadrant this warp may read
+        const unsigned eset = (unsigned)(warp - 2) >> 2;   // which of the two sets
         float* cs = sh.col_scale[warp - 2];
         int* ct = sh.col_token[warp - 2];
         const unsigned dep_total = 4u * (unsigned)tiles0;
@@ -419,7 +507,8 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
             if (got_tile == 0) break;
             if (got_tile == 2) continue;          // causal cross tile with no admissible pair
             const unsigned acc = tile_it & 1u, acc_ph = (tile_it >> 1) & 1u;
-                ++tile_it;
+            ++tile_it;
+            if (SHORTK && acc != eset) continue;      // the other set's tile
             const int64_t o = (int64_t)pc.b * p.cap;
             const int ncols = pc.ncols;
             const int ncols32 = (ncols + 31) & ~31;   // TMEM is read 32 columns at a time
@@ -554,7 +643,7 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
                 if (lane == 0) atomicAdd(dep_ctr, 1u);
             }
         }
-    } else if (norms.X != nullptr) {
+    } else if (!SHORTK && norms.X != nullptr) {
         // ------------------------------------------------ row norms (warps 6 and up)
         norm_rows(norms, blockIdx.x * NORM_WARPS + (warp - 6), gridDim.x * NORM_WARPS, lane,
                   dep_ctr + 1, status);
@@ -605,8 +694,11 @@ cudaError_t launch_selftest_wait(ada_ctx* ctx, int limit_ms, cudaStream_t s) {
 cudaError_t launch_gram_tc(ada_ctx* ctx, const GramProblem* tri, const GramProblem* cross,
                            const NormJob* norms, cudaStream_t s) {
     if (!ctx->tc_attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_gram_tc, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             SMEM_TC_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(k_gram_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             smem_tc_bytes<true>());
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(k_gram_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 smem_tc_bytes<false>());
         if (e != cudaSuccess) return e;
         ctx->tc_attr_set = true;
     }
@@ -624,12 +716,13 @@ cudaError_t launch_gram_tc(ada_ctx* ctx, const GramProblem* tri, const GramProbl
         if (n_cap <= 0 || a_rows <= 0) continue;
         // rows beyond the matrices (and k beyond d) are zero-filled by the TMA unit
         if (!make_map(&maps.a[nseg], p->A, p->d, p->tri ? p->cap : p->rows, p->B, p->lda, p->a_batch, BM) ||
-            !make_map(&maps.b[nseg], p->Bm, p->d, p->cap, p->B, p->ldb, p->b_batch, BOX_N))
+            !make_map(&maps.b[nseg], p->Bm, p->d, p->cap, p->B, p->ldb, p->b_batch, BOX_N) ||
+            !make_map(&maps.bw[nseg], p->Bm, p->d, p->cap, p->B, p->ldb, p->b_batch, BN))
             return cudaErrorInvalidValue;
         segs[nseg++] = *p;
     }
     if (nseg == 0) return cudaSuccess;
-    if (nseg == 1) { maps.a[1] = maps.a[0]; maps.b[1] = maps.b[0]; segs[1] = segs[0]; segs[1].B = 0; }
+    if (nseg == 1) { maps.a[1] = maps.a[0]; maps.b[1] = maps.b[0]; maps.bw[1] = maps.bw[0]; segs[1] = segs[0]; segs[1].B = 0; }
     NormJob nj;
     memset(&nj, 0, sizeof(nj));
     if (norms != nullptr) nj = *norms;
@@ -638,16 +731,20 @@ cudaError_t launch_gram_tc(ada_ctx* ctx, const GramProblem* tri, const GramProbl
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3(ctx->sm_count);
-    cfg.blockDim = dim3(NUM_THREADS);
-    cfg.dynamicSmemBytes = SMEM_TC_BYTES;
+    // short contraction and no norm warps needed: the epilogue-bound shape
+    const bool shortk = nj.X == nullptr && segs[0].d <= 512;
+    cfg.blockDim = dim3(shortk ? Shape<true>::THREADS : Shape<false>::THREADS);
+    cfg.dynamicSmemBytes = shortk ? smem_tc_bytes<true>() : smem_tc_bytes<false>();
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeCooperative;
     attr[0].val.cooperative = 1;
     cfg.attrs = attr;
     cfg.numAttrs = (fused && ctx->cooperative) ? 1 : 0;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, k_gram_tc, maps, segs[0], segs[1], nseg, nj, ctx->tile_ctr,
-                                       ctx->status);
+    cudaError_t e = shortk ? cudaLaunchKernelEx(&cfg, k_gram_tc<true>, maps, segs[0], segs[1], nseg, nj,
+                                                ctx->tile_ctr, ctx->status)
+                           : cudaLaunchKernelEx(&cfg, k_gram_tc<false>, maps, segs[0], segs[1], nseg, nj,
+                                                ctx->tile_ctr, ctx->status);
     prof_end(ctx, s);
     return e;
 }

@@ -147,9 +147,8 @@ static __device__ __forceinline__ void tmem_ld32(unsigned taddr, float (&v)[32])
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-// The same load split in two, so that the next 32 columns are on their way while the
-// previous ones are consumed.  After tmem_ld32_issue the registers are undefined; the wait
-// takes them as in/out operands, so every use in the code that follows depends on it.
+// The same load as two statements.  After tmem_ld32_issue the registers are undefined; the
+// wait takes them as in/out operands, so every use in the code that follows depends on it.
 static __device__ __forceinline__ void tmem_ld32_issue(unsigned taddr, unsigned (&r)[32]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "

@@ -156,6 +156,115 @@ k_norm_gather(const T* __restrict__ X, int64_t n_rows, int Tseq, int d, int64_t 
     }
 }
 
+constexpr int NORM_U = 4;   // rows per lane group of the short-row kernel
+
+// The same work for short rows (at most 16 vectors, e.g. one attention head), where a warp
+// per row would leave most lanes idle behind a single load.  Warps [0, n_norm_warps) take
+// rpw rows each, the warps after them rpw consecutive positions of one sequence's list.
+template <typename T>
+__global__ void __launch_bounds__(256)
+k_norm_gather_short(const T* __restrict__ X, int64_t n_rows, int Tseq, int d, int64_t ldx, int64_t xb,
+                    int rpw, int64_t n_norm_warps, float* __restrict__ inv_norm, T* __restrict__ Xhat,
+                    const int32_t* __restrict__ rep_in, const int32_t* __restrict__ rep_in_cnt,
+                    int32_t* __restrict__ role, int32_t* __restrict__ r_eff, T* __restrict__ Xrep,
+                    float* __restrict__ inv_rep, unsigned* __restrict__ status) {
+    const int lane = threadIdx.x & 31;
+    int64_t w = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (inv_norm == nullptr && Xhat == nullptr) w += n_norm_warps;   // gather-only launch: list warps only
+    constexpr int N = Vec16<T>::N;
+    const int nvec = d / N;  // d*es is a multiple of 16 bytes
+    if (w < n_norm_warps) {
+        // Short rows (at most 16 vectors, e.g. one attention head): a group of G lanes owns a
+        // row, the warp's 32/G groups take NORM_U rows each, and every lane has NORM_U loads in
+        // flight; a warp per row would leave most lanes idle behind one load.  Rows are taken
+        // in memory order: head-fastest when the heads of a token lie side by side.
+        const int R = rpw / NORM_U, G = 32 / R, sub = lane / G, gl = lane % G;
+        const int64_t nseq = n_rows / Tseq;
+        uint4 x[NORM_U];
+        int64_t orow[NORM_U];
+#pragma unroll
+        for (int u = 0; u < NORM_U; ++u) {
+            const int64_t r = w * rpw + u * R + sub;
+            x[u] = make_uint4(0u, 0u, 0u, 0u);
+            orow[u] = -1;
+            if (r < n_rows) {
+                const int64_t b = xb < ldx ? r % nseq : r / Tseq, t = xb < ldx ? r / nseq : r % Tseq;
+                orow[u] = b * Tseq + t;
+                if (gl < nvec) x[u] = __ldg(reinterpret_cast<const uint4*>(X + b * xb + t * ldx) + gl);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < NORM_U; ++u) {
+            float ss = Vec16<T>::sumsq(x[u]);
+            for (int o = G >> 1; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+            if (orow[u] < 0) continue;
+            float inv = 0.f;
+            if (!(ss <= 3.0e38f)) {
+                if (gl == 0) atomicOr(status, ST_NONFINITE);
+            } else if (ss > 0.f) {
+                inv = 1.0f / sqrtf(ss);
+            } else if (gl == 0) {
+                atomicAdd(status + 1, 1u);
+            }
+            if (inv_norm != nullptr && gl == 0) inv_norm[orow[u]] = inv;
+            if (Xhat != nullptr && gl < nvec)
+                reinterpret_cast<uint4*>(Xhat + orow[u] * (int64_t)d)[gl] = Vec16<T>::scale(x[u], inv);
+        }
+        return;
+    }
+    w -= n_norm_warps;
+    if (rep_in == nullptr) return;
+    {
+        // short rows: a lane group per list entry, NORM_U entries per group, as above; a warp
+        // covers rpw consecutive positions of one sequence's list
+        const int R = rpw / NORM_U, G = 32 / R, sub = lane / G, gl = lane % G;
+        const int64_t wps = (Tseq + rpw - 1) / rpw;          // warps per sequence
+        if (w >= wps * (n_rows / Tseq)) return;
+        const int b = (int)(w / wps);
+        const int i0 = (int)(w % wps) * rpw;
+        int cnt = rep_in_cnt[b];
+        if (cnt < 0 || cnt > Tseq) {
+            if (i0 == 0 && lane == 0) atomicOr(status, ST_BAD_COUNT);
+            cnt = cnt < 0 ? 0 : Tseq;
+        }
+        if (i0 == 0 && lane == 0 && r_eff != nullptr) r_eff[b] = cnt;
+        if (i0 >= cnt) return;
+        const int32_t* list = rep_in + (int64_t)b * Tseq;
+        int32_t idx[NORM_U], prev[NORM_U];
+#pragma unroll
+        for (int u = 0; u < NORM_U; ++u) {
+            const int i = i0 + u * R + sub;
+            idx[u] = i < cnt ? list[i] : -1;
+            prev[u] = (i < cnt && i > 0) ? list[i - 1] : -1;
+        }
+        uint4 x[NORM_U];
+        bool ok[NORM_U];
+#pragma unroll
+        for (int u = 0; u < NORM_U; ++u) {
+            const int i = i0 + u * R + sub;
+            ok[u] = i < cnt && idx[u] >= 0 && idx[u] < Tseq && prev[u] < idx[u];
+            if (i < cnt && !ok[u] && gl == 0) atomicOr(status, ST_BAD_INDEX);
+            x[u] = make_uint4(0u, 0u, 0u, 0u);
+            if (ok[u] && gl < nvec)
+                x[u] = __ldg(reinterpret_cast<const uint4*>(X + (int64_t)b * xb + (int64_t)idx[u] * ldx) + gl);
+        }
+#pragma unroll
+        for (int u = 0; u < NORM_U; ++u) {
+            const int i = i0 + u * R + sub;
+            float ss = Vec16<T>::sumsq(x[u]);
+            for (int o = G >> 1; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+            if (!ok[u]) continue;
+            const int64_t prow = (int64_t)b * Tseq + i;
+            if (gl < nvec) reinterpret_cast<uint4*>(Xrep + prow * (int64_t)d)[gl] = x[u];
+            if (gl == 0) {
+                inv_rep[prow] = (ss <= 3.0e38f && ss > 0.f) ? 1.0f / sqrtf(ss) : 0.f;
+                if (role != nullptr) role[(int64_t)b * Tseq + idx[u]] = i + 1;
+            }
+        }
+        return;
+    }
+}
+
 cudaError_t launch_norm_gather(ada_ctx* ctx, const void* X, int B, int T, int d, int64_t ldx,
                                int64_t xb, ada_dtype dt, float* inv_norm, void* Xhat, const int32_t* rep_in,
                                const int32_t* rep_in_cnt, int32_t* role, int32_t* r_eff, void* Xrep,
@@ -163,10 +272,30 @@ cudaError_t launch_norm_gather(ada_ctx* ctx, const void* X, int B, int T, int d,
     const int64_t n_rows = (int64_t)B * T;
     const int warps = 8;
     const bool gather_only = inv_norm == nullptr && Xhat == nullptr;
-    const int64_t n_warps = (rep_in != nullptr && !gather_only) ? 2 * n_rows : n_rows;
+    // rows per norm warp: lane groups of the next power of two at or above the row's vector count
+    const int nvec = d / (dt == ADA_F32 ? 4 : 8);
+    int G = 32;
+    if (nvec <= 16) for (G = 1; G < nvec; G <<= 1) {}
+    const int rpw = G == 32 ? 1 : (32 / G) * NORM_U;
+    const int64_t n_norm_warps = (n_rows + rpw - 1) / rpw;
+    // list warps: one per list position, or one per rpw positions of a sequence (short rows)
+    const int64_t n_list_warps = rpw == 1 ? n_rows : (int64_t)B * ((T + rpw - 1) / rpw);
+    const int64_t n_warps = gather_only ? n_list_warps
+                                        : (rep_in != nullptr ? n_norm_warps + n_list_warps : n_norm_warps);
     const unsigned grid = (unsigned)((n_warps + warps - 1) / warps);
     prof_begin(ctx, K_NORM_GATHER, s);
-    if (dt == ADA_F32) {
+    if (rpw > 1) {
+        if (dt == ADA_F32) {
+            k_norm_gather_short<float><<<grid, warps * 32, 0, s>>>(
+                (const float*)X, n_rows, T, d, ldx, xb, rpw, n_norm_warps, inv_norm, (float*)Xhat, rep_in,
+                rep_in_cnt, role, r_eff, (float*)Xrep, inv_rep, ctx->status);
+        } else {
+            k_norm_gather_short<__nv_bfloat16><<<grid, warps * 32, 0, s>>>(
+                (const __nv_bfloat16*)X, n_rows, T, d, ldx, xb, rpw, n_norm_warps, inv_norm,
+                (__nv_bfloat16*)Xhat, rep_in, rep_in_cnt, role, r_eff, (__nv_bfloat16*)Xrep, inv_rep,
+                ctx->status);
+        }
+    } else if (dt == ADA_F32) {
         k_norm_gather<float><<<grid, warps * 32, 0, s>>>(
             (const float*)X, n_rows, T, d, ldx, xb, inv_norm, (float*)Xhat, rep_in, rep_in_cnt, role,
             r_eff, (float*)Xrep, inv_rep, ctx->status);
