@@ -42,10 +42,12 @@ namespace {
 // alternate tiles (one accumulator each, so that one set's bookkeeping -- tile lookup, column
 // factors, barrier, atomics -- overlaps the other's TMEM reads), a ring geometry fixed per
 // segment (no drain between tiles of different width), one 256-row TMA box for a full-width
-// right operand, and a 208 KiB ring to make room for the second set's column factors.
+// right operand, a table of every sequence's length and first tile in shared memory (dozens of
+// heads are dozens of sequences), and a 200 KiB ring to make room for all that.
 template <bool SHORTK>
 struct Shape {
-    static constexpr int RING = SHORTK ? 208 * 1024 : RING_BYTES;
+    static constexpr int RING = SHORTK ? 200 * 1024 : RING_BYTES;
+    static constexpr int PLAN_B = SHORTK ? 64 : 0;   // sequences whose tile ranges are kept in shared memory
     static constexpr int EPI_WARPS = SHORTK ? 8 : 4;
     static constexpr int THREADS = SHORTK ? 64 + 32 * 8 : NUM_THREADS;
 };
@@ -109,12 +111,31 @@ struct TileCursor {
     int b, base;
 };
 // tile `id` of segment p -> piece; false when id is past the segment's last tile
+// s_n / s_first (shared memory, or NULL): length and first tile id of every sequence of the
+// segment, s_first[B] = number of tiles; without them the lengths are read from global memory
+// sequence by sequence.
 __device__ __forceinline__ bool decode_tile(const GramProblem& p, int par, int id, Piece& t,
-                                            TileCursor& cur) {
+                                            TileCursor& cur, const int* s_n = nullptr,
+                                            const int* s_first = nullptr) {
     const int tw = par;
+    if (s_first != nullptr) {
+        if (id >= s_first[p.B]) return false;
+        int lo = cur.b;
+        if (id >= s_first[lo + 1]) {                     // not the cursor's sequence: bisect above it
+            int hi = p.B - 1;
+            ++lo;
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if (id >= s_first[mid + 1]) lo = mid + 1;
+                else hi = mid;
+            }
+        }
+        cur.b = lo;
+        cur.base = s_first[lo];
+    }
     for (; cur.b < p.B; ++cur.b) {
         const int b = cur.b;
-        const int n = seq_n(p, b);
+        const int n = s_n != nullptr ? s_n[b] : seq_n(p, b);
         int cnt = 0, nct = 0, w = 0;
         if (n > 0) {
             if (p.tri) cnt = tri_tiles(n, tw);
@@ -191,6 +212,8 @@ struct alignas(16) SharedTc {
     int tiles0, tiles1, par0, par1;
     int wide0, wide1;           // widest tile of each segment (fixes the segment's ring geometry)
     uint4 tile_tab[TAB];
+    int seq_len[2][Shape<SHORTK>::PLAN_B + 1];     // per segment: sequence lengths ...
+    int seq_first[2][Shape<SHORTK>::PLAN_B + 1];   // ... and first tile ids (entry B: tile count)
     // per epilogue warp, so that staging needs no barrier across warps
     alignas(16) float col_scale[Shape<SHORTK>::EPI_WARPS][BN];
     alignas(16) int col_token[Shape<SHORTK>::EPI_WARPS][BN];
@@ -204,7 +227,8 @@ static_assert(smem_tc_bytes<false>() <= 227 * 1024 && smem_tc_bytes<true>() <= 2
 
 // 0: no such tile, 1: tile in pc, 2: tile in pc but nothing to do (dead_tile)
 __device__ __forceinline__ int next_tile(const uint4* tab, int it, const GramProblem& p, int par,
-                                         int local_id, Piece& pc, TileCursor& cur) {
+                                         int local_id, Piece& pc, TileCursor& cur,
+                                         const int* s_n, const int* s_first) {
     if (it < TAB) {
         const uint4 e = tab[it];
         if (e.z == 0u) return 0;
@@ -216,7 +240,7 @@ __device__ __forceinline__ int next_tile(const uint4* tab, int it, const GramPro
         pc.m = p.tri ? pc.n : p.rows;
         return (e.x >> 31) ? 2 : 1;
     }
-    if (!decode_tile(p, par, local_id, pc, cur)) return 0;
+    if (!decode_tile(p, par, local_id, pc, cur, s_n, s_first)) return 0;
     return dead_tile(p, pc) ? 2 : 1;
 }
 
@@ -291,43 +315,84 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
         if (seg0.tri && 2 * t0 < G) { par0 = BM / 2; t0 = s64; }
         if (!seg0.tri) par0 = rt0 > 0 ? max(1, G / rt0) : 1;
         const int par1 = (nseg > 1 && !seg1.tri) ? (rt1 > 0 ? max(1, G / rt1) : 1) : BN;
+        // second pass: tile count and widest tile of each segment; with few enough sequences
+        // also every sequence's length and first tile id, for the tile search
         int c0 = 0, c1 = 0, w0 = 16, w1 = 16;
-        for (int b = lane; b < seg0.B; b += 32) {
-            const int n = seq_n(seg0, b);
-            if (n <= 0) continue;
-            if (seg0.tri) {
-                w0 = max(w0, min(par0, (n + 15) & ~15));
-            } else {
-                int nct, w;
-                cross_cols(n, par0, nct, w);
-                c0 += ((seg0.rows + BM - 1) / BM) * nct;
-                w0 = max(w0, w);
-            }
-        }
-        if (nseg > 1)
-            for (int b = lane; b < seg1.B; b += 32) {
-                const int n = seq_n(seg1, b);
+        constexpr int PLAN_B = Shape<SHORTK>::PLAN_B;
+        if constexpr (!SHORTK) {
+            for (int b = lane; b < seg0.B; b += 32) {
+                const int n = seq_n(seg0, b);
                 if (n <= 0) continue;
-                if (seg1.tri) {
-                    c1 += tri_tiles(n, BN);
-                    w1 = max(w1, min(BN, (n + 15) & ~15));
+                if (seg0.tri) {
+                    c0 += tri_tiles(n, par0);
                 } else {
                     int nct, w;
-                    cross_cols(n, par1, nct, w);
-                    c1 += ((seg1.rows + BM - 1) / BM) * nct;
-                    w1 = max(w1, w);
+                    cross_cols(n, par0, nct, w);
+                    c0 += ((seg0.rows + BM - 1) / BM) * nct;
                 }
             }
+            if (nseg > 1)
+                for (int b = lane; b < seg1.B; b += 32) {
+                    const int n = seq_n(seg1, b);
+                    if (n <= 0) continue;
+                    if (seg1.tri) {
+                        c1 += tri_tiles(n, BN);
+                    } else {
+                        int nct, w;
+                        cross_cols(n, par1, nct, w);
+                        c1 += ((seg1.rows + BM - 1) / BM) * nct;
+                    }
+                }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            c0 += __shfl_xor_sync(0xffffffffu, c0, o);
-            c1 += __shfl_xor_sync(0xffffffffu, c1, o);
-            w0 = max(w0, __shfl_xor_sync(0xffffffffu, w0, o));
-            w1 = max(w1, __shfl_xor_sync(0xffffffffu, w1, o));
+            for (int o = 16; o > 0; o >>= 1) {
+                c0 += __shfl_xor_sync(0xffffffffu, c0, o);
+                c1 += __shfl_xor_sync(0xffffffffu, c1, o);
+            }
+        } else {
+            for (int sgi = 0; sgi < nseg; ++sgi) {
+                const GramProblem& p = sgi ? seg1 : seg0;
+                const int par = sgi ? par1 : par0;
+                const bool keep = p.B <= PLAN_B;
+                int run = 0, wide = 16;                      // tiles of the sequences before this round
+                for (int b0 = 0; b0 < p.B; b0 += 32) {
+                    const int b = b0 + lane;
+                    int n = 0, cnt = 0;
+                    if (b < p.B) {
+                        n = max(seq_n(p, b), 0);
+                        if (n > 0) {
+                            if (p.tri) {
+                                cnt = tri_tiles(n, par);
+                                wide = max(wide, min(par, (n + 15) & ~15));
+                            } else {
+                                int nct, w;
+                                cross_cols(n, par, nct, w);
+                                cnt = ((p.rows + BM - 1) / BM) * nct;
+                                wide = max(wide, w);
+                            }
+                        }
+                    }
+                    int incl = cnt;
+    #pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                        if (lane >= o) incl += v;
+                    }
+                    if (keep && b < p.B) {
+                        sh.seq_len[sgi][b] = n;
+                        sh.seq_first[sgi][b] = run + incl - cnt;
+                    }
+                    run += __shfl_sync(0xffffffffu, incl, 31);
+                }
+    #pragma unroll
+                for (int o = 16; o > 0; o >>= 1) wide = max(wide, __shfl_xor_sync(0xffffffffu, wide, o));
+                if (keep && lane == 0) sh.seq_first[sgi][p.B] = run;
+                if (sgi == 0) { c0 = run; w0 = wide; }
+                else { c1 = run; w1 = wide; }
+            }
         }
         if (lane == 0) {
             sh.par0 = par0;
-            sh.tiles0 = seg0.tri ? t0 : c0;
+            sh.tiles0 = c0;
             sh.wide0 = min(w0, BN);
             sh.par1 = nseg > 1 ? par1 : 1;
             sh.tiles1 = nseg > 1 ? c1 : 0;
@@ -347,6 +412,11 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
     const int tiles0 = sh.tiles0, total = sh.tiles0 + sh.tiles1, par0 = sh.par0, par1 = sh.par1;
     const int wide0 = sh.wide0, wide1 = sh.wide1;
     Piece pc;
+    // per-segment sequence tables (NULL: too many sequences, or the long-contraction shape)
+    const int* sn0 = seg0.B <= Shape<SHORTK>::PLAN_B ? sh.seq_len[0] : nullptr;
+    const int* sf0 = seg0.B <= Shape<SHORTK>::PLAN_B ? sh.seq_first[0] : nullptr;
+    const int* sn1 = seg1.B <= Shape<SHORTK>::PLAN_B ? sh.seq_len[1] : nullptr;
+    const int* sf1 = seg1.B <= Shape<SHORTK>::PLAN_B ? sh.seq_first[1] : nullptr;
     if (threadIdx.x < TAB) {
         const int id = blockIdx.x + (int)threadIdx.x * (int)gridDim.x;
         uint4 e = make_uint4(0u, 0u, 0u, 0u);
@@ -354,7 +424,7 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
             const int sg = id < tiles0 ? 0 : 1;
             const GramProblem& p = sg ? seg1 : seg0;
             TileCursor c0 = {0, 0};
-            if (decode_tile(p, sg ? par1 : par0, id - (sg ? tiles0 : 0), pc, c0))
+            if (decode_tile(p, sg ? par1 : par0, id - (sg ? tiles0 : 0), pc, c0, sg ? sn1 : sn0, sg ? sf1 : sf0))
                 e = make_uint4((unsigned)pc.row0 | ((unsigned)(pc.ncols >> 4) << 24) |
                                    (dead_tile(p, pc) ? 0x80000000u : 0u),
                                (unsigned)pc.col0, (unsigned)pc.n, (unsigned)pc.b);
@@ -379,7 +449,8 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
                 const GramProblem& p = sg ? seg1 : seg0;
                 if (sg != cur_sg) { cur.b = 0; cur.base = 0; cur_sg = sg; }
                 const int got_tile = next_tile(sh.tile_tab, it, p, sg ? par1 : par0,
-                                               id - (sg ? tiles0 : 0), pc, cur);
+                                               id - (sg ? tiles0 : 0), pc, cur, sg ? sn1 : sn0,
+                                               sg ? sf1 : sf0);
                 if (got_tile == 0) break;
                 if (got_tile == 2) continue;      // causal cross tile with no admissible pair
                 // ring geometry is fixed per segment by its widest tile, so that a narrower
@@ -443,7 +514,8 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
                 const GramProblem& p = sg ? seg1 : seg0;
                 if (sg != cur_sg) { cur.b = 0; cur.base = 0; cur_sg = sg; }
                 const int got_tile = next_tile(sh.tile_tab, it, p, sg ? par1 : par0,
-                                               id - (sg ? tiles0 : 0), pc, cur);
+                                               id - (sg ? tiles0 : 0), pc, cur, sg ? sn1 : sn0,
+                                               sg ? sf1 : sf0);
                 if (got_tile == 0) break;
                 if (got_tile == 2) continue;      // causal cross tile with no admissible pair
                 const int wide = SHORTK ? (sg ? wide1 : wide0) : pc.ncols;
@@ -503,7 +575,7 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
             const GramProblem& p = sg ? seg1 : seg0;
             if (sg != cur_sg) { cur.b = 0; cur.base = 0; cur_sg = sg; }
             const int got_tile = next_tile(sh.tile_tab, it, p, sg ? par1 : par0,
-                                           id - (sg ? tiles0 : 0), pc, cur);
+                                           id - (sg ? tiles0 : 0), pc, cur, sg ? sn1 : sn0, sg ? sf1 : sf0);
             if (got_tile == 0) break;
             if (got_tile == 2) continue;          // causal cross tile with no admissible pair
             const unsigned acc = tile_it & 1u, acc_ph = (tile_it >> 1) & 1u;

@@ -179,7 +179,8 @@ k_norm_gather_short(const T* __restrict__ X, int64_t n_rows, int Tseq, int d, in
         // flight; a warp per row would leave most lanes idle behind one load.  Rows are taken
         // in memory order: head-fastest when the heads of a token lie side by side.
         const int R = rpw / NORM_U, G = 32 / R, sub = lane / G, gl = lane % G;
-        const int64_t nseq = n_rows / Tseq;
+        // (row counts fit 31 bits; 32-bit division is several times cheaper than 64-bit)
+        const unsigned nseq = (unsigned)n_rows / (unsigned)Tseq;
         uint4 x[NORM_U];
         int64_t orow[NORM_U];
 #pragma unroll
@@ -188,7 +189,9 @@ k_norm_gather_short(const T* __restrict__ X, int64_t n_rows, int Tseq, int d, in
             x[u] = make_uint4(0u, 0u, 0u, 0u);
             orow[u] = -1;
             if (r < n_rows) {
-                const int64_t b = xb < ldx ? r % nseq : r / Tseq, t = xb < ldx ? r / nseq : r % Tseq;
+                const unsigned r32 = (unsigned)r;
+                const int64_t b = xb < ldx ? r32 % nseq : r32 / (unsigned)Tseq,
+                              t = xb < ldx ? r32 / nseq : r32 % (unsigned)Tseq;
                 orow[u] = b * Tseq + t;
                 if (gl < nvec) x[u] = __ldg(reinterpret_cast<const uint4*>(X + b * xb + t * ldx) + gl);
             }
@@ -218,10 +221,10 @@ k_norm_gather_short(const T* __restrict__ X, int64_t n_rows, int Tseq, int d, in
         // short rows: a lane group per list entry, NORM_U entries per group, as above; a warp
         // covers rpw consecutive positions of one sequence's list
         const int R = rpw / NORM_U, G = 32 / R, sub = lane / G, gl = lane % G;
-        const int64_t wps = (Tseq + rpw - 1) / rpw;          // warps per sequence
-        if (w >= wps * (n_rows / Tseq)) return;
-        const int b = (int)(w / wps);
-        const int i0 = (int)(w % wps) * rpw;
+        const unsigned wps = (unsigned)(Tseq + rpw - 1) / (unsigned)rpw;   // warps per sequence
+        if (w >= (int64_t)wps * ((unsigned)n_rows / (unsigned)Tseq)) return;
+        const int b = (int)((unsigned)w / wps);
+        const int i0 = (int)((unsigned)w % wps) * rpw;
         int cnt = rep_in_cnt[b];
         if (cnt < 0 || cnt > Tseq) {
             if (i0 == 0 && lane == 0) atomicOr(status, ST_BAD_COUNT);
