@@ -6,7 +6,7 @@
 // admissible columns j (Definition 1; Algorithm 1 lines 3-4 and 7-8).  Both operands
 // are row-major (K-major) bf16 matrices, so G = A B^T needs no transpose.
 //
-// One persistent CTA per SM, 14 warps:
+// One persistent CTA per SM.  Long-contraction shape, 14 warps:
 //   warp 0      TMA producer: one lane issues cp.async.bulk.tensor loads of a 128 x 64
 //               A box and up to four 64 x 64 B boxes per K block into a ring of 4 to 9
 //               stages (fewer bytes per stage for narrow tiles, hence more K blocks in
@@ -22,6 +22,8 @@
 //   warps 6..13 optional row norms (Section 2.1): 1/||x_t|| of every row of X with plain
 //               128-bit loads, overlapped with the main loops; the epilogues wait (bounded)
 //               for them before they scale, so a long-K call needs no separate norm pass
+// Short-contraction shape (d <= 512, no norm warps), 10 warps: warps 6..9 are a second
+// epilogue set; see Shape below.
 // Every wait is bounded: when a limit expires the CTA raises the context's TIMEOUT
 // status, drains its own outstanding copies and MMAs (again bounded), frees its TMEM
 // and returns.
