@@ -349,26 +349,50 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
                 norm_ok = true;
             }
             __syncwarp();
-            for (int c = lane; c < ncols; c += 32) {
-                const int col = pc.col0 + c;
-                float f = 0.f;
-                int tok = col;
-                if (col < pc.n) {
-                    f = __ldcg(p.inv_b + o + col);
-                    if (!p.tri) {
-                        if (!(__ldcg(p.col_gate + o + col) < p.thr_bits)) f = 0.f;
-                        if (p.causal) tok = p.col_token[o + col];
+            {
+                // all of the tile's global loads are issued before the first is used (columns
+                // past the tile are clamped to its last one and discarded afterwards, so that
+                // no load hangs on a data-dependent branch): eight dependent round trips to L2
+                // would otherwise sit on the path from a finished accumulator to its maxima
+                float fb[BN / 32];
+                unsigned gate[BN / 32] = {};
+                int tk[BN / 32] = {};
+                const int last = pc.n - 1;
+#pragma unroll
+                for (int q = 0; q < BN / 32; ++q)
+                    fb[q] = __ldcg(p.inv_b + o + min(pc.col0 + lane + 32 * q, last));
+                if (!p.tri) {
+                    // representative removed at line 5 (written earlier in this launch: read at L2)
+#pragma unroll
+                    for (int q = 0; q < BN / 32; ++q)
+                        gate[q] = __ldcg(p.col_gate + o + min(pc.col0 + lane + 32 * q, last));
+                }
+                if (!p.tri && p.causal) {
+#pragma unroll
+                    for (int q = 0; q < BN / 32; ++q)
+                        tk[q] = p.col_token[o + min(pc.col0 + lane + 32 * q, last)];
+                }
+#pragma unroll
+                for (int q = 0; q < BN / 32; ++q) {
+                    const int c = lane + 32 * q, col = pc.col0 + c;
+                    const bool live = col < pc.n;
+                    if (c < ncols) {
+                        cs[c] = (live && (p.tri || gate[q] < p.thr_bits)) ? fb[q] : 0.f;
+                        ct[c] = (live && !p.tri && p.causal) ? tk[q] : col;
                     }
                 }
-                cs[c] = f;
-                ct[c] = tok;
             }
             __syncwarp();
+            // this thread's row: its role and inverse norm are fetched while the MMAs finish
+            const int row_base = pc.row0 + (int)rank * BM;
+            const int row = row_base + quad * 32 + lane;
+            const bool row_live = row < pc.m;
+            const bool skip = row_live && !p.tri && p.row_role[o + row] != 0;   // inherited reps are not candidates
+            const bool inv_early = !(p.wait_norm_a && !norm_ok);
+            float inv_row = (row_live && inv_early) ? __ldcg(p.inv_a + o + row) : 0.f;
             const bool got = mbar_wait(&sh.tmem_full[acc], acc_ph, abort_flag, 4);
             if (!__all_sync(0xffffffffu, got)) break;
             tcgen05_fence_after();
-            const int row_base = pc.row0 + (int)rank * BM;
-            const int row = row_base + quad * 32 + lane;
             const bool need_cmp = p.tri ? (pc.col0 + ncols > row_base) : (p.causal != 0);
             float mx = 0.f;
             for (int c0 = 0; c0 < ncols; c0 += 32) {
@@ -398,10 +422,10 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
                 if (!wait_counter(dep_ctr + 1, norm_total, lane, abort_flag, 9)) break;
                 norm_ok = true;
             }
-            if (row < pc.m) {
-                const bool skip = !p.tri && p.row_role[o + row] != 0;   // inherited reps are not candidates
+            if (row_live) {
                 if (!skip) {
-                    mx *= __ldcg(p.inv_a + o + row);
+                    if (!inv_early) inv_row = __ldcg(p.inv_a + o + row);
+                    mx *= inv_row;
                     if (mx > 0.f) atomicMax(p.out + o + row, __float_as_uint(mx));
                 }
             }
