@@ -334,6 +334,8 @@ def main():
                     help="cascade steps with ADA_CROSS_CAUSAL (line 8 restricted to s < t)")
     ap.add_argument("--no-cooperative", action="store_true",
                     help="launch the fused cascade kernel as an ordinary grid (for profilers)")
+    ap.add_argument("--no-dep-launch", action="store_true",
+                    help="launch the kernels without programmatic stream serialization")
     ap.add_argument("--no-graph", action="store_true",
                     help="launch every call from Python instead of replaying a CUDA graph of one step")
     ap.add_argument("--heads", type=int, default=0,
@@ -393,6 +395,8 @@ def main():
     ada.ada_set_engine(ctx, args.engine)
     if args.no_cooperative:
         ada.ada_set_cooperative(ctx, False)
+    if args.no_dep_launch:
+        ada.ada_set_dependent_launch(ctx, False)
     stream = torch.cuda.current_stream()
     cflags = ada.ADA_CROSS_CAUSAL if args.causal else 0
 

@@ -100,6 +100,15 @@ ada_status ada_set_engine(ada_ctx* ctx, ada_engine e);
  * launches.  Default: on. */
 ada_status ada_set_cooperative(ada_ctx* ctx, int on);
 
+/* Programmatic dependent launch of the library's kernels (on by default).  When on, every
+ * kernel is launched with the stream-serialization attribute and begins with a grid-dependency
+ * wait, so that its blocks can be placed, and its set-up that reads nothing (barriers, TMEM
+ * allocation) can run, while the previous kernel of the stream drains; results do not change.
+ * It concerns only the order between consecutive kernels of one stream; work from other
+ * sources enqueued between two calls is ordered as usual.  Turn it off for tools that cannot
+ * follow such launches.  Host-only: ADA_ERR_INVALID_ARG for a NULL context. */
+ada_status ada_set_dependent_launch(ada_ctx* ctx, int on);
+
 /*
  * Row normalisation and representative gather (Section 2.1; Algorithm 1
  * lines 1-2).  Each output may be NULL:

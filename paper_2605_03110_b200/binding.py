@@ -26,7 +26,7 @@ SYMBOLS = [
     "ada_cascade_step", "ada_select_full_host", "ada_cascade_step_host", "ada_gram_op_count",
     "ada_device_status", "ada_profile_enable", "ada_profile_read", "ada_status_string",
     "ada_select_full_noalloc", "ada_set_cooperative", "ada_selftest_wait_timeout", "ada_nearest_rep",
-    "ada_select_full_heads", "ada_cascade_step_heads",
+    "ada_select_full_heads", "ada_cascade_step_heads", "ada_set_dependent_launch",
 ]
 ADA_NOALLOC_MAX_T = 16384
 
@@ -52,6 +52,7 @@ def lib() -> C.CDLL:
         L.ada_destroy.argtypes = [vp]
         L.ada_set_engine.argtypes = [vp, C.c_int]
         L.ada_set_cooperative.argtypes = [vp, C.c_int]
+        L.ada_set_dependent_launch.argtypes = [vp, C.c_int]
         L.ada_selftest_wait_timeout.argtypes = [vp, C.c_int, vp]
         L.ada_normalize.argtypes = [vp, vp, i64, i64, i64, i64, C.c_int, vp, fp, i32p, i32p, vp, vp]
         L.ada_select_full.argtypes = [vp, vp, i64, i64, i64, i64, C.c_int, C.c_double, i32p, i32p,
@@ -154,6 +155,10 @@ def ada_set_engine(ctx: Context, engine: int) -> None:
 
 def ada_set_cooperative(ctx: Context, on: bool) -> None:
     _check(lib().ada_set_cooperative(ctx.h, int(bool(on))), "ada_set_cooperative")
+
+
+def ada_set_dependent_launch(ctx: Context, on: bool) -> None:
+    _check(lib().ada_set_dependent_launch(ctx.h, int(bool(on))), "ada_set_dependent_launch")
 
 
 def ada_selftest_wait_timeout(ctx: Context, limit_ms: int = 50, stream=None) -> None:

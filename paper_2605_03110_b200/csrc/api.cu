@@ -154,6 +154,7 @@ ada_status ada_create(ada_ctx** out, int device, int64_t maxB, int64_t maxT, int
     ctx->stage = nullptr; ctx->stage_bytes = 0; ctx->host_stream = nullptr;
     ctx->tc_attr_set = false;
     ctx->cooperative = true;
+    ctx->dep_launch = true;
     ctx->tc2_attr_set = false;
     ctx->tc2_pairs = 0;
     cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
@@ -233,6 +234,12 @@ ada_status ada_set_engine(ada_ctx* ctx, ada_engine e) {
 ada_status ada_set_cooperative(ada_ctx* ctx, int on) {
     if (ctx == nullptr) return ADA_ERR_INVALID_ARG;
     ctx->cooperative = on != 0;
+    return ADA_OK;
+}
+
+ada_status ada_set_dependent_launch(ada_ctx* ctx, int on) {
+    if (ctx == nullptr) return ADA_ERR_INVALID_ARG;
+    ctx->dep_launch = on != 0;
     return ADA_OK;
 }
 

@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <string.h>
 
 #include "../../include/ada.h"
 
@@ -101,6 +102,7 @@ struct ada_ctx {
     int sm_count;
     bool tc_attr_set;
     bool cooperative;    // fused launches use the cooperative attribute
+    bool dep_launch;     // kernels are launched with programmatic stream serialization
     bool tc2_attr_set;   // pair-CTA kernel configured
     int tc2_pairs;       // clusters of two that fit on the device at once
     // device workspace
@@ -129,6 +131,35 @@ struct ada_ctx {
 };
 
 namespace ada {
+
+// Programmatic dependent launch.  Every kernel of the library starts with grid_dep_wait()
+// -- before any early return, so that a grid never completes ahead of its predecessor -- and is
+// launched with the stream-serialization attribute: its blocks may be placed on an SM, and run
+// what precedes the wait (barrier set-up, TMEM allocation), as soon as the blocks of the kernel
+// before it in the stream have left, instead of after that whole grid has drained; the wait
+// returns once the predecessor has completed and its writes are visible.  Without the
+// attribute the wait is a no-op.
+#ifdef __CUDACC__
+static __device__ __forceinline__ void grid_dep_wait() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+#endif
+template <typename... KArgs, typename... Args>
+cudaError_t launch_k(ada_ctx* ctx, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                     cudaStream_t s, Args&&... args) {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = ctx->dep_launch ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 // RAII-free launch bracket used by every launcher.
 void prof_begin(ada_ctx* ctx, int kid, cudaStream_t s);

@@ -32,6 +32,7 @@ __device__ __forceinline__ void load4<__nv_bfloat16>(const __nv_bfloat16* p, flo
 template <typename T>
 __global__ void __launch_bounds__(256)
 k_gram_ffma(const GramProblem p) {
+    grid_dep_wait();
     const int b = blockIdx.z;
     const int n = p.n_dev != nullptr ? p.n_dev[b] : p.n_host;   // columns (and rows when tri)
     const int m = p.tri ? n : p.rows;
@@ -146,8 +147,8 @@ cudaError_t launch_gram_ffma(ada_ctx* ctx, const GramProblem& p, ada_dtype dt, c
     if (n_cap <= 0 || m_cap <= 0) return cudaSuccess;
     dim3 grid((n_cap + BN - 1) / BN, (m_cap + BM - 1) / BM, p.B);
     prof_begin(ctx, p.tri ? K_GRAM_FFMA_TRI : K_GRAM_FFMA_CROSS, s);
-    if (dt == ADA_F32) k_gram_ffma<float><<<grid, 256, 0, s>>>(p);
-    else k_gram_ffma<__nv_bfloat16><<<grid, 256, 0, s>>>(p);
+    if (dt == ADA_F32) launch_k(ctx, k_gram_ffma<float>, grid, dim3(256), 0, s, p);
+    else launch_k(ctx, k_gram_ffma<__nv_bfloat16>, grid, dim3(256), 0, s, p);
     prof_end(ctx, s);
     return cudaGetLastError();
 }

@@ -280,6 +280,14 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&sh.tmem_base)), "r"(TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    // everything above is local to the CTA; from here on the predecessor's results are read
+    grid_dep_wait();
     if (warp == 2) {
         // Work plan.  Everything per sequence -- its length, its tile counts -- is computed by
         // the lanes in parallel and reduced with shuffles: the lengths live in global memory, and
@@ -400,12 +408,6 @@ k_gram_tc(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPro
             sh.tiles1 = nseg > 1 ? c1 : 0;
             sh.wide1 = min(w1, BN);
         }
-    }
-    if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(&sh.tmem_base)), "r"(TMEM_COLS)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tcgen05_fence_before();
     __syncthreads();
@@ -745,6 +747,7 @@ namespace {
 // One warp waits on a counter that stays at zero; the limit expires and the status is raised.
 __global__ void k_selftest_wait(const unsigned* counter, unsigned long long limit_ns,
                                 unsigned* status) {
+    grid_dep_wait();
     __shared__ int abort_flag;
     if (threadIdx.x == 0) abort_flag = 0;
     __syncwarp();
@@ -758,8 +761,8 @@ __global__ void k_selftest_wait(const unsigned* counter, unsigned long long limi
 
 cudaError_t launch_selftest_wait(ada_ctx* ctx, int limit_ms, cudaStream_t s) {
     // tile_ctr[2] is never written by any kernel
-    k_selftest_wait<<<1, 32, 0, s>>>(ctx->tile_ctr + 2, (unsigned long long)limit_ms * 1000000ull,
-                                     ctx->status);
+    launch_k(ctx, k_selftest_wait, dim3(1), dim3(32), 0, s, ctx->tile_ctr + 2,
+             (unsigned long long)limit_ms * 1000000ull, ctx->status);
     return cudaGetLastError();
 }
 
@@ -810,11 +813,20 @@ cudaError_t launch_gram_tc(ada_ctx* ctx, const GramProblem* tri, const GramProbl
     cfg.blockDim = dim3(shortk ? Shape<true>::THREADS : Shape<false>::THREADS);
     cfg.dynamicSmemBytes = shortk ? smem_tc_bytes<true>() : smem_tc_bytes<false>();
     cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeCooperative;
-    attr[0].val.cooperative = 1;
+    cudaLaunchAttribute attr[2];
+    int na = 0;
+    if (fused && ctx->cooperative) {
+        attr[na].id = cudaLaunchAttributeCooperative;
+        attr[na].val.cooperative = 1;
+        ++na;
+    }
+    if (ctx->dep_launch) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = (fused && ctx->cooperative) ? 1 : 0;
+    cfg.numAttrs = na;
     cudaError_t e = shortk ? cudaLaunchKernelEx(&cfg, k_gram_tc<true>, maps, segs[0], segs[1], nseg, nj,
                                                 ctx->tile_ctr, ctx->status)
                            : cudaLaunchKernelEx(&cfg, k_gram_tc<false>, maps, segs[0], segs[1], nseg, nj,

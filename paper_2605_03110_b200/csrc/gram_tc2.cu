@@ -202,15 +202,17 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (threadIdx.x == 64) {
-        sh.tiles0 = seg_tiles(seg0);
-        sh.tiles1 = nseg > 1 ? seg_tiles(seg1) : 0;
-    }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(&sh.tmem_base)), "r"(TMEM_COLS)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    // everything above is local to the CTA; from here on the predecessor's results are read
+    grid_dep_wait();
+    if (threadIdx.x == 64) {
+        sh.tiles0 = seg_tiles(seg0);
+        sh.tiles1 = nseg > 1 ? seg_tiles(seg1) : 0;
     }
     tcgen05_fence_before();
     __syncthreads();
@@ -512,13 +514,23 @@ cudaError_t launch_gram_tc2(ada_ctx* ctx, const GramProblem* tri, const GramProb
     cfg.blockDim = dim3(NUM_THREADS);
     cfg.dynamicSmemBytes = SMEM_BYTES;
     cfg.stream = s;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    attr[1].id = cudaLaunchAttributeCooperative;
-    attr[1].val.cooperative = 1;
+    cudaLaunchAttribute attr[3];
+    int na = 0;
+    attr[na].id = cudaLaunchAttributeClusterDimension;
+    attr[na].val.clusterDim.x = 2; attr[na].val.clusterDim.y = 1; attr[na].val.clusterDim.z = 1;
+    ++na;
+    if (fused && ctx->cooperative) {
+        attr[na].id = cudaLaunchAttributeCooperative;
+        attr[na].val.cooperative = 1;
+        ++na;
+    }
+    if (ctx->dep_launch) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = (fused && ctx->cooperative) ? 2 : 1;
+    cfg.numAttrs = na;
     cudaError_t e = cudaLaunchKernelEx(&cfg, k_gram_tc2, maps, segs[0], segs[1], nseg, nj, ctx->tile_ctr,
                                        ctx->status);
     prof_end(ctx, s);

@@ -84,6 +84,7 @@ k_norm_gather(const T* __restrict__ X, int64_t n_rows, int Tseq, int d, int64_t 
               const int32_t* __restrict__ rep_in, const int32_t* __restrict__ rep_in_cnt,
               int32_t* __restrict__ role, int32_t* __restrict__ r_eff, T* __restrict__ Xrep,
               float* __restrict__ inv_rep, unsigned* __restrict__ status) {
+    grid_dep_wait();
     const int lane = threadIdx.x & 31;
     int64_t w = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (inv_norm == nullptr && Xhat == nullptr) w += n_rows;   // gather-only launch: list warps only
@@ -168,6 +169,7 @@ k_norm_gather_short(const T* __restrict__ X, int64_t n_rows, int Tseq, int d, in
                     const int32_t* __restrict__ rep_in, const int32_t* __restrict__ rep_in_cnt,
                     int32_t* __restrict__ role, int32_t* __restrict__ r_eff, T* __restrict__ Xrep,
                     float* __restrict__ inv_rep, unsigned* __restrict__ status) {
+    grid_dep_wait();
     const int lane = threadIdx.x & 31;
     int64_t w = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (inv_norm == nullptr && Xhat == nullptr) w += n_norm_warps;   // gather-only launch: list warps only
@@ -289,21 +291,21 @@ cudaError_t launch_norm_gather(ada_ctx* ctx, const void* X, int B, int T, int d,
     prof_begin(ctx, K_NORM_GATHER, s);
     if (rpw > 1) {
         if (dt == ADA_F32) {
-            k_norm_gather_short<float><<<grid, warps * 32, 0, s>>>(
+            launch_k(ctx, k_norm_gather_short<float>, dim3(grid), dim3(warps * 32), 0, s,
                 (const float*)X, n_rows, T, d, ldx, xb, rpw, n_norm_warps, inv_norm, (float*)Xhat, rep_in,
                 rep_in_cnt, role, r_eff, (float*)Xrep, inv_rep, ctx->status);
         } else {
-            k_norm_gather_short<__nv_bfloat16><<<grid, warps * 32, 0, s>>>(
+            launch_k(ctx, k_norm_gather_short<__nv_bfloat16>, dim3(grid), dim3(warps * 32), 0, s,
                 (const __nv_bfloat16*)X, n_rows, T, d, ldx, xb, rpw, n_norm_warps, inv_norm,
                 (__nv_bfloat16*)Xhat, rep_in, rep_in_cnt, role, r_eff, (__nv_bfloat16*)Xrep, inv_rep,
                 ctx->status);
         }
     } else if (dt == ADA_F32) {
-        k_norm_gather<float><<<grid, warps * 32, 0, s>>>(
+        launch_k(ctx, k_norm_gather<float>, dim3(grid), dim3(warps * 32), 0, s,
             (const float*)X, n_rows, T, d, ldx, xb, inv_norm, (float*)Xhat, rep_in, rep_in_cnt, role,
             r_eff, (float*)Xrep, inv_rep, ctx->status);
     } else {
-        k_norm_gather<__nv_bfloat16><<<grid, warps * 32, 0, s>>>(
+        launch_k(ctx, k_norm_gather<__nv_bfloat16>, dim3(grid), dim3(warps * 32), 0, s,
             (const __nv_bfloat16*)X, n_rows, T, d, ldx, xb, inv_norm, (__nv_bfloat16*)Xhat, rep_in,
             rep_in_cnt, role, r_eff, (__nv_bfloat16*)Xrep, inv_rep, ctx->status);
     }
@@ -344,6 +346,7 @@ __device__ __forceinline__ void split3(float x, __nv_bfloat16& hi, __nv_bfloat16
 
 __global__ void __launch_bounds__(256)
 k_split_bf16(const SplitJob j0, const SplitJob j1, int64_t n_rows, int d, unsigned* __restrict__ status) {
+    grid_dep_wait();
     const int lane = threadIdx.x & 31;
     int64_t w = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const bool second = w >= n_rows;
@@ -416,7 +419,7 @@ cudaError_t launch_split(ada_ctx* ctx, const void* X, int B, int T, int d, int64
     const int warps = 8;
     const int64_t n_warps = with_rep ? 2 * n_rows : n_rows;
     prof_begin(ctx, K_SPLIT, s);
-    k_split_bf16<<<(unsigned)((n_warps + warps - 1) / warps), warps * 32, 0, s>>>(j0, j1, n_rows, d,
+    launch_k(ctx, k_split_bf16, dim3((unsigned)((n_warps + warps - 1) / warps)), dim3(warps * 32), 0, s, j0, j1, n_rows, d,
                                                                                   ctx->status);
     prof_end(ctx, s);
     return cudaGetLastError();
@@ -482,6 +485,7 @@ __device__ __forceinline__ unsigned long long block_exclusive_scan(unsigned long
 
 __global__ void __launch_bounds__(1024) k_compact(const CompactArgs a) {
     __shared__ unsigned long long s_warp[33];
+    grid_dep_wait();
     const int b = blockIdx.y, blk = blockIdx.x, nblk = gridDim.x;
     const int t = blk * 1024 + threadIdx.x;
     const int64_t o = (int64_t)b * a.T;
@@ -580,6 +584,7 @@ k_nearest_finish(unsigned long long* __restrict__ near_key, int32_t* __restrict_
                  const int32_t* __restrict__ r_eff, const float* __restrict__ inv_norm,
                  const int32_t* __restrict__ rep_idx, int T, int32_t* __restrict__ nearest_idx,
                  float* __restrict__ nearest_gamma) {
+    grid_dep_wait();
     const int b = blockIdx.y, t = blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= T) return;
     const int64_t o = (int64_t)b * T;
@@ -610,7 +615,7 @@ k_nearest_finish(unsigned long long* __restrict__ near_key, int32_t* __restrict_
 cudaError_t launch_nearest_finish(ada_ctx* ctx, int B, int T, const int32_t* rep_idx,
                                   int32_t* nearest_idx, float* nearest_gamma, cudaStream_t s) {
     prof_begin(ctx, K_NEAREST_FINISH, s);
-    k_nearest_finish<<<dim3((T + 255) / 256, B), 256, 0, s>>>(ctx->near_key, ctx->role, ctx->r_eff,
+    launch_k(ctx, k_nearest_finish, dim3((T + 255) / 256, B), dim3(256), 0, s, ctx->near_key, ctx->role, ctx->r_eff,
                                                                ctx->inv_norm, rep_idx, T, nearest_idx,
                                                                nearest_gamma);
     prof_end(ctx, s);
@@ -621,7 +626,7 @@ static cudaError_t launch_compact(ada_ctx* ctx, int kid, const CompactArgs& a, i
     const int nblk = (a.T + 1023) / 1024;
     if (nblk > a.agg_stride) return cudaErrorInvalidValue;
     prof_begin(ctx, kid, s);
-    k_compact<<<dim3(nblk, B), 1024, 0, s>>>(a);
+    launch_k(ctx, k_compact, dim3(nblk, B), dim3(1024), 0, s, a);
     prof_end(ctx, s);
     return cudaGetLastError();
 }

@@ -466,3 +466,32 @@ def test_repeated_runs_are_bit_identical(ada):
     b = ada.ada_select_full(ctx, Xd, cfg.tau)
     assert torch.equal(a[2], b[2]) and torch.equal(a[1], b[1])
     ada.ada_destroy(ctx)
+
+
+@pytest.mark.parametrize("cfg_id", [1, 2])
+def test_dependent_launch_on_and_off_give_identical_results(ada, cfg_id):
+    """The launch attribute changes when a kernel's blocks may be placed, never what it computes:
+    a chain of calls with programmatic dependent launch on (default) and off, bit for bit."""
+    from parity import to_device
+    cfg = wl.scaled(wl.CONFIGS[cfg_id], L=4)
+    layers = [to_device(lb.X) for lb in wl.generate_layers(cfg, seed=1)]
+    res = []
+    for on in (True, False):
+        ctx = ada.ada_create(cfg.B, cfg.T, cfg.d, ada.ADA_F32 if cfg.dtype == "f32" else ada.ADA_BF16)
+        ada.ada_set_dependent_launch(ctx, on)
+        idx, cnt, g = ada.ada_select_full(ctx, layers[0], cfg.tau)
+        out = [cnt.clone(), g.clone()] + [idx[b, :int(cnt[b])].clone() for b in range(cfg.B)]
+        for X in layers[1:]:
+            o = ada.ada_cascade_step(ctx, X, cfg.tau, idx, cnt)
+            idx, cnt = o.rep_out, o.rep_out_cnt
+            out += [o.rep_out_cnt.clone(), o.add_cnt.clone(), o.rem_cnt.clone(), o.gamma_rep.clone(),
+                    o.gamma_cross.clone()]
+            for b in range(cfg.B):
+                out.append(o.rep_out[b, :int(o.rep_out_cnt[b])].clone())
+        st, _ = ada.ada_device_status(ctx)
+        assert st == 0
+        res.append(out)
+        ada.ada_destroy(ctx)
+    assert len(res[0]) == len(res[1])
+    for a, b in zip(*res):
+        assert torch.equal(a, b)
