@@ -143,6 +143,12 @@ namespace ada {
 static __device__ __forceinline__ void grid_dep_wait() {
     asm volatile("griddepcontrol.wait;" ::: "memory");
 }
+// Lets the next kernel's blocks be placed now instead of when this block exits (they still wait,
+// in their own grid_dep_wait, for this whole grid to complete).  Worth it in kernels that leave
+// most SMs idle or whose blocks are short.
+static __device__ __forceinline__ void grid_dep_launch_next() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
 #endif
 template <typename... KArgs, typename... Args>
 cudaError_t launch_k(ada_ctx* ctx, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,

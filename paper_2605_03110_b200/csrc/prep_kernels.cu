@@ -486,6 +486,7 @@ __device__ __forceinline__ unsigned long long block_exclusive_scan(unsigned long
 __global__ void __launch_bounds__(1024) k_compact(const CompactArgs a) {
     __shared__ unsigned long long s_warp[33];
     grid_dep_wait();
+    grid_dep_launch_next();
     const int b = blockIdx.y, blk = blockIdx.x, nblk = gridDim.x;
     const int t = blk * 1024 + threadIdx.x;
     const int64_t o = (int64_t)b * a.T;
