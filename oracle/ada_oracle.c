@@ -265,6 +265,26 @@ double ada_oracle_jaccard(const int32_t* a, int64_t na, const int32_t* b, int64_
     return uni == 0 ? 1.0 : (double)inter / (double)uni;
 }
 
+/* Section 8.1 (adaptive threshold across depth): the paper proposes to set tau^(l+1) from the
+ * turnover of layer l -- a stable set (low turnover) tolerates a tighter threshold (larger tau:
+ * fewer representatives), an evolving one needs a looser threshold -- and gives no formula.
+ * Reading taken: a clipped proportional step toward a target turnover,
+ *     tau' = min(tau_max, max(tau_min, tau + gain * (target - rho))),
+ * with tau' = clip(tau) when rho is undefined (empty inherited set).  Each operation is one
+ * rounded fp64 operation, in this order. */
+double ada_oracle_tau_update(double tau, double rho, double target, double gain, double tau_min,
+                             double tau_max) {
+    double t = tau;
+    if (rho == rho) {
+        const double diff = target - rho;
+        const double step = gain * diff;
+        t = tau + step;
+    }
+    if (t < tau_min) t = tau_min;
+    if (t > tau_max) t = tau_max;
+    return t;
+}
+
 /* Eq. (6): (|additions| + |removals|) / |R^(l)|; NaN when the set is empty. */
 double ada_oracle_turnover(int64_t n_add, int64_t n_rem, int64_t r) {
     if (r == 0) return NAN;

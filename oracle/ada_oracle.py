@@ -21,7 +21,8 @@ _lib = None
 def build(force: bool = False) -> str:
     """Compile the oracle with gcc (plain -O2, OpenMP over rows)."""
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
-        cmd = ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", _LIB, _SRC, "-lm"]
+        cmd = ["gcc", "-O2", "-ffp-contract=off", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", _LIB,
+               _SRC, "-lm"]
         subprocess.run(cmd, check=True)
     return _LIB
 
@@ -52,6 +53,8 @@ def _load():
         lib.ada_oracle_jaccard.restype = C.c_double
         lib.ada_oracle_turnover.argtypes = [i64, i64, i64]
         lib.ada_oracle_turnover.restype = C.c_double
+        lib.ada_oracle_tau_update.argtypes = [C.c_double] * 6
+        lib.ada_oracle_tau_update.restype = C.c_double
         _lib = lib
     return _lib
 
@@ -173,6 +176,13 @@ def jaccard(a, b) -> float:
     a = np.ascontiguousarray(a, dtype=np.int32)
     b = np.ascontiguousarray(b, dtype=np.int32)
     return float(_load().ada_oracle_jaccard(_ip(a), a.size, _ip(b), b.size))
+
+
+def tau_update(tau: float, rho: float, target: float, gain: float, tau_min: float,
+               tau_max: float) -> float:
+    """Section 8.1, reading: clipped proportional step of tau toward a target turnover."""
+    return float(_load().ada_oracle_tau_update(float(tau), float(rho), float(target), float(gain),
+                                               float(tau_min), float(tau_max)))
 
 
 def turnover(n_add: int, n_rem: int, r: int) -> float:

@@ -413,3 +413,33 @@ def test_nearest_ties_go_to_the_lowest_index_and_labels_agree():
     nonrep = np.setdiff1d(np.arange(lab.size), st["R"])
     # a redundant token's nearest representative carries its prototype label
     assert np.all(lab[near[nonrep]] == lab[nonrep]) and np.all(g[nonrep] > 0.9)
+
+
+def test_tau_update_rule_by_hand_and_by_fractions():
+    """Section 8.1, reading: tau' = clip(tau + gain * (target - rho)).  Pinned by values worked
+    by hand in binary-exact numbers, by exact rational arithmetic, and by its properties: a
+    stable set (turnover below target) tightens the threshold (tau grows), an evolving one
+    loosens it, gain 0 or an undefined turnover leave tau alone, the bounds hold."""
+    from fractions import Fraction
+    f = oracle.tau_update
+    # binary-exact operands: every intermediate is exact, so the result is too
+    assert f(0.25, 0.125, 0.25, 0.5, 0.0625, 0.75) == 0.3125        # 0.25 + 0.5 * 0.125
+    assert f(0.25, 0.5, 0.25, 0.5, 0.0625, 0.75) == 0.125           # 0.25 - 0.5 * 0.25
+    assert f(0.25, 4.0, 0.25, 0.5, 0.0625, 0.75) == 0.0625          # clipped below
+    assert f(0.5, 0.0, 1.0, 1.0, 0.0625, 0.75) == 0.75              # clipped above
+    assert f(0.3, 0.05, 0.1, 0.0, 0.1, 0.6) == 0.3                  # gain 0
+    assert f(0.3, float("nan"), 0.1, 0.5, 0.1, 0.6) == 0.3          # empty inherited set
+    assert f(0.05, float("nan"), 0.1, 0.5, 0.1, 0.6) == 0.1         # ... still clipped
+    rng = np.random.default_rng(3)
+    for _ in range(200):
+        tau, rho, target, gain = rng.uniform(0.05, 0.9), rng.uniform(0, 1.5), rng.uniform(0, 0.5), \
+            rng.uniform(0, 2)
+        got = f(tau, rho, target, gain, 0.05, 0.9)
+        exact = Fraction(tau) + Fraction(gain) * (Fraction(target) - Fraction(rho))
+        exact = min(Fraction(0.9), max(Fraction(0.05), exact))
+        assert abs(Fraction(got) - exact) <= Fraction(1, 2 ** 50)    # three roundings of fp64
+        assert 0.05 <= got <= 0.9
+        if 0.05 < got < 0.9:
+            assert (got > tau) == (rho < target) or got == tau
+    # the turnover it is fed is Eq. 6
+    assert oracle.turnover(3, 1, 8) == 0.5 and np.isnan(oracle.turnover(2, 0, 0))
