@@ -59,7 +59,8 @@ typedef enum {
     ADA_ERR_CUDA = 4,          /* a CUDA runtime / driver call failed                       */
     ADA_ERR_BAD_INDEX_SET = 5, /* device: inherited list not ascending / out of range       */
     ADA_ERR_NONFINITE = 6,     /* device: NaN or Inf in X                                   */
-    ADA_ERR_TIMEOUT = 7        /* device: a bounded wait inside a kernel expired            */
+    ADA_ERR_TIMEOUT = 7,       /* device: a bounded wait inside a kernel expired            */
+    ADA_ERR_BAD_TAU = 8        /* device: a threshold state outside (0,1) (adaptive step)   */
 } ada_status;
 
 typedef enum { ADA_F32 = 0, ADA_BF16 = 1 } ada_dtype;
@@ -155,6 +156,40 @@ ada_status ada_cascade_step(ada_ctx* ctx, const void* X, int64_t B, int64_t T, i
                             int32_t* add_idx, int32_t* add_cnt, int32_t* rem_idx,
                             int32_t* rem_cnt, float* gamma_rep, float* gamma_cross,
                             uint32_t flags, void* stream);
+
+/*
+ * Cascade step with a device-resident, per-sequence threshold that follows the turnover
+ * (Section 8.1: tau^(l) set from the turnover rate of Eq. (6), which the cascade step yields as
+ * a by-product; a stable set tolerates a tighter threshold, an evolving one needs a looser one).
+ * The paper proposes this and gives no formula; the rule built here is a clipped proportional
+ * step toward a target turnover, each operation rounded once in fp64, in this order:
+ *     rho  = (|add| + |rem|) / |R_in|                        (Eq. 6; undefined for |R_in| = 0)
+ *     tau' = min(tau_max, max(tau_min, tau + gain * (target_turnover - rho)))
+ * and tau' = clip(tau) when rho is undefined.
+ *   tau_state  DEVICE double[B], in/out: sequence b's step uses tau = tau_state[b] (threshold
+ *              (float)(1 - tau^2), as for a host-side tau) and, if policy != NULL, leaves tau'
+ *              there for the next layer.  Nothing returns to the host between layers.  A value
+ *              outside (0,1) or NaN is reported by ada_device_status as ADA_ERR_BAD_TAU.
+ *   policy     HOST struct, read during the call; NULL = leave tau_state unchanged (a fixed
+ *              per-sequence threshold read from device memory).  ADA_ERR_INVALID_ARG unless
+ *              gain >= 0, target_turnover >= 0, 0 < tau_min <= tau_max < 1.
+ *   turnover   DEVICE float[B], optional: rho of this step (NaN where undefined).
+ * Every other argument, the lists and the error behaviour are those of ada_cascade_step.
+ */
+typedef struct {
+    double target_turnover;
+    double gain;
+    double tau_min, tau_max;
+} ada_tau_policy;
+
+ada_status ada_cascade_step_adaptive(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d,
+                                     int64_t ldx, ada_dtype dt, double* tau_state,
+                                     const ada_tau_policy* policy, const int32_t* rep_in,
+                                     const int32_t* rep_in_cnt, int32_t* rep_out,
+                                     int32_t* rep_out_cnt, int32_t* add_idx, int32_t* add_cnt,
+                                     int32_t* rem_idx, int32_t* rem_cnt, float* gamma_rep,
+                                     float* gamma_cross, float* turnover, uint32_t flags,
+                                     void* stream);
 
 /*
  * Per-head selection (Section 8.5: one representative set per attention head, h separate

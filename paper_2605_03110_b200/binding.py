@@ -27,10 +27,17 @@ SYMBOLS = [
     "ada_device_status", "ada_profile_enable", "ada_profile_read", "ada_status_string",
     "ada_select_full_noalloc", "ada_set_cooperative", "ada_selftest_wait_timeout", "ada_nearest_rep",
     "ada_select_full_heads", "ada_cascade_step_heads", "ada_set_dependent_launch",
+    "ada_cascade_step_adaptive",
 ]
 ADA_NOALLOC_MAX_T = 16384
 
 _lib = None
+
+
+class TauPolicy(C.Structure):
+    """ada_tau_policy: tau' = clip(tau + gain * (target_turnover - rho), tau_min, tau_max)."""
+    _fields_ = [("target_turnover", C.c_double), ("gain", C.c_double), ("tau_min", C.c_double),
+                ("tau_max", C.c_double)]
 
 
 class AdaError(RuntimeError):
@@ -60,6 +67,9 @@ def lib() -> C.CDLL:
         L.ada_cascade_step.argtypes = [vp, vp, i64, i64, i64, i64, C.c_int, C.c_double,
                                        i32p, i32p, i32p, i32p, i32p, i32p, i32p, i32p, fp, fp,
                                        C.c_uint32, vp]
+        L.ada_cascade_step_adaptive.argtypes = [vp, vp, i64, i64, i64, i64, C.c_int, vp,
+                                                C.POINTER(TauPolicy), i32p, i32p, i32p, i32p, i32p,
+                                                i32p, i32p, i32p, fp, fp, fp, C.c_uint32, vp]
         L.ada_select_full_heads.argtypes = L.ada_select_full.argtypes
         L.ada_cascade_step_heads.argtypes = L.ada_cascade_step.argtypes
         L.ada_nearest_rep.argtypes = [vp, vp, i64, i64, i64, i64, C.c_int, i32p, i32p, i32p, fp, vp]
@@ -238,6 +248,27 @@ def ada_cascade_step(ctx: Context, X: torch.Tensor, tau: float, rep_in: torch.Te
                                   out.rem_cnt.data_ptr(), _ptr(out.gamma_rep),
                                   _ptr(out.gamma_cross), flags, _stream(stream)),
            "ada_cascade_step")
+    return out
+
+
+def ada_cascade_step_adaptive(ctx: Context, X: torch.Tensor, tau_state: torch.Tensor,
+                              policy: Optional[TauPolicy], rep_in: torch.Tensor,
+                              rep_in_cnt: torch.Tensor, out: Optional[CascadeOut] = None,
+                              flags: int = 0, want_gamma=True, turnover: Optional[torch.Tensor] = None,
+                              stream=None) -> CascadeOut:
+    """Section 8.1: Algorithm 1 with the per-sequence threshold tau_state (float64[B] on the
+    device, updated in place when a policy is given); `turnover` (float32[B]) receives Eq. 6."""
+    X, B, T, d, ldx = _shape(X)
+    assert tau_state.dtype == torch.float64 and tau_state.is_cuda and tau_state.numel() == B
+    if out is None:
+        out = CascadeOut(B, T, X.device, want_gamma)
+    _check(lib().ada_cascade_step_adaptive(
+        ctx.h, X.data_ptr(), B, T, d, ldx, dtype_of(X), tau_state.data_ptr(),
+        None if policy is None else C.byref(policy), rep_in.data_ptr(), rep_in_cnt.data_ptr(),
+        out.rep_out.data_ptr(), out.rep_out_cnt.data_ptr(), out.add_idx.data_ptr(),
+        out.add_cnt.data_ptr(), out.rem_idx.data_ptr(), out.rem_cnt.data_ptr(),
+        _ptr(out.gamma_rep), _ptr(out.gamma_cross), _ptr(turnover), flags, _stream(stream)),
+        "ada_cascade_step_adaptive")
     return out
 
 

@@ -121,6 +121,7 @@ const char* ada_status_string(ada_status s) {
         case ADA_ERR_BAD_INDEX_SET: return "ADA_ERR_BAD_INDEX_SET";
         case ADA_ERR_NONFINITE: return "ADA_ERR_NONFINITE";
         case ADA_ERR_TIMEOUT: return "ADA_ERR_TIMEOUT";
+        case ADA_ERR_BAD_TAU: return "ADA_ERR_BAD_TAU";
     }
     return "ADA_ERR_UNKNOWN";
 }
@@ -169,7 +170,7 @@ ada_status ada_create(ada_ctx** out, int device, int64_t maxB, int64_t maxT, int
     const size_t o_done = take(32), o_agg = take((size_t)maxB * agg_stride * 8);
     const size_t o_near = take(n_tok * 8);
     const size_t o_inv = take(n_tok * 4), o_invr = take(n_tok * 4);
-    const size_t o_reff = take((size_t)maxB * 4), o_stat = take(32);
+    const size_t o_reff = take((size_t)maxB * 4), o_stat = take(32), o_thr = take((size_t)maxB * 4);
     const size_t o_xrep = take(n_tok * (size_t)maxd * ctx->es + 1024);
     const size_t split_bytes = dt == ADA_F32 ? n_tok * (size_t)maxd * 12 + 1024 : 0;
     const size_t o_sxa = take(split_bytes), o_sxb = take(split_bytes), o_sra = take(split_bytes),
@@ -185,6 +186,7 @@ ada_status ada_create(ada_ctx** out, int device, int64_t maxB, int64_t maxT, int
     ctx->inv_norm = reinterpret_cast<float*>(ctx->ws + o_inv);
     ctx->inv_rep = reinterpret_cast<float*>(ctx->ws + o_invr);
     ctx->r_eff = reinterpret_cast<int32_t*>(ctx->ws + o_reff);
+    ctx->thr_seq = reinterpret_cast<float*>(ctx->ws + o_thr);
     ctx->status = reinterpret_cast<unsigned*>(ctx->ws + o_stat);
     ctx->tile_ctr = reinterpret_cast<unsigned*>(ctx->ws + o_ctr);
     ctx->done_ctr = reinterpret_cast<unsigned*>(ctx->ws + o_done);
@@ -335,7 +337,8 @@ static ada_status cascade_impl(ada_ctx* ctx, const void* X, int64_t B, int64_t T
                                const int32_t* rep_in, const int32_t* rep_in_cnt, int32_t* rep_out,
                                int32_t* rep_out_cnt, int32_t* add_idx, int32_t* add_cnt,
                                int32_t* rem_idx, int32_t* rem_cnt, float* gamma_rep,
-                               float* gamma_cross, uint32_t flags, void* stream) {
+                               float* gamma_cross, uint32_t flags, void* stream,
+                               const TauUpdate* tu = nullptr) {
     if (rep_in == nullptr || rep_in_cnt == nullptr || rep_out == nullptr ||
         rep_out_cnt == nullptr || add_idx == nullptr || add_cnt == nullptr ||
         rem_idx == nullptr || rem_cnt == nullptr || !tau_ok(tau))
@@ -344,6 +347,11 @@ static ada_status cascade_impl(ada_ctx* ctx, const void* X, int64_t B, int64_t T
     DeviceGuard guard(ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const float thr = (float)(1.0 - tau * tau);
+    TauUpdate tau_upd;
+    memset(&tau_upd, 0, sizeof(tau_upd));
+    if (tu != nullptr) tau_upd = *tu;
+    const bool adaptive = tau_upd.tau_state != nullptr;
+    if (adaptive) CU(launch_tau_thr(ctx, (int)B, tau_upd.tau_state, s));   // thresholds of this step
 
     // role map, gamma scratch and dependency counter are zero on entry (workspace invariant
     // kept by the compaction kernels).
@@ -387,6 +395,7 @@ static ada_status cascade_impl(ada_ctx* ctx, const void* X, int64_t B, int64_t T
     q.col_gate = ctx->g_rep;
     q.thr_bits = 0;
     memcpy(&q.thr_bits, &thr, 4);
+    q.thr_seq = adaptive ? reinterpret_cast<const unsigned*>(ctx->thr_seq) : nullptr;
     q.col_token = rep_in;
     q.row_role = ctx->role;
     q.causal = (flags & ADA_CROSS_CAUSAL) ? 1 : 0;
@@ -402,8 +411,38 @@ static ada_status cascade_impl(ada_ctx* ctx, const void* X, int64_t B, int64_t T
     else CU(run_gram(ctx, q, dt, s));
     // lines 5, 9, 10-11
     CU(launch_compact_cascade(ctx, (int)B, (int)T, thr, rep_out, rep_out_cnt, add_idx, add_cnt,
-                              rem_idx, rem_cnt, gamma_rep, gamma_cross, s));
+                              rem_idx, rem_cnt, gamma_rep, gamma_cross, tau_upd, s));
     return ADA_OK;
+}
+
+ada_status ada_cascade_step_adaptive(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d,
+                                     int64_t ldx, ada_dtype dt, double* tau_state,
+                                     const ada_tau_policy* policy, const int32_t* rep_in,
+                                     const int32_t* rep_in_cnt, int32_t* rep_out,
+                                     int32_t* rep_out_cnt, int32_t* add_idx, int32_t* add_cnt,
+                                     int32_t* rem_idx, int32_t* rem_cnt, float* gamma_rep,
+                                     float* gamma_cross, float* turnover, uint32_t flags,
+                                     void* stream) {
+    ada_status st = check_common(ctx, X, B, T, d, ldx, dt);
+    if (st != ADA_OK) return st;
+    if (tau_state == nullptr) return ADA_ERR_INVALID_ARG;
+    TauUpdate tu;
+    memset(&tu, 0, sizeof(tu));
+    tu.tau_state = tau_state;
+    tu.turnover = turnover;
+    if (policy != nullptr) {
+        // also rejects NaN in any field
+        if (!(policy->gain >= 0.0) || !(policy->target_turnover >= 0.0) || !(policy->tau_min > 0.0) ||
+            !(policy->tau_max < 1.0) || !(policy->tau_min <= policy->tau_max))
+            return ADA_ERR_INVALID_ARG;
+        tu.update = 1;
+        tu.target = policy->target_turnover; tu.gain = policy->gain;
+        tu.tau_min = policy->tau_min; tu.tau_max = policy->tau_max;
+    }
+    // the host-side tau of the fixed-threshold call is not used; 0.5 passes its range check
+    return cascade_impl(ctx, X, B, T, d, ldx, T * ldx, dt, 0.5, rep_in, rep_in_cnt, rep_out,
+                        rep_out_cnt, add_idx, add_cnt, rem_idx, rem_cnt, gamma_rep, gamma_cross,
+                        flags, stream, &tu);
 }
 
 ada_status ada_cascade_step(ada_ctx* ctx, const void* X, int64_t B, int64_t T, int64_t d,
@@ -490,6 +529,7 @@ ada_status ada_device_status(ada_ctx* ctx, void* stream, int64_t* n_zero_norm_ro
     if (h[0] & ST_TIMEOUT) return ADA_ERR_TIMEOUT;
     if (h[0] & (ST_BAD_INDEX | ST_BAD_COUNT)) return ADA_ERR_BAD_INDEX_SET;
     if (h[0] & ST_NONFINITE) return ADA_ERR_NONFINITE;
+    if (h[0] & ST_BAD_TAU) return ADA_ERR_BAD_TAU;
     return ADA_OK;
 }
 

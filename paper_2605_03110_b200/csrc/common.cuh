@@ -16,6 +16,7 @@ enum : unsigned {
     ST_BAD_COUNT = 1u << 1,  // a count outside [0,T]
     ST_NONFINITE = 1u << 2,  // NaN / Inf met while normalising
     ST_TIMEOUT = 1u << 3,    // a bounded wait in a kernel ran out
+    ST_BAD_TAU = 1u << 4,    // a device-resident threshold state outside (0,1)
 };
 // status[1] counts zero-norm rows, status[2] records where a wait gave up.
 
@@ -61,6 +62,7 @@ struct GramProblem {
     // cross only
     const unsigned* col_gate; // [B*cap] gamma_rep bits by position
     unsigned thr_bits;        // bit pattern of (float)thr
+    const unsigned* thr_seq;  // per-sequence bit patterns instead (adaptive threshold), or NULL
     const int32_t* col_token; // [B*cap] token index of each column (causal) or NULL
     const int32_t* row_role;  // [B*cap] 0 for non-representatives
     int causal;
@@ -113,6 +115,7 @@ struct ada_ctx {
     unsigned* g_rep;     // [maxB*maxT] gamma_rep by position, bit patterns
     int32_t* role;       // [maxB*maxT] 0 = not inherited, p+1 = position p in the inherited list
     int32_t* r_eff;      // [maxB] sanitised inherited counts
+    float* thr_seq;      // [maxB] per-sequence (float)(1 - tau^2) of an adaptive step
     unsigned* status;    // [8]
     unsigned* tile_ctr;  // [8] dependency counter of the fused Gram launch
     unsigned long long* agg;  // [maxB][agg_stride] block counts published by the compaction
@@ -182,10 +185,19 @@ cudaError_t launch_nearest_finish(ada_ctx* ctx, int B, int T, const int32_t* rep
                                   int32_t* nearest_idx, float* nearest_gamma, cudaStream_t s);
 cudaError_t launch_compact_full(ada_ctx* ctx, int B, int T, float thr, int32_t* rep_idx,
                                 int32_t* rep_cnt, float* gamma, cudaStream_t s);
+// adaptive threshold (Section 8.1): tau_state != NULL makes the step use ctx->thr_seq and update
+// tau_state / write the turnover of Eq. (6) once the counts are known
+struct TauUpdate {
+    double* tau_state;     // [B] device, in/out; NULL = fixed threshold
+    float* turnover;       // [B] device, optional
+    int update;            // 0: leave tau_state as it is
+    double target, gain, tau_min, tau_max;
+};
+cudaError_t launch_tau_thr(ada_ctx* ctx, int B, const double* tau_state, cudaStream_t s);
 cudaError_t launch_compact_cascade(ada_ctx* ctx, int B, int T, float thr, int32_t* rep_out,
                                    int32_t* rep_out_cnt, int32_t* add_idx, int32_t* add_cnt,
                                    int32_t* rem_idx, int32_t* rem_cnt, float* gamma_rep,
-                                   float* gamma_cross, cudaStream_t s);
+                                   float* gamma_cross, const TauUpdate& tu, cudaStream_t s);
 
 // gram_ffma.cu
 cudaError_t launch_gram_ffma(ada_ctx* ctx, const GramProblem& p, ada_dtype dt, cudaStream_t s);

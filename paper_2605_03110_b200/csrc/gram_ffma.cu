@@ -109,7 +109,7 @@ k_gram_ffma(const GramProblem p) {
         if (cok[j]) {
             cs[j] = p.inv_b[o + c];
             if (!p.tri) {
-                cok[j] = p.col_gate[o + c] < p.thr_bits;      // valid representative (line 5)
+                cok[j] = p.col_gate[o + c] < (p.thr_seq != nullptr ? p.thr_seq[b] : p.thr_bits);   // valid representative (line 5)
                 if (p.causal) ctok[j] = p.col_token[o + c];
             }
         }

@@ -360,6 +360,7 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
                 unsigned gate[BN / 32] = {};
                 int tk[BN / 32] = {};
                 const int last = pc.n - 1;
+                const unsigned thr_b = (!p.tri && p.thr_seq != nullptr) ? p.thr_seq[pc.b] : p.thr_bits;
 #pragma unroll
                 for (int q = 0; q < BN / 32; ++q)
                     fb[q] = __ldcg(p.inv_b + o + min(pc.col0 + lane + 32 * q, last));
@@ -379,7 +380,7 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
                     const int c = lane + 32 * q, col = pc.col0 + c;
                     const bool live = col < pc.n;
                     if (c < ncols) {
-                        cs[c] = (live && (p.tri || gate[q] < p.thr_bits)) ? fb[q] : 0.f;
+                        cs[c] = (live && (p.tri || gate[q] < thr_b)) ? fb[q] : 0.f;
                         ct[c] = (live && !p.tri && p.causal) ? tk[q] : col;
                     }
                 }

@@ -451,7 +451,22 @@ struct CompactArgs {
     float thr;
     int32_t *keep_idx, *keep_cnt, *add_idx, *add_cnt, *rem_idx, *rem_cnt;
     float *gamma_a, *gamma_b;    // full: gamma | cascade: gamma_rep, gamma_cross (optional)
+    // adaptive threshold (Section 8.1)
+    const float* thr_seq;        // [B] thresholds of this step, or NULL = thr
+    const int32_t* r_in;         // [B] inherited counts (Eq. 6 denominator)
+    TauUpdate tu;
 };
+
+// thr_seq[b] = (float)(1 - tau_b^2), 1 - tau^2 in fp64 as for a host-side tau
+__global__ void k_tau_thr(const double* __restrict__ tau_state, int B, float* __restrict__ thr_seq,
+                          unsigned* __restrict__ status) {
+    grid_dep_wait();
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    const double tau = tau_state[b];
+    if (!(tau > 0.0 && tau < 1.0)) atomicOr(status, ST_BAD_TAU);
+    thr_seq[b] = (float)__dsub_rn(1.0, __dmul_rn(tau, tau));
+}
 
 __device__ __forceinline__ unsigned long long block_exclusive_scan(unsigned long long v,
                                                                    unsigned long long* s_warp,
@@ -493,6 +508,7 @@ __global__ void __launch_bounds__(1024) k_compact(const CompactArgs a) {
     const bool in = t < a.T;
     const bool cascade = a.role != nullptr;
     const unsigned faulted = a.status[0];
+    const float thr = a.thr_seq != nullptr ? a.thr_seq[b] : a.thr;
 
     // independent loads first, the position-indexed gather second
     const int pos = (cascade && in) ? a.role[o + t] : 0;
@@ -503,13 +519,13 @@ __global__ void __launch_bounds__(1024) k_compact(const CompactArgs a) {
         float ga = 0.f, gb = 0.f;
         if (pos > 0) {                    // inherited representative: line 5
             ga = __uint_as_float(gp);
-            keep = ga < a.thr;
+            keep = ga < thr;
             rem = !keep;
             a.g_rep[o + pos - 1] = 0u;
             a.role[o + t] = 0;
         } else {                          // Definition 1 / line 9
             gb = __uint_as_float(gt);
-            keep = gb < a.thr;
+            keep = gb < thr;
             add = cascade && keep;
         }
         a.g_tok[o + t] = 0u;
@@ -557,8 +573,25 @@ __global__ void __launch_bounds__(1024) k_compact(const CompactArgs a) {
         const unsigned long long all = base + total;
         a.keep_cnt[b] = (int)(all & AGG_MASK);
         if (cascade) {
-            a.add_cnt[b] = (int)((all >> 21) & AGG_MASK);
-            a.rem_cnt[b] = (int)((all >> 42) & AGG_MASK);
+            const int n_add = (int)((all >> 21) & AGG_MASK), n_rem = (int)((all >> 42) & AGG_MASK);
+            a.add_cnt[b] = n_add;
+            a.rem_cnt[b] = n_rem;
+            if (a.tu.tau_state != nullptr) {
+                // Eq. (6), then the threshold of the next layer: one rounded fp64 operation at a
+                // time (no fused multiply-add), so that the state is reproducible bit for bit
+                const int r_in = a.r_in[b];
+                const bool defined = r_in > 0;
+                const double rho = defined ? __ddiv_rn((double)(n_add + n_rem), (double)r_in) : 0.0;
+                if (a.tu.turnover != nullptr)
+                    a.tu.turnover[b] = defined ? (float)rho : __int_as_float(0x7fc00000);
+                if (a.tu.update) {
+                    double t = a.tu.tau_state[b];
+                    if (defined) t = __dadd_rn(t, __dmul_rn(a.tu.gain, __dsub_rn(a.tu.target, rho)));
+                    if (t < a.tu.tau_min) t = a.tu.tau_min;
+                    if (t > a.tu.tau_max) t = a.tu.tau_max;
+                    a.tu.tau_state[b] = t;
+                }
+            }
         }
     }
     // the last block to finish restores the zero state of the shared words
@@ -641,13 +674,15 @@ cudaError_t launch_compact_full(ada_ctx* ctx, int B, int T, float thr, int32_t* 
     a.keep_idx = rep_idx; a.keep_cnt = rep_cnt;
     a.add_idx = nullptr; a.add_cnt = nullptr; a.rem_idx = nullptr; a.rem_cnt = nullptr;
     a.gamma_a = gamma; a.gamma_b = nullptr;
+    a.thr_seq = nullptr; a.r_in = nullptr;
+    memset(&a.tu, 0, sizeof(a.tu));
     return launch_compact(ctx, K_COMPACT_FULL, a, B, s);
 }
 
 cudaError_t launch_compact_cascade(ada_ctx* ctx, int B, int T, float thr, int32_t* rep_out,
                                    int32_t* rep_out_cnt, int32_t* add_idx, int32_t* add_cnt,
                                    int32_t* rem_idx, int32_t* rem_cnt, float* gamma_rep,
-                                   float* gamma_cross, cudaStream_t s) {
+                                   float* gamma_cross, const TauUpdate& tu, cudaStream_t s) {
     CompactArgs a;
     a.g_tok = ctx->g_tok; a.g_rep = ctx->g_rep; a.role = ctx->role;
     a.agg = ctx->agg; a.done_ctr = ctx->done_ctr; a.dep_ctr = ctx->tile_ctr; a.status = ctx->status;
@@ -655,7 +690,15 @@ cudaError_t launch_compact_cascade(ada_ctx* ctx, int B, int T, float thr, int32_
     a.keep_idx = rep_out; a.keep_cnt = rep_out_cnt;
     a.add_idx = add_idx; a.add_cnt = add_cnt; a.rem_idx = rem_idx; a.rem_cnt = rem_cnt;
     a.gamma_a = gamma_rep; a.gamma_b = gamma_cross;
+    a.thr_seq = tu.tau_state != nullptr ? ctx->thr_seq : nullptr;
+    a.r_in = ctx->r_eff;
+    a.tu = tu;
     return launch_compact(ctx, K_COMPACT_CASCADE, a, B, s);
+}
+
+cudaError_t launch_tau_thr(ada_ctx* ctx, int B, const double* tau_state, cudaStream_t s) {
+    launch_k(ctx, k_tau_thr, dim3((B + 127) / 128), dim3(128), 0, s, tau_state, B, ctx->thr_seq, ctx->status);
+    return cudaGetLastError();
 }
 
 }  // namespace ada

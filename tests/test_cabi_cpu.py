@@ -53,7 +53,7 @@ def test_status_strings(lib):
     f = lib.ada_status_string
     f.restype = ctypes.c_char_p
     f.argtypes = [ctypes.c_int]
-    assert f(0) == b"ADA_OK" and f(7) == b"ADA_ERR_TIMEOUT"
+    assert f(0) == b"ADA_OK" and f(7) == b"ADA_ERR_TIMEOUT" and f(8) == b"ADA_ERR_BAD_TAU"
     assert len({f(i) for i in range(8)}) == 8
 
 
