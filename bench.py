@@ -516,8 +516,13 @@ def main():
     if bound == "tensor" and cfg.dtype == "bf16":
         peak, unit, achieved = peaks["bf16_sustained"], "TFLOP/s", alg / secs / 1e12
         peak_note = f"cuBLAS bf16 sustained, {peaks['src']}"
+    elif bound == "tensor" and "tc" in dom:
+        # fp32 storage on the tensor cores: every fp32 product is six bf16 products (three-term
+        # split), so the ceiling for ALGORITHMIC fp32 flops is the bf16 peak / 6
+        peak, unit, achieved = peaks["bf16_sustained"] / 6.0, "TFLOP/s", alg / secs / 1e12
+        peak_note = f"cuBLAS bf16 sustained / 6 (fp32 as six bf16 products), {peaks['src']}"
     elif bound == "tensor":
-        # fp32 FFMA path: 148 SMs x 128 lanes x 2 flop x max SM clock
+        # fp32 FFMA kernel: 148 SMs x 128 lanes x 2 flop x max SM clock
         peak, unit, achieved = 148 * 128 * 2 * 1.965e9 / 1e12, "TFLOP/s", alg / secs / 1e12
         bound, peak_note = "alu", "148 SMs x 128 FFMA lanes x 2 flop x 1.965 GHz (derived)"
     else:
