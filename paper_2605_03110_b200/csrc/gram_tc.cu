@@ -22,7 +22,7 @@
 //   warps 6..13 optional row norms (Section 2.1): 1/||x_t|| of every row of X with plain
 //               128-bit loads, overlapped with the main loops; the epilogues wait (bounded)
 //               for them before they scale, so a long-K call needs no separate norm pass
-// Short-contraction shape (d <= 512, no norm warps), 10 warps: warps 6..9 are a second
+// Short-contraction shape (d < 2048, no norm warps), 10 warps: warps 6..9 are a second
 // epilogue set; see Shape below.
 // Every wait is bounded: when a limit expires the CTA raises the context's TIMEOUT
 // status, drains its own outstanding copies and MMAs (again bounded), frees its TMEM
@@ -38,8 +38,8 @@ namespace {
 
 // The kernel comes in two shapes.  The long-contraction shape (14 warps, the last eight for the
 // optional row norms) lives off its main loop: one epilogue set, a 216 KiB ring whose stage size
-// follows each tile's width.  The short-contraction shape (d <= 512, e.g. one attention head)
-// lives off its epilogue, because a 128 x 256 fp32 accumulator takes about 2300 cycles to read
+// follows each tile's width.  The short-contraction shape (d < 2048: one attention head, a small
+// model width) lives off its epilogue, because a 128 x 256 fp32 accumulator takes about 2300 cycles to read
 // out of TMEM, more than such a tile's main loop: 10 warps, two epilogue sets that take
 // alternate tiles (one accumulator each, so that one set's bookkeeping -- tile lookup, column
 // factors, barrier, atomics -- overlaps the other's TMEM reads), a ring geometry fixed per
@@ -810,7 +810,7 @@ cudaError_t launch_gram_tc(ada_ctx* ctx, const GramProblem* tri, const GramProbl
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3(ctx->sm_count);
     // short contraction and no norm warps needed: the epilogue-bound shape
-    const bool shortk = nj.X == nullptr && segs[0].d <= 512;
+    const bool shortk = nj.X == nullptr && segs[0].d < 2048;
     cfg.blockDim = dim3(shortk ? Shape<true>::THREADS : Shape<false>::THREADS);
     cfg.dynamicSmemBytes = shortk ? smem_tc_bytes<true>() : smem_tc_bytes<false>();
     cfg.stream = s;
