@@ -158,3 +158,36 @@ def test_heads_error_paths(ada):
     st, _ = ada.ada_device_status(ctx)
     assert st == 0
     ada.ada_destroy(ctx)
+
+
+def test_heads_on_long_sequence_past_the_tile_table(ada):
+    """T = 8192 as 32 heads x 128: every CTA gets a few hundred tiles, far more than the 80 its
+    shared-memory table holds, so most tiles are located by the on-the-fly search.  Two heads are
+    checked in full against the oracle, full selection and one cascade step."""
+    from parity import TOL, check_set, lists, to_device
+    cfg = wl.CONFIGS[4]
+    h, d_h, T = 32, cfg.d // 32, cfg.T
+    tol = TOL["bf16"]
+    thr = 1.0 - cfg.tau * cfg.tau
+    gen = wl.generate_layers(cfg, seed=0, n_layers=2)
+    X0, X1 = [lb.X[0].reshape(T, h, d_h) for lb in gen]
+    ctx = ada.ada_create(h, T, d_h, ada.ADA_BF16)
+    idx, cnt, gamma = ada.ada_select_full_heads(ctx, to_device(X0), cfg.tau)
+    out = ada.ada_cascade_step_heads(ctx, to_device(X1), cfg.tau, idx, cnt)
+    st, _ = ada.ada_device_status(ctx)
+    assert st == 0
+    reps, reps1 = lists(idx, cnt), lists(out.rep_out, out.rep_out_cnt)
+    g, gc, gr = gamma.cpu().numpy(), out.gamma_cross.cpu().numpy(), out.gamma_rep.cpu().numpy()
+    for j in (0, 17):
+        x0 = wl.as_f64(np.ascontiguousarray(X0[:, j]))
+        ref_rep, ref_g = oracle.select_full(x0, cfg.tau)
+        assert np.max(np.abs(g[j] - ref_g)) <= tol
+        assert check_set(reps[j], ref_g, np.arange(T), thr, tol) == 0
+        assert reps[j].tolist() == ref_rep.tolist()
+        ref = oracle.cascade_step(wl.as_f64(np.ascontiguousarray(X1[:, j])), cfg.tau, ref_rep)
+        g_rep_tok = np.zeros(T)
+        g_rep_tok[ref_rep] = ref.gamma_rep
+        assert np.max(np.abs(gr[j] - g_rep_tok)) <= tol
+        assert np.max(np.abs(gc[j] - ref.gamma_cross)) <= tol
+        assert reps1[j].tolist() == ref.rep.tolist()
+    ada.ada_destroy(ctx)
