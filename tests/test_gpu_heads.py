@@ -42,8 +42,9 @@ def perturbed(X, seed, scale=0.3):
 
 
 @pytest.mark.parametrize("dtype,engine", [("bf16", 0), ("bf16", 1), ("bf16", 2), ("f32", 0), ("f32", 1)])
+# (150, 80, 64): more sequences than the kernel keeps sequence tables for
 @pytest.mark.parametrize("T,h,d_h", [(1, 1, 8), (2, 3, 8), (129, 3, 72), (300, 8, 64), (600, 5, 128),
-                                     (257, 2, 256)])
+                                     (257, 2, 256), (150, 80, 64)])
 def test_heads_small_shapes(ada, dtype, engine, T, h, d_h):
     from parity import check_cascade, check_full
     ctx = ada.ada_create(h, T, d_h, ada.ADA_F32 if dtype == "f32" else ada.ADA_BF16)
