@@ -18,7 +18,7 @@ def ada():
     return binding
 
 
-def run_chain(ada, cfg, tau0, policy, causal=False, seed=0):
+def run_chain(ada, cfg, tau0, policy, causal=False, seed=0, engine=0):
     """Free-running GPU chain with per-sequence thresholds; every step is checked against the
     oracle run with the same threshold and the same inherited set, the threshold state against
     the oracle's update rule fed with the step's own counts (bit for bit)."""
@@ -26,6 +26,7 @@ def run_chain(ada, cfg, tau0, policy, causal=False, seed=0):
     tol = TOL[cfg.dtype]
     B, T = cfg.B, cfg.T
     ctx = ada.ada_create(B, T, cfg.d, ada.ADA_F32 if cfg.dtype == "f32" else ada.ADA_BF16)
+    ada.ada_set_engine(ctx, engine)
     tau = np.array(tau0, dtype=np.float64)
     tau_dev = torch.from_numpy(tau.copy()).cuda()
     turn = torch.empty(B, dtype=torch.float32, device="cuda")
@@ -95,9 +96,19 @@ def test_adaptive_chain_bf16_batched(ada, causal):
     assert not np.array_equal(hist[0], hist[-1])          # the thresholds did move
 
 
-def test_adaptive_chain_fp32(ada):
+# engines: 0 automatic, 1 FFMA kernel, 3 pair-CTA tensor-core kernel (each reads the per-sequence
+# threshold in its own epilogue)
+@pytest.mark.parametrize("engine", [0, 1, 3])
+def test_adaptive_chain_fp32(ada, engine):
     cfg = wl.scaled(wl.CONFIGS[1], T=500, d=192, L=6, P=50)
-    band, hist = run_chain(ada, cfg, [0.3], (0.05, 1.0, 0.15, 0.5))
+    band, hist = run_chain(ada, cfg, [0.3], (0.05, 1.0, 0.15, 0.5), engine=engine)
+    assert band == 0
+
+
+@pytest.mark.parametrize("engine", [1, 2, 3])
+def test_adaptive_chain_bf16_on_every_engine(ada, engine):
+    cfg = wl.scaled(wl.CONFIGS[2], B=2, T=520, d=320, L=5, P=50)
+    band, hist = run_chain(ada, cfg, [0.25, 0.4], (0.08, 0.5, 0.1, 0.6), engine=engine)
     assert band == 0
 
 
