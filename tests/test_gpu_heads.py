@@ -41,7 +41,8 @@ def perturbed(X, seed, scale=0.3):
     return X + scale * rng.standard_normal(X.shape).astype(np.float32)
 
 
-@pytest.mark.parametrize("dtype,engine", [("bf16", 0), ("bf16", 1), ("bf16", 2), ("f32", 0), ("f32", 1)])
+@pytest.mark.parametrize("dtype,engine", [("bf16", 0), ("bf16", 1), ("bf16", 2), ("bf16", 3), ("f32", 0),
+                                          ("f32", 1), ("f32", 3)])
 # (150, 80, 64): more sequences than the kernel keeps sequence tables for
 @pytest.mark.parametrize("T,h,d_h", [(1, 1, 8), (2, 3, 8), (129, 3, 72), (300, 8, 64), (600, 5, 128),
                                      (257, 2, 256), (150, 80, 64)])
