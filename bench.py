@@ -38,6 +38,10 @@ NCU_TRAFFIC_BYTES = {
     # fused cascade launch on configs[3]: mean of the captured layers 1 (76.9 MB) and 30 (108.4 MB),
     # profiles/gram_tc2_cascade_cfg4.md
     ("gram_tc_cascade", 4): 92.65e6,
+    # fused cascade launches of layers 1-2 on the smaller workloads, profiles/gram_tc_traffic_cfg1-3.md
+    ("gram_tc_cascade", 1): 9.53e6,
+    ("gram_tc_cascade", 2): 28.9e6,
+    ("gram_tc_cascade", 3): 21.08e6,
 }
 
 
