@@ -39,8 +39,8 @@ namespace {
 // The kernel comes in two shapes.  The long-contraction shape (14 warps, the last eight for the
 // optional row norms) lives off its main loop: one epilogue set, a 216 KiB ring whose stage size
 // follows each tile's width.  The short-contraction shape (d < 2048: one attention head, a small
-// model width) lives off its epilogue, because a 128 x 256 fp32 accumulator takes about 2300 cycles to read
-// out of TMEM, more than such a tile's main loop: 10 warps, two epilogue sets that take
+// model width) lives off its epilogue, because a 128 x 256 fp32 accumulator takes about 2300
+// cycles to read out of TMEM, more than such a tile's main loop: 10 warps, two epilogue sets that take
 // alternate tiles (one accumulator each, so that one set's bookkeeping -- tile lookup, column
 // factors, barrier, atomics -- overlaps the other's TMEM reads), a ring geometry fixed per
 // segment (no drain between tiles of different width), one 256-row TMA box for a full-width
