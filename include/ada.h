@@ -88,7 +88,9 @@ typedef struct ada_ctx ada_ctx; /* opaque */
 /* Create a context on `device` able to serve up to maxB sequences of maxT
  * tokens of width maxd in storage type dt.  Allocates the workspace
  * (cudaMalloc; about maxB*maxT*(maxd*es + 32) bytes, plus 48*maxB*maxT*maxd for ADA_F32).
- * *out is NULL on error. */
+ * maxT may not exceed ADA_MAX_T (the list counts of one sequence are kept in 21-bit fields),
+ * nor maxB*maxT 2^30: ADA_ERR_INVALID_ARG.  *out is NULL on error. */
+#define ADA_MAX_T ((int64_t)2097151)
 ada_status ada_create(ada_ctx** out, int device, int64_t maxB, int64_t maxT, int64_t maxd,
                       ada_dtype dt);
 ada_status ada_destroy(ada_ctx* ctx);
@@ -269,8 +271,12 @@ ada_status ada_cascade_step_host(ada_ctx* ctx, const void* X, int64_t B, int64_t
  *   - All calls on a device share the one scratch array, and it keeps the previous call's
  *     contents; the call itself clears what must start at zero.  Two calls whose kernels
  *     overlap on the GPU (different streams) race on it: keep them stream-ordered.
- *   - Device-detected faults (NaN/Inf) cannot be read back through a context here; check
- *     the inputs upstream if that matters.
+ *   - Device-detected faults (NaN/Inf in X, an expired bounded wait) cannot be read back
+ *     through a context here; check the inputs upstream if that matters.
+ *   - ADA_F32 input runs on the plain fp32 (FFMA) Gram kernel here, ADA_BF16 on the
+ *     one-CTA tensor-core kernel.
+ *   - The host side is safe to call from several threads (the per-device set-up runs once,
+ *     under a guard); the GPU work of concurrent callers must still be stream-ordered.
  */
 #define ADA_NOALLOC_MAX_T 16384
 ada_status ada_select_full_noalloc(const void* X, int64_t T, int64_t d, int64_t ldx,

@@ -140,7 +140,8 @@ ada_status ada_create(ada_ctx** out, int device, int64_t maxB, int64_t maxT, int
     *out = nullptr;
     if (maxB < 1 || maxT < 1 || maxd < 1 || (dt != ADA_F32 && dt != ADA_BF16))
         return ADA_ERR_INVALID_ARG;
-    if (maxT > (int64_t)1 << 24 || maxB * maxT > (int64_t)1 << 30) return ADA_ERR_INVALID_ARG;
+    // the compaction packs three per-sequence counts into 21-bit fields
+    if (maxT > ADA_MAX_T || maxB * maxT > (int64_t)1 << 30) return ADA_ERR_INVALID_ARG;
     int ndev = 0;
     if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev)
         return ADA_ERR_CUDA;
@@ -584,6 +585,9 @@ ada_status ada_select_full_host(ada_ctx* ctx, const void* X, int64_t B, int64_t 
     if (ctx == nullptr || X == nullptr || rep_idx == nullptr || rep_cnt == nullptr)
         return ADA_ERR_INVALID_ARG;
     if (B < 1 || T < 1 || d < 1) return ADA_ERR_INVALID_ARG;
+    if (dt != ADA_F32 && dt != ADA_BF16) return ADA_ERR_INVALID_ARG;
+    // before anything is copied: the copies below are sized by the context's element type
+    if (dt != ctx->dt || (d * ctx->es) % 16 != 0) return ADA_ERR_UNSUPPORTED;
     if (B > ctx->maxB || T > ctx->maxT || d > ctx->maxd) return ADA_ERR_WORKSPACE;
     DeviceGuard guard(ctx->device);
     ada_status st = ensure_stage(ctx);
@@ -612,6 +616,9 @@ ada_status ada_cascade_step_host(ada_ctx* ctx, const void* X, int64_t B, int64_t
         add_cnt == nullptr || rem_idx == nullptr || rem_cnt == nullptr)
         return ADA_ERR_INVALID_ARG;
     if (B < 1 || T < 1 || d < 1) return ADA_ERR_INVALID_ARG;
+    if (dt != ADA_F32 && dt != ADA_BF16) return ADA_ERR_INVALID_ARG;
+    // before anything is copied: the copies below are sized by the context's element type
+    if (dt != ctx->dt || (d * ctx->es) % 16 != 0) return ADA_ERR_UNSUPPORTED;
     if (B > ctx->maxB || T > ctx->maxT || d > ctx->maxd) return ADA_ERR_WORKSPACE;
     DeviceGuard guard(ctx->device);
     ada_status st = ensure_stage(ctx);

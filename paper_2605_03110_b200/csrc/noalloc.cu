@@ -8,6 +8,8 @@
 // allocator calls.  Such callers cannot create an ada_ctx, whose workspace is one cudaMalloc.
 #include <string.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 using namespace ada;
@@ -26,22 +28,25 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[kScratchBytes];
 
 constexpr int kMaxDevices = 16;
 struct PerDevice {
-    bool ready;
+    std::once_flag once;
+    ada_status setup_status;
     unsigned char* scratch;   // device address of g_noalloc_scratch on this device
-    ada_ctx ctx;              // host-side bookkeeping only; owns no memory
+    ada_ctx ctx;              // host-side bookkeeping only; owns no memory; written once, at set-up
 };
 PerDevice g_dev[kMaxDevices];
 
-// One-time set-up for the current device.  In host code the array's name is only a handle:
-// the address a kernel can use has to be asked for, with this device current.
+// One-time set-up for the current device (guarded: two host threads may make their first call
+// at once).  In host code the array's name is only a handle: the address a kernel can use has
+// to be asked for, with this device current.
 ada_status setup_device(int device, PerDevice** out) {
     if (device < 0 || device >= kMaxDevices) return ADA_ERR_UNSUPPORTED;
     PerDevice& pd = g_dev[device];
-    if (!pd.ready) {
+    std::call_once(pd.once, [&pd, device]() {
+        pd.setup_status = ADA_ERR_CUDA;
         void* ptr = nullptr;
         if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr) {
             cudaGetLastError();
-            return ADA_ERR_CUDA;
+            return;
         }
         pd.scratch = static_cast<unsigned char*>(ptr);
         ada_ctx& c = pd.ctx;
@@ -49,9 +54,12 @@ ada_status setup_device(int device, PerDevice** out) {
         c.maxB = 1;
         c.maxT = ADA_NOALLOC_MAX_T;
         c.maxd = 0;
+        c.dt = ADA_BF16;               // unused: the storage type travels as an argument
+        c.es = 2;
         c.engine = ADA_ENGINE_AUTO;
         c.tc_attr_set = false;
         c.cooperative = true;
+        c.dep_launch = false;          // plain stream order between this call's launches
         c.tc2_attr_set = false;
         c.tc2_pairs = 0;
         c.ws = nullptr;
@@ -59,7 +67,7 @@ ada_status setup_device(int device, PerDevice** out) {
         c.stage_bytes = 0;
         c.host_stream = nullptr;
         if (cudaDeviceGetAttribute(&c.sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
-            return ADA_ERR_CUDA;
+            return;
         c.g_tok = reinterpret_cast<unsigned*>(pd.scratch);
         c.inv_norm = reinterpret_cast<float*>(pd.scratch + kGammaBytes);
         c.status = reinterpret_cast<unsigned*>(pd.scratch + kGammaBytes + kInvBytes);
@@ -71,13 +79,14 @@ ada_status setup_device(int device, PerDevice** out) {
         c.inv_rep = nullptr;
         c.role = nullptr;
         c.r_eff = nullptr;
+        c.thr_seq = nullptr;
         c.Xrep = nullptr;
         c.near_key = nullptr;
         c.splitXA = c.splitXB = c.splitRA = c.splitRB = nullptr;
-        pd.ready = true;
-    }
+        pd.setup_status = ADA_OK;
+    });
     *out = &pd;
-    return ADA_OK;
+    return pd.setup_status;
 }
 
 }  // namespace
@@ -98,8 +107,6 @@ extern "C" ada_status ada_select_full_noalloc(const void* X, int64_t T, int64_t 
     ada_status st = setup_device(device, &pd);
     if (st != ADA_OK) return st;
     ada_ctx* ctx = &pd->ctx;
-    ctx->dt = dt;
-    ctx->es = (int)es;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const float thr = (float)(1.0 - tau * tau);
 

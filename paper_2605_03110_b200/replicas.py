@@ -35,11 +35,7 @@ def from_env() -> Replica:
 def init_process_group(rep: Replica, backend: str, device=None) -> None:
     if rep.world > 1 and not dist.is_initialized():
         kw = {"device_id": device} if (backend == "nccl" and device is not None) else {}
-        dist.init_process_group(backend, rank=rank_or_none(rep), world_size=rep.world, **kw)
-
-
-def rank_or_none(rep: Replica) -> int:
-    return rep.rank
+        dist.init_process_group(backend, rank=rep.rank, world_size=rep.world, **kw)
 
 
 def barrier(rep: Replica) -> None:

@@ -64,4 +64,7 @@ def test_create_rejects_bad_arguments_before_touching_a_device(lib):
     assert f(ctypes.byref(h), 0, 0, 128, 64, 0) == 1            # ADA_ERR_INVALID_ARG
     assert f(ctypes.byref(h), 0, 1, 128, 64, 5) == 1
     assert f(None, 0, 1, 128, 64, 0) == 1
+    # the per-sequence list counts live in 21-bit fields: longer sequences are refused
+    assert f(ctypes.byref(h), 0, 1, (1 << 21), 64, 1) == 1
+    assert f(ctypes.byref(h), 0, 1 << 12, 1 << 20, 64, 1) == 1   # maxB * maxT above 2^30
     assert h.value is None

@@ -120,7 +120,7 @@ def test_config2_and_3_on_both_tensor_core_kernels(ada, engine):
     assert run_config_chain(ada, wl.CONFIGS[3], n_layers=4, engine=engine) == 0
 
 
-def sampled_large(ada, cfg, n_layers, n_sample=48, engine=0):
+def sampled_large(ada, cfg, n_layers, n_sample=48, engine=0, per_tile=False):
     """Full-size check where the oracle cannot do a whole layer quickly: sets by the
     label-level prediction (exact, no Gram), gamma on sampled rows by the oracle."""
     from parity import TOL, lists, to_device
@@ -136,7 +136,8 @@ def sampled_large(ada, cfg, n_layers, n_sample=48, engine=0):
         rep_idx, rep_cnt, gamma = ada.ada_select_full(ctx, Xd, cfg.tau)
         full = lists(rep_idx, rep_cnt)[0]
         assert full.tolist() == full_from_labels(lab).tolist()
-        rows = np.sort(rng.choice(cfg.T, n_sample, replace=False)).astype(np.int32)
+        rows = tile_rows(rng, cfg.T, n_sample) if per_tile else \
+            np.sort(rng.choice(cfg.T, n_sample, replace=False)).astype(np.int32)
         g_ref = oracle.full_rows(X64, rows)
         assert np.max(np.abs(gamma.cpu().numpy()[0][rows] - g_ref)) <= tol
         if lb.layer == 0:
@@ -149,7 +150,10 @@ def sampled_large(ada, cfg, n_layers, n_sample=48, engine=0):
         assert lists(out.add_idx, out.add_cnt)[0].tolist() == exp_add.tolist()
         assert lists(out.rem_idx, out.rem_cnt)[0].tolist() == exp_rem.tolist()
         nonrep = np.setdiff1d(np.arange(cfg.T), R_lab)
-        rows = np.sort(rng.choice(nonrep, min(n_sample, nonrep.size), replace=False)).astype(np.int32)
+        if per_tile:
+            rows = np.setdiff1d(tile_rows(rng, cfg.T, 2 * n_sample), R_lab).astype(np.int32)
+        else:
+            rows = np.sort(rng.choice(nonrep, min(n_sample, nonrep.size), replace=False)).astype(np.int32)
         ref = oracle.cascade_step(X64, cfg.tau, R_lab, only_rows=rows)
         assert np.max(np.abs(out.gamma_cross.cpu().numpy()[0][rows] - ref.gamma_cross[rows])) <= tol
         g_rep_tok = np.zeros(cfg.T)
@@ -167,9 +171,86 @@ def test_config4_opt_shaped_full_size_sampled(ada, engine):
     sampled_large(ada, wl.CONFIGS[4], n_layers=3, engine=engine)
 
 
-@pytest.mark.parametrize("T,q", [(512, 0.01), (1024, 0.5), (4096, 0.05), (16384, 0.01), (16384, 0.2)])
+def elementwise_transition(ada, cfg, engine=0, causal=False):
+    """Layer 0 -> layer 1 of `cfg` against the oracle in full: every gamma of the full selection,
+    every gamma_rep and gamma_cross of the cascade step, sets and lists (both sides start the
+    step from the oracle's set)."""
+    from parity import check_cascade, check_full
+    ctx = ada.ada_create(cfg.B, cfg.T, cfg.d, ada.ADA_BF16)
+    ada.ada_set_engine(ctx, engine)
+    band = 0
+    R = None
+    for lb in wl.generate_layers(cfg, seed=0, n_layers=2):
+        if lb.layer == 0:
+            b0, R = check_full(ctx, lb.X, cfg.tau)
+            band += b0
+            assert b0 == 0      # the workloads keep every gamma far from the threshold
+            for b in range(cfg.B):
+                assert R[b].tolist() == full_from_labels(lb.labels[b]).tolist()
+        else:
+            b1, _, _ = check_cascade(ctx, lb.X, cfg.tau, R, causal=causal)
+            band += b1
+    assert ada.ada_device_status(ctx)[0] == 0
+    ada.ada_destroy(ctx)
+    return band
+
+
+@pytest.mark.parametrize("engine", [0, 3])
+def test_config4_opt_shaped_full_size_elementwise(ada, engine):
+    """configs[3] at full size (T = 8192, d = 4096): one full selection and one cascade step,
+    all 8192 gamma / gamma_rep / gamma_cross values and every list against the oracle."""
+    assert elementwise_transition(ada, wl.CONFIGS[4], engine=engine) == 0
+
+
+def test_config4_late_layer_cascade_step_elementwise(ada):
+    """A cascade step of configs[3] with a late layer's large inherited set (three rounds of
+    tiles on the pair kernel): the inherited set comes from the label-level replay of the
+    chain (no Gram), the step itself is compared with the oracle element by element."""
+    from parity import check_cascade
+    cfg = wl.CONFIGS[4]
+    n_layers = 24
+    R = None
+    for lb in wl.generate_layers(cfg, seed=0, n_layers=n_layers):
+        if lb.layer == 0:
+            R = full_from_labels(lb.labels[0])
+        elif lb.layer < n_layers - 1:
+            R = cascade_from_labels(lb.labels[0], R)[0]
+        else:
+            assert len(R) > 1024
+            ctx = ada.ada_create(1, cfg.T, cfg.d, ada.ADA_BF16)
+            band, rep, _ = check_cascade(ctx, lb.X, cfg.tau, [R])
+            assert band == 0
+            assert rep[0].tolist() == cascade_from_labels(lb.labels[0], R)[0].tolist()
+            assert ada.ada_device_status(ctx)[0] == 0
+            ada.ada_destroy(ctx)
+
+
+def tile_rows(rng, T, n_sample, tile=128):
+    """At least n_sample distinct rows, at least one from every `tile`-row block."""
+    n_tiles = (T + tile - 1) // tile
+    per = max(1, -(-n_sample // n_tiles))
+    rows = []
+    for i in range(n_tiles):
+        lo, hi = i * tile, min(T, (i + 1) * tile)
+        rows.extend(rng.choice(np.arange(lo, hi), min(per, hi - lo), replace=False).tolist())
+    return np.sort(np.asarray(rows, dtype=np.int32))
+
+
+# configs[4], the crossover sweep: every (T, r/T) point.  The oracle does whole layers up to
+# T = 8192 and at the two extreme points of T = 16384; the two middle points of T = 16384 are
+# checked by the label-level replay (sets) and the oracle on 512 rows, every 128-row tile hit.
+SWEEP_FULL = [(T, q) for T in wl.SWEEP_T for q in wl.SWEEP_Q if T <= 8192 or q in (0.01, 0.5)]
+SWEEP_SAMPLED = [(T, q) for T in wl.SWEEP_T for q in wl.SWEEP_Q if (T, q) not in SWEEP_FULL]
+
+
+@pytest.mark.parametrize("T,q", SWEEP_FULL)
+def test_sweep_points_elementwise(ada, T, q):
+    assert elementwise_transition(ada, wl.sweep_config(T, q)) == 0
+
+
+@pytest.mark.parametrize("T,q", SWEEP_SAMPLED)
 def test_sweep_points_sampled(ada, T, q):
-    sampled_large(ada, wl.sweep_config(T, q), n_layers=2, n_sample=24)
+    sampled_large(ada, wl.sweep_config(T, q), n_layers=2, n_sample=512, per_tile=True)
 
 
 def test_threshold_band_adversarial(ada):
@@ -269,6 +350,19 @@ def test_error_paths(ada):
     with pytest.raises(ada.AdaError) as e:                      # unknown flag bit
         ada.ada_cascade_step(ctx, X, TAU, idx, cnt, flags=4)
     assert e.value.status == 1
+    # host-buffer calls: storage type and alignment are checked before anything is copied
+    hx = torch.randn(1, 64, 32).pin_memory()
+    hi, hc = torch.empty(1, 64, dtype=torch.int32), torch.empty(1, dtype=torch.int32)
+    with pytest.raises(ada.AdaError) as e:
+        ada.ada_select_full_host(ctx, hx.bfloat16(), TAU, hi, hc)
+    assert e.value.status == 2
+    with pytest.raises(ada.AdaError) as e:
+        ada.ada_cascade_step_host(ctx, hx.bfloat16(), TAU, hi, hc, hi.clone(), hc.clone(), hi.clone(),
+                                  hc.clone(), hi.clone(), hc.clone())
+    assert e.value.status == 2
+    with pytest.raises(ada.AdaError) as e:
+        ada.ada_select_full_host(ctx, torch.randn(1, 64, 30), TAU, hi, hc)
+    assert e.value.status == 2
     # device-detected: unsorted inherited list, count out of range, NaN
     bad = torch.tensor([[3, 2] + [0] * 62], dtype=torch.int32, device="cuda")
     ada.ada_cascade_step(ctx, X, TAU, bad, torch.tensor([2], dtype=torch.int32, device="cuda"))

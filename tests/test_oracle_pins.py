@@ -345,7 +345,9 @@ def test_invariants_and_label_prediction(causal):
         # full selection: reps pairwise separated
         Gr = G[np.ix_(st["full"], st["full"])]
         assert np.all(Gr[np.tril_indices(st["full"].size, -1)] < thr)
-    assert causal or n_missed >= 0
+    # without the causal restriction the superset property of Proposition 3 does not hold: on this
+    # workload a later inherited representative shadows earlier tokens of its cluster
+    assert (n_missed == 0) if causal else (n_missed > 0)
 
 
 def test_unchanged_layer_keeps_inherited_set():
