@@ -32,17 +32,20 @@ from paper_2605_03110_b200 import workloads as wl  # noqa: E402
 METRIC = "selection tokens*layers/s (full at layer 0 + cascade at layers 1..L-1)"
 UNIT = "tokens*layers/s"
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant
-# kernel, from the ncu captures summarised under profiles/ (None until captured).
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant kernel.
+# These are NOT measured by this program: they are the figures of earlier `ncu` captures of the
+# same kernel on the same workload (one launch each), printed as `traffic_static` with their
+# origin beside them.  Keyed by (kernel, workload).
 NCU_TRAFFIC_BYTES = {
-    # fused cascade launch on configs[3]: mean of the captured layers 1 (76.9 MB) and 30 (108.4 MB),
-    # profiles/gram_tc2_cascade_cfg4.md
+    # fused cascade launch on configs[3]: mean of the captured layers 1 (76.9 MB) and 30 (108.4 MB)
     ("gram_tc_cascade", 4): 92.65e6,
-    # fused cascade launches of layers 1-2 on the smaller workloads, profiles/gram_tc_traffic_cfg1-3.md
+    # fused cascade launches of layers 1-2 on the smaller workloads
     ("gram_tc_cascade", 1): 9.53e6,
     ("gram_tc_cascade", 2): 28.9e6,
     ("gram_tc_cascade", 3): 21.08e6,
 }
+NCU_TRAFFIC_SOURCE = ("static: mean DRAM read+write bytes per launch from earlier ncu captures of this "
+                      "kernel on this workload (summaries under profiles/), not measured in this run")
 
 
 def measured_peaks():
@@ -131,9 +134,11 @@ def reference_arm(args, cfg):
 
     for _ in range(args.ref_warmup):
         one_step()
-    est = []
+    est, wall = [], []
     for _ in range(args.steps):
+        t0 = time.perf_counter()
         t_full, t_casc = one_step()
+        wall.append(time.perf_counter() - t0)
         est.append(t_full + (cfg.L - 1) * t_casc)      # scaled to the L-layer pipeline
     t_step = float(np.mean(est))
     value = cfg.B * cfg.T * cfg.L / t_step
@@ -148,6 +153,11 @@ def reference_arm(args, cfg):
                          "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
+        # ms_per_step is NOT the wall time of a step of this run: only `layers_computed` of the L
+        # layers are computed, the rest is scaled from the mean cascade step (a lower bound of the
+        # oracle's cost where the representative set grows over the layers)
+        "extrapolated": n_lay < cfg.L, "layers_computed": n_lay, "layers": cfg.L,
+        "wall_s_per_step": float(np.mean(wall)),
     }
     print(json.dumps(line))
 
@@ -246,6 +256,73 @@ def sweep(args):
           f"{peaks['bf16_sustained']} sustained")
 
 
+def hbm_point(ada, dev, T, q, peaks, args):
+    """One HBM-bound point of the crossover sweep (d = 4096, bf16, few representatives): the
+    cascade step on X1 from R(X0).  Reports the fused Gram launch (CUDA events around the launch,
+    L2 flushed by a 256 MiB write before every call) and the whole ada_cascade_step call (graph
+    replays of [flush, call], the flush-only graph subtracted) against the copy bandwidth, with
+    T*d*2 bytes (every row of X once) as the algorithmic traffic."""
+    import torch
+    cfg = wl.sweep_config(T, q)
+    X0, X1 = [torch.from_numpy(lb.X.view(np.int16)).view(torch.bfloat16).to(dev)
+              for lb in wl.generate_layers(cfg, seed=0)]
+    ctx = ada.ada_create(1, T, cfg.d, ada.ADA_BF16, device=dev.index or 0)
+    idx, cnt, _ = ada.ada_select_full(ctx, X0, cfg.tau, want_gamma=False)
+    out = ada.CascadeOut(1, T, dev, want_gamma=False)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    ada.ada_cascade_step(ctx, X1, cfg.tau, idx, cnt, out=out)          # first-call set-up
+    torch.cuda.synchronize()
+    r = int(cnt[0])
+    n = 10
+    ada.ada_profile_enable(ctx, True)
+    for _ in range(n):
+        flush.zero_()
+        ada.ada_cascade_step(ctx, X1, cfg.tau, idx, cnt, out=out)
+    torch.cuda.synchronize()
+    prof = {k: v for k, v in ada.ada_profile_read(ctx).items() if v[0]}
+    ada.ada_profile_enable(ctx, False)
+    k_gram = max(prof, key=lambda k: prof[k][1])
+    us_launch = prof[k_gram][1] * 1e3 / prof[k_gram][0]
+    # whole call, from graph replays
+    side = torch.cuda.Stream()
+
+    def graph_of(fn):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                for _ in range(n):
+                    flush.zero_()
+                    fn(side)
+        return g
+
+    def time_graph(g):
+        for _ in range(2):
+            g.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(5):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / (5 * n)
+
+    us_flush = time_graph(graph_of(lambda st: None))
+    us_call = time_graph(graph_of(lambda st: ada.ada_cascade_step(ctx, X1, cfg.tau, idx, cnt, out=out,
+                                                                  stream=st))) - us_flush
+    st_, _ = ada.ada_device_status(ctx)
+    assert st_ == 0
+    ada.ada_destroy(ctx)
+    nbytes = T * cfg.d * 2
+    gbs_launch, gbs_call = nbytes / us_launch / 1e3, nbytes / us_call / 1e3
+    return {"workload": f"configs[4] sweep point T={T}, r/T={q:g} (r={r}), d={cfg.d}, bf16", "kernel": k_gram,
+            "bound": "hbm", "algorithmic_bytes_per_launch": nbytes, "kernels_per_call": {k: v[0] // n for k, v in prof.items()},
+            "launch_us": us_launch, "achieved": gbs_launch, "unit": "GB/s", "peak": peaks["hbm_gbs"],
+            "frac": gbs_launch / peaks["hbm_gbs"], "peak_source": f"copy bandwidth, {peaks['src']}",
+            "whole_call_us": us_call, "whole_call_gbs": gbs_call, "whole_call_frac": gbs_call / peaks["hbm_gbs"],
+            "l2": "256 MiB write before every call"}
+
+
 def heads_bench(args, cfg):
     """Per-head selection (Section 8.5) on the layers of `cfg` read as (T, h, d/h): the whole
     L-layer cascade pipeline with one representative set per head, beside the shared-set pipeline
@@ -341,6 +418,9 @@ def main():
     ap.add_argument("--ref-warmup", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the >= 1 s replay loop")
+    ap.add_argument("--no-hbm-points", action="store_true",
+                    help="skip the two HBM-bound cross-Gram points (sweep, r/T = 0.01)")
     ap.add_argument("--sweep", action="store_true",
                     help="crossover sweep (configs[4]): full selection vs one cascade step per (T, r/T); "
                          "prints a table instead of the JSON line")
@@ -563,7 +643,50 @@ def main():
                 "frac": achieved / peak, "peak_source": peak_note,
                 "algorithmic_per_launch": per,
                 "avg_launch_ms": kernels[dom]["ms_per_step"] / kernels[dom]["launches"],
-                "traffic": NCU_TRAFFIC_BYTES.get((dom, cfg.cfg_id))}
+                "traffic": NCU_TRAFFIC_BYTES.get((dom, cfg.cfg_id)),
+                "traffic_source": NCU_TRAFFIC_SOURCE if (dom, cfg.cfg_id) in NCU_TRAFFIC_BYTES else None}
+    if bound == "tensor" and cfg.dtype == "bf16":
+        roofline["frac_sustained"] = achieved / peaks["bf16_sustained"]
+        roofline["frac_burst"] = achieved / peaks["bf16_burst"]
+
+    # ---- sustained: the same graph replayed for at least a second (a 1 kW part settles to lower
+    # clocks under load; the K-step figure above is the short-run one) ----
+    sustained = None
+    if not args.no_sustained:
+        n_sus = max(args.steps, int(np.ceil(1100.0 / ms_step)))
+        ms_sus, clk_sus = timed(step_fn, n_sus, 1)
+        sustained = {"ms_per_step": ms_sus, "steps": n_sus,
+                     "value": replicas.whole_job_throughput(rep, B * T * L, ms_sus * 1e-3), "unit": UNIT,
+                     "clocks": clk_sus,
+                     "ms_x_sm_mhz": (ms_sus * clk_sus["sm_mhz"]) if clk_sus.get("sm_mhz") else None}
+
+    # ---- the full-selection Gram on this workload (Definition 1 at every layer), per launch ----
+    roofline_full = None
+    ada.ada_profile_enable(ctx, True)
+    for _ in range(n_prof):
+        torch.cuda._sleep(int(2.0e7))
+        independent_pipeline()
+        torch.cuda.synchronize()
+    prof_i = {k: v for k, v in ada.ada_profile_read(ctx).items() if v[0] and "tri" in k}
+    ada.ada_profile_enable(ctx, False)
+    if prof_i:
+        k_full = max(prof_i, key=lambda k: prof_i[k][1])
+        n_l, ms_l = prof_i[k_full]
+        secs_full = ms_l * 1e-3 / n_l
+        ach = flops["tri_full"] / secs_full / 1e12
+        roofline_full = {"kernel": k_full, "bound": "tensor" if "tc" in k_full else "alu",
+                         "algorithmic_per_launch": "d*T*(T-1) flop per launch (lower triangle)",
+                         "avg_launch_ms": secs_full * 1e3, "achieved": ach, "unit": "TFLOP/s"}
+        if cfg.dtype == "bf16" and "tc" in k_full:
+            roofline_full.update({"peak_burst": peaks["bf16_burst"], "peak_sustained": peaks["bf16_sustained"],
+                                  "frac_burst": ach / peaks["bf16_burst"],
+                                  "frac_sustained": ach / peaks["bf16_sustained"],
+                                  "peak_source": f"cuBLAS bf16, {peaks['src']}"})
+
+    # ---- cross-Gram where it is HBM-bound: the r/T = 0.01 points of the crossover sweep ----
+    roofline_cross_hbm = None
+    if cfg.cfg_id == 4 and not args.no_hbm_points and rank == 0:
+        roofline_cross_hbm = [hbm_point(ada, dev, Tq, 0.01, peaks, args) for Tq in (16384, 8192)]
 
     # ---- set statistics: consecutive-layer Jaccard (independent) and cascade-vs-full Jaccard ----
     keep = []
@@ -672,7 +795,9 @@ def main():
             "data": "synthetic", "config": workload_dict(cfg), "clocks": clocks, "e2e": e2e,
             "warm_l2_ms_per_step": ms_warm,
             "gpu_launches": args.steps * sum(k["launches"] for k in kernels.values()),
-            "roofline": roofline, "cpu_baseline": cpu_baseline,
+            "roofline": roofline, "roofline_full": roofline_full,
+            "roofline_cross_hbm": roofline_cross_hbm, "sustained": sustained,
+            "cpu_baseline": cpu_baseline,
             "independent": {"value": world * B * T * L / (ms_indep * 1e-3), "unit": UNIT,
                             "ms_per_step": ms_indep},
             "cascade_speedup": ms_indep / ms_step,
