@@ -59,17 +59,19 @@ bool use_split(const ada_ctx* ctx, ada_dtype dt) {
            gram_tc_available();
 }
 
+// the pair-CTA form of the tensor-core kernel, or the one-CTA form?
+bool use_pair(const ada_ctx* ctx, int64_t B, int64_t T, int64_t d) {
+    if (ctx->engine == ADA_ENGINE_TCGEN05_PAIR) return true;
+    // The pair kernel pays off once there are several 256-row tiles per SM pair and a long
+    // contraction; small problems are covered better by the finer one-CTA tiles.
+    return ctx->engine == ADA_ENGINE_AUTO && B * T >= 8192 && d >= 2048;
+}
+
 // tensor-core launch of one or two segments, in the one-CTA or the pair-CTA form
 cudaError_t launch_tc(ada_ctx* ctx, const GramProblem* tri, const GramProblem* cross,
                       const NormJob* norms, cudaStream_t s) {
-    bool pair = ctx->engine == ADA_ENGINE_TCGEN05_PAIR;
-    if (ctx->engine == ADA_ENGINE_AUTO) {
-        // The pair kernel pays off once there are several 256-row tiles per SM pair and a long
-        // contraction; small problems are covered better by the finer one-CTA tiles.
-        const GramProblem* p = cross != nullptr ? cross : tri;
-        pair = (int64_t)p->B * p->rows >= 8192 && p->d >= 2048;
-    }
-    if (pair) return launch_gram_tc2(ctx, tri, cross, norms, s);
+    const GramProblem* p = cross != nullptr ? cross : tri;
+    if (use_pair(ctx, p->B, p->rows, p->d)) return launch_gram_tc2(ctx, tri, cross, norms, nullptr, s);
     return launch_gram_tc(ctx, tri, cross, norms, s);
 }
 
@@ -285,6 +287,7 @@ static ada_status select_full_impl(ada_ctx* ctx, const void* X, int64_t B, int64
                               nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, s));
     NormJob nj;
     nj.X = X; nj.ldx = ldx; nj.n_rows = B * T; nj.d = (int)d; nj.inv_norm = ctx->inv_norm;
+    nj.batch = 0; nj.rows_per_seq = 0;
     GramProblem p;
     memset(&p, 0, sizeof(p));
     p.A = X; p.Bm = X;
@@ -354,20 +357,34 @@ static ada_status cascade_impl(ada_ctx* ctx, const void* X, int64_t B, int64_t T
     const bool adaptive = tau_upd.tau_state != nullptr;
     if (adaptive) CU(launch_tau_thr(ctx, (int)B, tau_upd.tau_state, s));   // thresholds of this step
 
-    // role map, gamma scratch and dependency counter are zero on entry (workspace invariant
+    // role map, gamma scratch and dependency counters are zero on entry (workspace invariant
     // kept by the compaction kernels).
-    // lines 1-2: inverse norms of all rows; inherited list validated, scattered into the role
-    // map and its rows gathered into Xrep
-    // tensor cores: one launch does lines 3-8; for long K it also computes line 1's row norms
     const bool split = use_split(ctx, dt);
-    const bool fuse = use_tc(ctx, dt) || split,
-               fuse_norm = !split && fuse && d >= 2048 && B * T >= 4096 && xb == T * ldx;
-    CU(launch_norm_gather(ctx, X, (int)B, (int)T, (int)d, ldx, xb, dt,
-                          (fuse_norm || split) ? nullptr : ctx->inv_norm,
-                          nullptr, rep_in, rep_in_cnt, ctx->role, ctx->r_eff, ctx->Xrep,
-                          ctx->inv_rep, s));
+    const bool fuse = use_tc(ctx, dt) || split;
+    // bf16 on the pair kernel: ONE Gram launch does lines 1-8.  Its helper warps validate the
+    // inherited list, scatter the role map and gather the rows (lines 1-2); the r x r tiles
+    // (lines 3-5) and the cross tiles (lines 6-8) follow; the norms of X come out of the cross
+    // tiles while they sit in shared memory, and the row's own factor 1/||x_t|| is left to the
+    // compaction.
+    const bool inl = fuse && !split && use_pair(ctx, B, T, d);
+    // otherwise lines 1-2 are a launch of their own: inverse norms of all rows, inherited list
+    // validated, scattered into the role map and its rows gathered into Xrep; for long K the
+    // one-CTA tensor-core launch computes line 1's row norms itself
+    const bool fuse_norm = !inl && !split && fuse && d >= 2048 && B * T >= 4096 && xb == T * ldx;
+    if (!inl)
+        CU(launch_norm_gather(ctx, X, (int)B, (int)T, (int)d, ldx, xb, dt,
+                              (fuse_norm || split) ? nullptr : ctx->inv_norm,
+                              nullptr, rep_in, rep_in_cnt, ctx->role, ctx->r_eff, ctx->Xrep,
+                              ctx->inv_rep, s));
     NormJob nj;
     nj.X = X; nj.ldx = ldx; nj.n_rows = B * T; nj.d = (int)d; nj.inv_norm = ctx->inv_norm;
+    nj.batch = 0; nj.rows_per_seq = 0;
+    GatherJob gj;
+    memset(&gj, 0, sizeof(gj));
+    gj.X = X; gj.ldx = ldx; gj.xb = xb;
+    gj.rep_in = rep_in; gj.rep_in_cnt = rep_in_cnt;
+    gj.role = ctx->role; gj.r_eff = ctx->r_eff; gj.Xrep = ctx->Xrep; gj.inv_rep = ctx->inv_rep;
+    gj.T = (int)T; gj.d = (int)d; gj.B = (int)B;
     if (split)   // 1/||x|| of all rows; bf16 terms of X and of the gathered rows
         CU(launch_split(ctx, X, (int)B, (int)T, (int)d, ldx, xb, true, s));
     // lines 3-4: r x r Gram among inherited reps, max over earlier ones
@@ -378,7 +395,8 @@ static ada_status cascade_impl(ada_ctx* ctx, const void* X, int64_t B, int64_t T
     p.a_batch = T * d; p.b_batch = T * d;
     p.inv_a = ctx->inv_rep; p.inv_b = ctx->inv_rep;
     p.out = ctx->g_rep;
-    p.n_dev = ctx->r_eff; p.n_host = 0;
+    p.n_dev = inl ? rep_in_cnt : ctx->r_eff; p.n_host = 0;
+    p.n_clamp = inl ? 1 : 0;
     p.rows = (int)T; p.cap = (int)T; p.d = (int)d; p.B = (int)B;
     p.tri = 1;
     if (!fuse) CU(run_gram(ctx, p, dt, s));
@@ -390,7 +408,8 @@ static ada_status cascade_impl(ada_ctx* ctx, const void* X, int64_t B, int64_t T
     q.a_batch = xb; q.b_batch = T * d;
     q.inv_a = ctx->inv_norm; q.inv_b = ctx->inv_rep;
     q.out = ctx->g_tok;
-    q.n_dev = ctx->r_eff; q.n_host = 0;
+    q.n_dev = p.n_dev; q.n_host = 0;
+    q.n_clamp = p.n_clamp;
     q.rows = (int)T; q.cap = (int)T; q.d = (int)d; q.B = (int)B;
     q.tri = 0;
     q.col_gate = ctx->g_rep;
@@ -401,6 +420,12 @@ static ada_status cascade_impl(ada_ctx* ctx, const void* X, int64_t B, int64_t T
     q.row_role = ctx->role;
     q.causal = (flags & ADA_CROSS_CAUSAL) ? 1 : 0;
     q.wait_norm_a = fuse_norm ? 1 : 0;
+    if (inl) {
+        q.defer_row = 1;
+        q.inv_out = ctx->inv_norm;
+        q.hb_rows = gram_tc2_hb_rows(ctx, (int)B, (int)T);
+        if (q.hb_rows == 0) return ADA_ERR_CUDA;
+    }
     if (split) {
         p.A = ctx->splitRA; p.Bm = ctx->splitRB;
         q.A = ctx->splitXA; q.Bm = ctx->splitRB;
@@ -408,11 +433,12 @@ static ada_status cascade_impl(ada_ctx* ctx, const void* X, int64_t B, int64_t T
         p.a_batch = p.b_batch = q.a_batch = q.b_batch = T * 6 * d;
         p.d = q.d = (int)(6 * d);
     }
-    if (fuse) CU(launch_tc(ctx, &p, &q, fuse_norm ? &nj : nullptr, s));
+    if (inl) CU(launch_gram_tc2(ctx, &p, &q, nullptr, &gj, s));
+    else if (fuse) CU(launch_tc(ctx, &p, &q, fuse_norm ? &nj : nullptr, s));
     else CU(run_gram(ctx, q, dt, s));
     // lines 5, 9, 10-11
     CU(launch_compact_cascade(ctx, (int)B, (int)T, thr, rep_out, rep_out_cnt, add_idx, add_cnt,
-                              rem_idx, rem_cnt, gamma_rep, gamma_cross, tau_upd, s));
+                              rem_idx, rem_cnt, gamma_rep, gamma_cross, tau_upd, inl, s));
     return ADA_OK;
 }
 

@@ -72,6 +72,35 @@ struct GramProblem {
     // nearest-representative mode (cross only): instead of `out`, combine per row the packed
     // key (value bits << 32 | ~column) with a 64-bit atomicMax: largest value, lowest column
     unsigned long long* out_arg;
+    // n_dev holds the caller's raw counts: clamp them to [0, cap] (nobody has sanitised them yet)
+    int n_clamp;
+    // pair kernel, cross only -----------------------------------------------------------------
+    // out[] receives the row maximum WITHOUT the factor inv_a[i] (a positive factor common to the
+    // row commutes with the maximum, rounding included); the compaction applies it.  No row
+    // norm is then needed inside the launch.
+    int defer_row;
+    // 1/||a_i|| of every row of A, computed from the A tiles while they sit in shared memory (by
+    // the tiles of the first column tile) and stored here; NULL: not wanted
+    float* inv_out;
+    // rows of A per CTA when a single column tile covers every sequence's columns (a cross-Gram
+    // bound by streaming A once: shorter row tiles put every SM pair to work); 0 or 128: 128
+    int hb_rows;
+};
+
+// Algorithm 1 lines 1-2 inside a pair-kernel launch: the inherited list is validated, scattered
+// into the role map, and its rows of X are copied (raw) to Xrep with their inverse norms, by
+// spare warps of every CTA before the first tile; loads of Xrep and the epilogues wait for it.
+// X == NULL: nothing to do.
+struct GatherJob {
+    const void* X;            // bf16 rows
+    int64_t ldx, xb;          // row / sequence strides of X in elements
+    const int32_t* rep_in;    // [B*T]
+    const int32_t* rep_in_cnt;// [B]
+    int32_t* role;            // [B*T] position + 1 of inherited tokens
+    int32_t* r_eff;           // [B] sanitised counts
+    void* Xrep;               // [B*T][d]
+    float* inv_rep;           // [B*T] by position
+    int T, d, B;
 };
 
 // Row norms computed inside a tensor-core Gram launch by four extra warps per CTA
@@ -83,6 +112,10 @@ struct NormJob {
     int64_t n_rows;
     int d;
     float* inv_norm;
+    // rows_per_seq > 0: row i is row (i % rows_per_seq) of sequence (i / rows_per_seq), which
+    // starts `batch` elements after the previous one; 0: rows are ldx apart throughout
+    int64_t batch;
+    int rows_per_seq;
 };
 
 struct Profiler {
@@ -194,10 +227,12 @@ struct TauUpdate {
     double target, gain, tau_min, tau_max;
 };
 cudaError_t launch_tau_thr(ada_ctx* ctx, int B, const double* tau_state, cudaStream_t s);
+// row_scale: the cross maxima in the scratch still lack the factor 1/||x_t|| (GramProblem::defer_row)
 cudaError_t launch_compact_cascade(ada_ctx* ctx, int B, int T, float thr, int32_t* rep_out,
                                    int32_t* rep_out_cnt, int32_t* add_idx, int32_t* add_cnt,
                                    int32_t* rem_idx, int32_t* rem_cnt, float* gamma_rep,
-                                   float* gamma_cross, const TauUpdate& tu, cudaStream_t s);
+                                   float* gamma_cross, const TauUpdate& tu, bool row_scale,
+                                   cudaStream_t s);
 
 // gram_ffma.cu
 cudaError_t launch_gram_ffma(ada_ctx* ctx, const GramProblem& p, ada_dtype dt, cudaStream_t s);
@@ -210,6 +245,8 @@ cudaError_t launch_selftest_wait(ada_ctx* ctx, int limit_ms, cudaStream_t s);
 
 // gram_tc2.cu (bf16, tcgen05.cta_group::2: two CTAs per 256-row tile)
 cudaError_t launch_gram_tc2(ada_ctx* ctx, const GramProblem* tri, const GramProblem* cross,
-                            const NormJob* norms, cudaStream_t s);
+                            const NormJob* norms, const GatherJob* gather, cudaStream_t s);
+// rows of the left operand per CTA for a cross-Gram that a single column tile covers
+int gram_tc2_hb_rows(ada_ctx* ctx, int B, int T);
 
 }  // namespace ada

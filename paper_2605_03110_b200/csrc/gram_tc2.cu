@@ -15,6 +15,16 @@
 //               tcgen05.commit multicast to both CTAs.  Both CTAs: TMEM allocation
 //   warps 2..5  epilogue in both CTAs, each on its own 128 rows; the peer's epilogue
 //               returns the accumulator by a remote arrive on the leader's mbarrier
+//   warps 6..13 helpers.  Full selection: 1/||x_t|| of every row with plain loads, behind the
+//               main loops.  Cascade step: first the gather of Algorithm 1 lines 1-2 (list
+//               checked, role map, rows copied to Xrep with their inverse norms; loads of Xrep
+//               and the epilogues wait for it), then warps 6..9 take the row norms of X out of
+//               the left-operand tiles while those sit in shared memory (tiles of the first
+//               column tile only; one thread per row), so X is read from memory exactly once
+// The cross segment's row maxima are published WITHOUT the factor 1/||x_t|| (it commutes with
+// the maximum; the compaction applies it), so no epilogue waits for a norm.  When one column
+// tile covers all representatives the step is bound by streaming X once: the row tiles are
+// then cut shorter than 128 rows per CTA so that every SM pair streams a share.
 // Every wait is bounded; the two CTAs meet at a cluster barrier before either frees TMEM
 // or exits.
 #include "gram_tc_dev.cuh"
@@ -22,6 +32,14 @@
 namespace ada {
 
 using namespace tc;
+
+// Time stamps for in-kernel timelines (development builds only: -DADA_TRACE).
+#ifdef ADA_TRACE
+__device__ unsigned long long g_trace[160 * 64];
+#define TRACE(slot) do { g_trace[blockIdx.x * 64 + (slot)] = tc::global_ns(); } while (0)
+#else
+#define TRACE(slot) do { } while (0)
+#endif
 
 namespace {
 
@@ -93,39 +111,43 @@ __device__ __forceinline__ unsigned instr_desc_pair(int n) {
 
 // ---------------------------------------------------------------- tile list (256-row tiles)
 __device__ __forceinline__ int seq_n(const GramProblem& p, int b) {
-    return p.n_dev != nullptr ? p.n_dev[b] : p.n_host;
+    int n = p.n_dev != nullptr ? p.n_dev[b] : p.n_host;
+    if (p.n_clamp) n = min(max(n, 0), p.cap);
+    return n;
 }
 __device__ __forceinline__ int tri_tiles(int n) {           // row pair P needs column tiles 0..P
     const int M = (n + PM - 1) / PM;
     return M * (M + 1) / 2;
 }
-__device__ __forceinline__ void cross_cols(int n, int& nct, int& w) {
+// column tiles of a cross problem with n columns.  With in-launch norms (inv_out) a sequence
+// without columns still gets one (empty) column tile: its rows have to be read for their norms.
+__device__ __forceinline__ void cross_cols(const GramProblem& p, int n, int& nct, int& w) {
     nct = (n + BN - 1) / BN;
-    w = nct > 0 ? ((((n + nct - 1) / nct) + 31) & ~31) : 0;    // each CTA holds w/2 columns: keep w/2 a multiple of 16
+    if (nct == 0 && p.inv_out != nullptr && n == 0) nct = 1;
+    w = nct > 0 ? max(32, (((n + nct - 1) / nct) + 31) & ~31) : 0;    // each CTA holds w/2 columns: keep w/2 a multiple of 16
 }
-__device__ __forceinline__ int seg_tiles(const GramProblem& p) {
+// hrows: rows of the left operand per CTA in cross tiles (128, or fewer in the streaming form)
+__device__ __forceinline__ int seg_tiles(const GramProblem& p, int hrows) {
     int total = 0;
     for (int b = 0; b < p.B; ++b) {
         const int n = seq_n(p, b);
-        if (n <= 0) continue;
-        if (p.tri) total += tri_tiles(n);
+        if (p.tri) { if (n > 0) total += tri_tiles(n); }
         else {
             int nct, w;
-            cross_cols(n, nct, w);
-            total += ((p.rows + PM - 1) / PM) * nct;
+            cross_cols(p, n, nct, w);
+            total += ((p.rows + 2 * hrows - 1) / (2 * hrows)) * nct;
         }
     }
     return total;
 }
-__device__ __forceinline__ bool decode_tile(const GramProblem& p, int id, Piece& t) {
+__device__ __forceinline__ bool decode_tile(const GramProblem& p, int hrows, int id, Piece& t) {
     for (int b = 0; b < p.B; ++b) {
         const int n = seq_n(p, b);
-        if (n <= 0) continue;
-        int cnt, nct = 0, w = 0;
-        if (p.tri) cnt = tri_tiles(n);
+        int cnt = 0, nct = 0, w = 0;
+        if (p.tri) cnt = n > 0 ? tri_tiles(n) : 0;
         else {
-            cross_cols(n, nct, w);
-            cnt = ((p.rows + PM - 1) / PM) * nct;
+            cross_cols(p, n, nct, w);
+            cnt = ((p.rows + 2 * hrows - 1) / (2 * hrows)) * nct;
         }
         if (id >= cnt) { id -= cnt; continue; }
         t.b = b;
@@ -140,7 +162,7 @@ __device__ __forceinline__ bool decode_tile(const GramProblem& p, int id, Piece&
             t.m = n;
             nc = min(n - t.col0, BN);
         } else {
-            t.row0 = (id / nct) * PM;
+            t.row0 = (id / nct) * 2 * hrows;
             t.col0 = (id % nct) * w;
             t.m = p.rows;
             nc = min(n - t.col0, w);
@@ -150,38 +172,146 @@ __device__ __forceinline__ bool decode_tile(const GramProblem& p, int id, Piece&
     }
     return false;
 }
-// per-CTA stage: 128 rows of A and ncols/2 rows of B (in 64-row boxes)
-// bytes of one 64-element K block of a stage, and of the whole stage
-__device__ __forceinline__ int sub_bytes_pair(int ncols) {
-    return A_BYTES + (((ncols >> 1) + BOX_N - 1) / BOX_N) * BOX_BYTES;
+// per-CTA stage: the CTA's rows of A (a_bytes per 64-element K block, a multiple of 1024) and
+// ncols/2 rows of B (in 64-row boxes)
+__device__ __forceinline__ int a_bytes_of(int hrows) { return (hrows * 128 + 1023) & ~1023; }
+__device__ __forceinline__ int sub_bytes_pair(int a_bytes, int ncols) {
+    return a_bytes + (((ncols >> 1) + BOX_N - 1) / BOX_N) * BOX_BYTES;
 }
-__device__ __forceinline__ int stage_bytes_pair(int ncols) { return KSUB * sub_bytes_pair(ncols); }
-__device__ __forceinline__ int stage_count(int sbytes) {
-    return min(MAX_STAGES, RING_BYTES / sbytes);
+__device__ __forceinline__ int stage_count(int sbytes, int a_bytes) {
+    // the MMA reads 128 rows of A whatever was loaded: keep what it reads past a shorter tile
+    // inside the ring
+    return min(MAX_STAGES, (RING_BYTES - (A_BYTES - a_bytes)) / sbytes);
 }
 
+// Row norms of the cross segment's left operand (inv_out).  When one column tile covers all
+// columns every row tile is loaded exactly once and the launch is bound by streaming them: the
+// norms are then taken from the tiles in shared memory (`from_smem`; the stage release waits for
+// the readers, which costs nothing while the tensor pipe idles).  With several column tiles the
+// main loops are bound by the tensor pipe and by what an SM can draw from L2, a stage release
+// that waits for readers slows them, and the helper warps read the rows with plain loads
+// instead (X then stays resident in L2 between the column tiles anyway).
+__device__ __forceinline__ bool norm_duty(const GramProblem& p, const Piece& pc, bool from_smem) {
+    return from_smem && !p.tri && p.inv_out != nullptr && pc.col0 == 0;
+}
 // Under ADA_CROSS_CAUSAL a cross tile whose first (lowest) column token is not below the
 // tile's last row has no admissible (row, column) pair: every role skips it, so neither
-// its loads nor its MMAs are issued.  Column tokens ascend with the column index.
-__device__ __forceinline__ bool dead_tile(const GramProblem& p, const Piece& pc) {
-    if (p.tri || !p.causal || p.col_token == nullptr) return false;
-    return p.col_token[(int64_t)pc.b * p.cap + pc.col0] >= pc.row0 + PM;
+// its loads nor its MMAs are issued.  Column tokens ascend with the column index.  (A tile
+// that has to yield row norms is never skipped.)
+__device__ __forceinline__ bool dead_tile(const GramProblem& p, const Piece& pc, int hrows, bool from_smem) {
+    if (p.tri || !p.causal || p.col_token == nullptr || pc.n <= 0 || norm_duty(p, pc, from_smem)) return false;
+    return p.col_token[(int64_t)pc.b * p.cap + pc.col0] >= pc.row0 + 2 * hrows;
 }
 
 struct GramMaps {
     CUtensorMap a[2], b[2];
+    CUtensorMap ah;          // left operand of the cross segment in boxes of hb_rows rows
 };
 
+// bounded wait of ONE thread until a global counter reaches `target`
+__device__ __forceinline__ bool wait_counter_1(const unsigned* counter, unsigned target,
+                                               volatile int* abort_flag, int where) {
+    const unsigned long long t0 = global_ns();
+    unsigned seen;
+    while (true) {
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
+        if (seen >= target) return true;
+        if (*abort_flag != 0) return false;
+        if (global_ns() - t0 > WAIT_LIMIT_NS) { *abort_flag = where; return false; }
+        __nanosleep(64);
+    }
+}
+
+// Algorithm 1 lines 1-2, by the helper warps of every CTA (warp `g` of `nw`): entry i of
+// sequence b is checked (in range, strictly above entry i-1), role[token] = i + 1, the raw row
+// goes to Xrep[b, i] and its inverse norm to inv_rep[b, i]; a rejected entry gets inverse norm
+// 0 (its column then counts for nothing) and raises the status.  Ends with one arrival per warp
+// on `counter`.
+__device__ __forceinline__ void gather_rows(const GatherJob& gj, int g, int nw, int lane,
+                                            unsigned* counter, unsigned* status) {
+    const __nv_bfloat16* X = reinterpret_cast<const __nv_bfloat16*>(gj.X);
+    __nv_bfloat16* Xrep = reinterpret_cast<__nv_bfloat16*>(gj.Xrep);
+    const int nvec = gj.d >> 3;
+    int b = 0;
+    int64_t item = g;
+    while (b < gj.B) {
+        int cnt = gj.rep_in_cnt[b];
+        if (cnt < 0 || cnt > gj.T) {
+            if (g == 0 && lane == 0) atomicOr(status, ST_BAD_COUNT);
+            cnt = cnt < 0 ? 0 : gj.T;
+        }
+        if (g == 0 && lane == 0) gj.r_eff[b] = cnt;
+        if (item >= cnt) { item -= cnt; ++b; continue; }
+        const int i = (int)item;
+        item += nw;                                   // this warp's next entry (maybe in a later sequence)
+        const int32_t* list = gj.rep_in + (int64_t)b * gj.T;
+        const int32_t idx = list[i];
+        bool ok = idx >= 0 && idx < gj.T;
+        if (ok && i > 0) ok = list[i - 1] < idx;
+        const int64_t prow = (int64_t)b * gj.T + i;
+        if (!ok) {
+            if (lane == 0) { atomicOr(status, ST_BAD_INDEX); gj.inv_rep[prow] = 0.f; }
+            continue;
+        }
+        const uint4* src = reinterpret_cast<const uint4*>(X + (int64_t)b * gj.xb + (int64_t)idx * gj.ldx);
+        uint4* dst = reinterpret_cast<uint4*>(Xrep + prow * (int64_t)gj.d);
+        float ss = 0.f;
+        int v = lane;
+        for (; v + 480 < nvec; v += 512) {            // sixteen loads in flight per lane
+            uint4 x[16];
+#pragma unroll
+            for (int q = 0; q < 16; ++q) x[q] = __ldg(src + v + 32 * q);
+#pragma unroll
+            for (int q = 0; q < 16; ++q) { ss += sumsq_bf16x8(x[q]); dst[v + 32 * q] = x[q]; }
+        }
+        for (; v < nvec; v += 32) {
+            const uint4 x = __ldg(src + v);
+            ss += sumsq_bf16x8(x);
+            dst[v] = x;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        if (lane == 0) {
+            gj.inv_rep[prow] = (ss <= 3.0e38f && ss > 0.f) ? 1.0f / sqrtf(ss) : 0.f;
+            gj.role[(int64_t)b * gj.T + idx] = i + 1;
+        }
+    }
+    // the rows just written are read by TMA (async proxy) from other CTAs
+    asm volatile("fence.proxy.async.global;" ::: "memory");
+    __threadfence();
+    __syncwarp();
+    if (lane == 0) atomicAdd(counter, 1u);
+}
+
 // ---------------------------------------------------------------- the kernel
+struct alignas(16) SharedPair {
+    unsigned long long full[MAX_STAGES];
+    unsigned long long empty[MAX_STAGES];
+    unsigned long long consumed[MAX_STAGES];   // MMAs of a norm-duty stage retired: its A tile may be read
+    unsigned long long tmem_full[2];
+    unsigned long long tmem_empty[2];
+    unsigned long long drain;
+    unsigned tmem_base;
+    int abort_flag;
+    int tiles0, tiles1, hrows, one_col_tile;
+    unsigned norm_cnt[MAX_STAGES];             // norm warps done with a stage
+    // per epilogue warp, so that staging needs no barrier across warps
+    alignas(16) float col_scale[4][BN];
+    alignas(16) int col_token[4][BN];
+};
+constexpr int SMEM_PAIR_BYTES = RING_BYTES + (int)sizeof(SharedPair) + 1024;
+static_assert(SMEM_PAIR_BYTES <= 227 * 1024, "shared memory budget");
+constexpr int SMEM_NORM_WARPS = 4;             // warps 6..9 read the A tiles
+
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramProblem seg0,
            const __grid_constant__ GramProblem seg1, const int nseg,
-          const __grid_constant__ NormJob norms, unsigned* __restrict__ dep_ctr,
-           unsigned* __restrict__ status) {
+           const __grid_constant__ NormJob norms, const __grid_constant__ GatherJob gather,
+           unsigned* __restrict__ dep_ctr, unsigned* __restrict__ status) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-    Shared& sh = *reinterpret_cast<Shared*>(smem + RING_BYTES);
+    SharedPair& sh = *reinterpret_cast<SharedPair*>(smem + RING_BYTES);
     volatile int* abort_flag = &sh.abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -192,6 +322,8 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
         for (int s = 0; s < MAX_STAGES; ++s) {
             mbar_init(&sh.full[s], 1);
             mbar_init(&sh.empty[s], 1);
+            mbar_init(&sh.consumed[s], 1);
+            sh.norm_cnt[s] = 0u;
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(&sh.tmem_full[a], 1);
@@ -210,9 +342,20 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
     }
     // everything above is local to the CTA; from here on the predecessor's results are read
     grid_dep_wait();
+    if (threadIdx.x == 0) TRACE(0);
     if (threadIdx.x == 64) {
-        sh.tiles0 = seg_tiles(seg0);
-        sh.tiles1 = nseg > 1 ? seg_tiles(seg1) : 0;
+        // streaming form: one column tile covers the columns of every sequence, so the launch is
+        // one pass over the rows of A and shorter row tiles put every pair to work
+        const GramProblem& cx = (nseg > 1) ? seg1 : seg0;
+        int hrows = BM;
+        bool one = !cx.tri;
+        if (one)
+            for (int b = 0; b < cx.B; ++b) one = one && seq_n(cx, b) <= BN;
+        if (one && cx.hb_rows > 0 && cx.hb_rows < BM) hrows = cx.hb_rows;
+        sh.hrows = hrows;
+        sh.one_col_tile = one ? 1 : 0;
+        sh.tiles0 = seg_tiles(seg0, hrows);
+        sh.tiles1 = nseg > 1 ? seg_tiles(seg1, hrows) : 0;
     }
     tcgen05_fence_before();
     __syncthreads();
@@ -220,7 +363,12 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
     tcgen05_fence_after();
     const unsigned tmem_base = sh.tmem_base;
     const int tiles0 = sh.tiles0, total = sh.tiles0 + sh.tiles1;
+    const int hrows = sh.hrows;                          // rows per CTA of a cross tile
+    const bool smem_norms = sh.one_col_tile != 0;        // row norms out of the tiles in shared memory
+    const unsigned gather_total = (unsigned)(gridDim.x * NORM_WARPS);
+    const bool has_gather = gather.X != nullptr;
     Piece pc;
+    if (threadIdx.x == 0) TRACE(1);
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer (both CTAs)
@@ -228,37 +376,48 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
             unsigned fills = 0, used = 0, ever = 0;
             int cur_sb = 0, cur_nst = 0, s = 0;
             bool ok = true;
+            // the right operand (and the triangle's left operand) is the gathered copy
+            if (has_gather && total > 0) {
+                ok = wait_counter_1(dep_ctr + 3, gather_total, abort_flag, 12);
+                asm volatile("fence.proxy.async.global;" ::: "memory");
+            }
+            TRACE(3);
             for (int id = pair; ok && id < total; id += npairs) {
                 const int sg = id < tiles0 ? 0 : 1;
                 const GramProblem& p = sg ? seg1 : seg0;
-                if (!decode_tile(p, id - (sg ? tiles0 : 0), pc)) break;
-                if (dead_tile(p, pc)) continue;   // causal cross tile with no admissible pair
+                if (!decode_tile(p, hrows, id - (sg ? tiles0 : 0), pc)) break;
+                if (dead_tile(p, pc, hrows, smem_norms)) continue;   // causal cross tile with no admissible pair
                 const int num_kb = (p.d + BKS - 1) / BKS;
                 const int half = pc.ncols >> 1;
                 const int nbox = (half + BOX_N - 1) / BOX_N;
-                const int sb = stage_bytes_pair(pc.ncols);
+                const int arows = p.tri ? BM : hrows;
+                const int a_bytes = a_bytes_of(arows);
+                const int subb = sub_bytes_pair(a_bytes, pc.ncols);
+                const int sb = KSUB * subb;
+                const unsigned tx = (unsigned)(KSUB * (arows * 128 + nbox * BOX_BYTES));
+                const CUtensorMap* amap = (!p.tri && hrows != BM) ? &maps.ah : &maps.a[sg];
                 if (sb != cur_sb) {
                     for (int q = 0; q < cur_nst && ok; ++q)
                         if ((used >> q) & 1u)
                             ok = mbar_wait(&sh.empty[q], ((fills >> q) & 1u) ^ 1u, abort_flag, 6);
                     if (!ok) break;
-                    cur_sb = sb; cur_nst = stage_count(sb); s = 0; used = 0;
+                    cur_sb = sb; cur_nst = stage_count(sb, a_bytes); s = 0; used = 0;
                 }
-                const int a_row = pc.row0 + (int)rank * BM;
+                const int a_row = pc.row0 + (int)rank * arows;
                 const int b_row = pc.col0 + (int)rank * half;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(&sh.empty[s], ((fills >> s) & 1u) ^ 1u, abort_flag, 1)) { ok = false; break; }
                     unsigned char* sa = smem + s * sb;
                     // the leader's barrier counts the bytes of both CTAs
-                    if (rank == 0) mbar_expect_tx(&sh.full[s], 2u * (unsigned)sb);
+                    if (rank == 0) mbar_expect_tx(&sh.full[s], 2u * tx);
                     // K blocks past d are zero-filled by the TMA unit
 #pragma unroll
                     for (int u = 0; u < KSUB; ++u) {
-                        unsigned char* su = sa + u * (sb / KSUB);
+                        unsigned char* su = sa + u * subb;
                         const int k0 = kb * BKS + u * BK;
-                        tma_load_3d_pair(&maps.a[sg], &sh.full[s], su, k0, a_row, pc.b);
+                        tma_load_3d_pair(amap, &sh.full[s], su, k0, a_row, pc.b);
                         for (int j = 0; j < nbox; ++j)
-                            tma_load_3d_pair(&maps.b[sg], &sh.full[s], su + A_BYTES + j * BOX_BYTES, k0,
+                            tma_load_3d_pair(&maps.b[sg], &sh.full[s], su + a_bytes + j * BOX_BYTES, k0,
                                              b_row + j * BOX_N, pc.b);
                     }
                     fills ^= 1u << s; used |= 1u << s; ever |= 1u << s;
@@ -284,11 +443,14 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
             for (int id = pair; ok && id < total; id += npairs) {
                 const int sg = id < tiles0 ? 0 : 1;
                 const GramProblem& p = sg ? seg1 : seg0;
-                if (!decode_tile(p, id - (sg ? tiles0 : 0), pc)) break;
-                if (dead_tile(p, pc)) continue;   // causal cross tile with no admissible pair
+                if (!decode_tile(p, hrows, id - (sg ? tiles0 : 0), pc)) break;
+                if (dead_tile(p, pc, hrows, smem_norms)) continue;   // causal cross tile with no admissible pair
                 const int num_kb = (p.d + BKS - 1) / BKS;
-                const int sb = stage_bytes_pair(pc.ncols);
-                if (sb != cur_sb) { cur_sb = sb; cur_nst = stage_count(sb); s = 0; }
+                const int a_bytes = a_bytes_of(p.tri ? BM : hrows);
+                const int subb = sub_bytes_pair(a_bytes, pc.ncols);
+                const int sb = KSUB * subb;
+                if (sb != cur_sb) { cur_sb = sb; cur_nst = stage_count(sb, a_bytes); s = 0; }
+                const bool duty = norm_duty(p, pc, smem_norms);
                 const unsigned acc = tile_it & 1u, acc_ph = (tile_it >> 1) & 1u;
                 ++tile_it;
                 if (!mbar_wait(&sh.tmem_empty[acc], acc_ph ^ 1u, abort_flag, 2)) { ok = false; break; }
@@ -297,22 +459,27 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
                 const unsigned d_tmem = tmem_base + acc * BN;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(&sh.full[s], (uses >> s) & 1u, abort_flag, 3)) { ok = false; break; }
+                    if (tile_it == 1 && kb == 0) TRACE(5);
                     tcgen05_fence_after();
 #pragma unroll
                     for (int u = 0; u < KSUB; ++u) {
-                        const unsigned a_addr = smem_u32(smem + s * sb + u * (sb / KSUB));
+                        const unsigned a_addr = smem_u32(smem + s * sb + u * subb);
                         const unsigned long long adesc = smem_desc_sw128(a_addr);
-                        const unsigned long long bdesc = smem_desc_sw128(a_addr + A_BYTES);
+                        const unsigned long long bdesc = smem_desc_sw128(a_addr + a_bytes);
 #pragma unroll
                         for (int k = 0; k < BK / UMMA_K; ++k)
                             umma_bf16_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | u | k) != 0);
                     }
-                    umma_commit_pair_both(&sh.empty[s]);   // both producers may refill this stage
+                    // both producers may refill this stage -- after the norm warps have read the
+                    // A tiles, where those yield the row norms
+                    umma_commit_pair_both(duty ? &sh.consumed[s] : &sh.empty[s]);
                     uses ^= 1u << s;
                     s = (s + 1 == cur_nst) ? 0 : s + 1;
                 }
                 if (ok) umma_commit_pair_both(&sh.tmem_full[acc]);   // both epilogues may read
+                TRACE(8 + 2 * (int)min(tile_it - 1, 8u));
             }
+            TRACE(6);
             umma_commit_pair_local(&sh.drain);
             const unsigned long long t0 = global_ns();
             while (!mbar_try(&sh.drain, 0)) {
@@ -327,6 +494,7 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
         const unsigned dep_total = 8u * (unsigned)tiles0;
         bool dep_ok = !(nseg > 1 && tiles0 > 0);
         bool norm_ok = norms.X == nullptr;           // row norms computed by this launch's norm warps
+        bool gather_ok = !has_gather;
         const unsigned norm_total = (unsigned)(gridDim.x * NORM_WARPS);
         // the accumulator goes back to the leader's barrier
         const unsigned empty_addr[2] = {map_to_cta(smem_u32(&sh.tmem_empty[0]), 0),
@@ -335,16 +503,22 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
         for (int id = pair; id < total; id += npairs) {
             const int sg = id < tiles0 ? 0 : 1;
             const GramProblem& p = sg ? seg1 : seg0;
-            if (!decode_tile(p, id - (sg ? tiles0 : 0), pc)) break;
-                if (dead_tile(p, pc)) continue;   // causal cross tile with no admissible pair
+            if (!decode_tile(p, hrows, id - (sg ? tiles0 : 0), pc)) break;
+            if (dead_tile(p, pc, hrows, smem_norms)) continue;   // causal cross tile with no admissible pair
             const unsigned acc = tile_it & 1u, acc_ph = (tile_it >> 1) & 1u;
-                ++tile_it;
+            ++tile_it;
             const int64_t o = (int64_t)pc.b * p.cap;
             const int ncols = pc.ncols;
+            if (!gather_ok) {
+                // the gathered rows' inverse norms (column factors, and the triangle's row factors)
+                if (!wait_counter(dep_ctr + 3, gather_total, lane, abort_flag, 13)) break;
+                gather_ok = true;
+            }
             if (sg == 1 && !dep_ok) {
                 // every triangular tile of this launch first (line 5 before line 7)
                 if (!wait_counter(dep_ctr, dep_total, lane, abort_flag, 5)) break;
                 dep_ok = true;
+                if (warp == 2 && lane == 0) TRACE(4);
             }
             if (p.wait_norm_b && !norm_ok) {
                 if (!wait_counter(dep_ctr + 1, norm_total, lane, abort_flag, 9)) break;
@@ -359,7 +533,7 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
                 float fb[BN / 32];
                 unsigned gate[BN / 32] = {};
                 int tk[BN / 32] = {};
-                const int last = pc.n - 1;
+                const int last = max(pc.n - 1, 0);
                 const unsigned thr_b = (!p.tri && p.thr_seq != nullptr) ? p.thr_seq[pc.b] : p.thr_bits;
 #pragma unroll
                 for (int q = 0; q < BN / 32; ++q)
@@ -387,17 +561,22 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
             }
             __syncwarp();
             // this thread's row: its role and inverse norm are fetched while the MMAs finish
-            const int row_base = pc.row0 + (int)rank * BM;
-            const int row = row_base + quad * 32 + lane;
-            const bool row_live = row < pc.m;
-            const bool skip = row_live && !p.tri && p.row_role[o + row] != 0;   // inherited reps are not candidates
+            const int arows = p.tri ? BM : hrows;
+            const int lrow = quad * 32 + lane;
+            const int row_base = pc.row0 + (int)rank * arows;
+            const int row = row_base + lrow;
+            const bool row_live = lrow < arows && row < pc.m;
+            const bool defer = !p.tri && p.defer_row != 0;   // the row's own factor is applied later
+            // inherited reps are not candidates (with a deferred factor the compaction ignores them)
+            const bool skip = row_live && !p.tri && !defer && p.row_role[o + row] != 0;
             const bool inv_early = !(p.wait_norm_a && !norm_ok);
-            float inv_row = (row_live && inv_early) ? __ldcg(p.inv_a + o + row) : 0.f;
+            float inv_row = defer ? 1.0f : ((row_live && inv_early) ? __ldcg(p.inv_a + o + row) : 0.f);
             const bool got = mbar_wait(&sh.tmem_full[acc], acc_ph, abort_flag, 4);
             if (!__all_sync(0xffffffffu, got)) break;
             tcgen05_fence_after();
             const bool need_cmp = p.tri ? (pc.col0 + ncols > row_base) : (p.causal != 0);
             float mx = 0.f;
+            // (a warp whose 32 rows lie past a short tile's rows still joins the aligned loads)
             for (int c0 = 0; c0 < ncols; c0 += 32) {
                 float v[32];
                 tmem_ld32(tmem_base + ((unsigned)(quad * 32) << 16) + acc * BN + c0, v);
@@ -421,13 +600,13 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
             tcgen05_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_remote(empty_addr[acc]);
-            if (p.wait_norm_a && !norm_ok) {
+            if (!defer && p.wait_norm_a && !norm_ok) {
                 if (!wait_counter(dep_ctr + 1, norm_total, lane, abort_flag, 9)) break;
                 norm_ok = true;
             }
             if (row_live) {
                 if (!skip) {
-                    if (!inv_early) inv_row = __ldcg(p.inv_a + o + row);
+                    if (!defer && !inv_early) inv_row = __ldcg(p.inv_a + o + row);
                     mx *= inv_row;
                     if (mx > 0.f) atomicMax(p.out + o + row, __float_as_uint(mx));
                 }
@@ -437,11 +616,92 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
                 __syncwarp();
                 if (lane == 0) atomicAdd(dep_ctr, 1u);
             }
+            if (warp == 2 && lane == 0) TRACE(9 + 2 * (int)min(tile_it - 1, 8u));
         }
-    } else if (norms.X != nullptr) {
-        // ------------------------------------------------ row norms (warps 6 and up)
-        norm_rows(norms, blockIdx.x * NORM_WARPS + (warp - 6), gridDim.x * NORM_WARPS, lane,
-                  dep_ctr + 1, status);
+    } else {
+        // ------------------------------------------------ helper warps (6 and up)
+        if (norms.X != nullptr)       // full selection: row norms with plain loads
+            norm_rows(norms, blockIdx.x * NORM_WARPS + (warp - 6), gridDim.x * NORM_WARPS, lane,
+                      dep_ctr + 1, status);
+        if (has_gather)               // Algorithm 1 lines 1-2
+            gather_rows(gather, blockIdx.x * NORM_WARPS + (warp - 6), gridDim.x * NORM_WARPS, lane,
+                        dep_ctr + 3, status);
+        if (warp == 6 && lane == 0) TRACE(2);
+        const GramProblem& cx = (nseg > 1) ? seg1 : seg0;
+        if (!cx.tri && cx.inv_out != nullptr && !smem_norms) {
+            // several column tiles: 1/||x_t|| of every row with plain loads, behind the main loops
+            // (nothing in this launch waits for them: the row factor is applied by the compaction)
+            NormJob nj;
+            nj.X = cx.A; nj.ldx = cx.lda; nj.n_rows = (int64_t)cx.B * cx.rows; nj.d = cx.d;
+            nj.inv_norm = cx.inv_out;
+            nj.batch = cx.a_batch; nj.rows_per_seq = cx.rows;
+            norm_rows(nj, blockIdx.x * NORM_WARPS + (warp - 6), gridDim.x * NORM_WARPS, lane,
+                      dep_ctr + 1, status);
+        } else if (warp < 6 + SMEM_NORM_WARPS && !cx.tri && cx.inv_out != nullptr) {
+            // row norms of X out of the A tiles in shared memory: thread lrow owns row lrow of
+            // the CTA's tile; this role follows the ring exactly as the producer fills it
+            const int lrow = (warp - 6) * 32 + lane;
+            unsigned cons = 0;
+            int cur_sb = 0, cur_nst = 0, s = 0;
+            bool ok = true;
+            for (int id = pair; ok && id < total; id += npairs) {
+                const int sg = id < tiles0 ? 0 : 1;
+                const GramProblem& p = sg ? seg1 : seg0;
+                if (!decode_tile(p, hrows, id - (sg ? tiles0 : 0), pc)) break;
+                if (dead_tile(p, pc, hrows, smem_norms)) continue;
+                const int num_kb = (p.d + BKS - 1) / BKS;
+                const int arows = p.tri ? BM : hrows;
+                const int a_bytes = a_bytes_of(arows);
+                const int subb = sub_bytes_pair(a_bytes, pc.ncols);
+                const int sb = KSUB * subb;
+                if (sb != cur_sb) { cur_sb = sb; cur_nst = stage_count(sb, a_bytes); s = 0; }
+                if (!norm_duty(p, pc, smem_norms)) { s = (s + num_kb) % cur_nst; continue; }
+                float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    int good = 1;
+                    if (lane == 0) good = mbar_wait(&sh.consumed[s], (cons >> s) & 1u, abort_flag, 14) ? 1 : 0;
+                    if (__shfl_sync(0xffffffffu, good, 0) == 0) { ok = false; break; }
+                    if (lrow < arows) {
+#pragma unroll
+                        for (int u = 0; u < KSUB; ++u) {
+                            // the 16-byte chunks of a row are permuted by the swizzle, which a sum
+                            // of squares need not undo; lanes start at different chunks so that a
+                            // warp's loads spread over all banks
+                            const unsigned char* rowp = smem + s * sb + u * subb + lrow * 128;
+                            uint4 x[8];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j)
+                                x[j] = *reinterpret_cast<const uint4*>(rowp + (((j + lane) & 7) << 4));
+                            s0 += sumsq_bf16x8(x[0]) + sumsq_bf16x8(x[4]);
+                            s1 += sumsq_bf16x8(x[1]) + sumsq_bf16x8(x[5]);
+                            s2 += sumsq_bf16x8(x[2]) + sumsq_bf16x8(x[6]);
+                            s3 += sumsq_bf16x8(x[3]) + sumsq_bf16x8(x[7]);
+                        }
+                    }
+                    __syncwarp();
+                    // the last of the four warps releases the stage to the producer
+                    if (lane == 0) {
+                        if (atomicAdd(&sh.norm_cnt[s], 1u) == SMEM_NORM_WARPS - 1) {
+                            sh.norm_cnt[s] = 0u;
+                            mbar_arrive(&sh.empty[s]);
+                        }
+                    }
+                    cons ^= 1u << s;
+                    s = (s + 1 == cur_nst) ? 0 : s + 1;
+                }
+                if (!ok) break;
+                const int row = pc.row0 + (int)rank * arows + lrow;
+                if (lrow < arows && row < pc.m) {
+                    const float ss = (s0 + s1) + (s2 + s3);
+                    float inv = 0.f;
+                    if (!(ss <= 3.0e38f)) atomicOr(status, ST_NONFINITE);
+                    else if (ss > 0.f) inv = 1.0f / sqrtf(ss);
+                    else atomicAdd(status + 1, 1u);
+                    p.inv_out[(int64_t)pc.b * p.cap + row] = inv;
+                }
+                if (lrow == 0) TRACE(40);
+            }
+        }
     }
 
     tcgen05_fence_before();
@@ -457,34 +717,54 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
         atomicOr(status, ST_TIMEOUT);
         status[2] = 100u + (unsigned)sh.abort_flag;
     }
+    if (threadIdx.x == 0) TRACE(63);
 }
 
 }  // namespace
 
+static cudaError_t ensure_tc2(ada_ctx* ctx) {
+    if (ctx->tc2_attr_set) return cudaSuccess;
+    cudaError_t e = cudaFuncSetAttribute(k_gram_tc2, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         SMEM_PAIR_BYTES);
+    if (e != cudaSuccess) return e;
+    // how many clusters of two fit on the device at once
+    cudaLaunchConfig_t q;
+    memset(&q, 0, sizeof(q));
+    q.gridDim = dim3(2 * (ctx->sm_count / 2));
+    q.blockDim = dim3(NUM_THREADS);
+    q.dynamicSmemBytes = SMEM_PAIR_BYTES;
+    cudaLaunchAttribute qa[1];
+    qa[0].id = cudaLaunchAttributeClusterDimension;
+    qa[0].val.clusterDim.x = 2; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
+    q.attrs = qa; q.numAttrs = 1;
+    int nclusters = 0;
+    e = cudaOccupancyMaxActiveClusters(&nclusters, k_gram_tc2, &q);
+    if (e != cudaSuccess || nclusters < 1) { cudaGetLastError(); return cudaErrorLaunchOutOfResources; }
+    ctx->tc2_pairs = nclusters < ctx->sm_count / 2 ? nclusters : ctx->sm_count / 2;
+    ctx->tc2_attr_set = true;
+    return cudaSuccess;
+}
+
+// Rows of X per CTA for a cross-Gram whose columns fit one column tile (at most 256
+// representatives per sequence): such a launch is one pass over X, so the row tiles are cut to
+// give every SM pair but the ones that take the small triangular problems a share.  128 = the
+// ordinary tile.  (0 if the kernel cannot be configured.)
+int gram_tc2_hb_rows(ada_ctx* ctx, int B, int T) {
+    if (ensure_tc2(ctx) != cudaSuccess) return 0;
+    const int free_pairs = ctx->tc2_pairs - B;            // one triangular tile per sequence
+    if (free_pairs < B) return BM;
+    const int tiles_per_seq = free_pairs / B;
+    int h = (T + 2 * tiles_per_seq - 1) / (2 * tiles_per_seq);
+    if (h < 16) h = 16;
+    return h >= BM ? BM : h;
+}
+
 // Pair-CTA launch.  tri and/or cross may be NULL; with both the cross epilogues wait in-kernel
 // for the triangular segment (ctx->tile_ctr must be zero at launch).
 cudaError_t launch_gram_tc2(ada_ctx* ctx, const GramProblem* tri, const GramProblem* cross,
-                            const NormJob* norms, cudaStream_t s) {
-    if (!ctx->tc2_attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(k_gram_tc2, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             SMEM_BYTES);
-        if (e != cudaSuccess) return e;
-        // how many clusters of two fit on the device at once
-        cudaLaunchConfig_t q;
-        memset(&q, 0, sizeof(q));
-        q.gridDim = dim3(2 * (ctx->sm_count / 2));
-        q.blockDim = dim3(NUM_THREADS);
-        q.dynamicSmemBytes = SMEM_BYTES;
-        cudaLaunchAttribute qa[1];
-        qa[0].id = cudaLaunchAttributeClusterDimension;
-        qa[0].val.clusterDim.x = 2; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
-        q.attrs = qa; q.numAttrs = 1;
-        int nclusters = 0;
-        e = cudaOccupancyMaxActiveClusters(&nclusters, k_gram_tc2, &q);
-        if (e != cudaSuccess || nclusters < 1) { cudaGetLastError(); return cudaErrorLaunchOutOfResources; }
-        ctx->tc2_pairs = nclusters < ctx->sm_count / 2 ? nclusters : ctx->sm_count / 2;
-        ctx->tc2_attr_set = true;
-    }
+                            const NormJob* norms, const GatherJob* gather, cudaStream_t s) {
+    cudaError_t e0 = ensure_tc2(ctx);
+    if (e0 != cudaSuccess) return e0;
     GramMaps maps;
     memset(&maps, 0, sizeof(maps));
     GramProblem segs[2];
@@ -500,27 +780,38 @@ cudaError_t launch_gram_tc2(ada_ctx* ctx, const GramProblem* tri, const GramProb
         if (!make_map(&maps.a[nseg], p->A, p->d, p->tri ? p->cap : p->rows, p->B, p->lda, p->a_batch, BM) ||
             !make_map(&maps.b[nseg], p->Bm, p->d, p->cap, p->B, p->ldb, p->b_batch, BOX_N))
             return cudaErrorInvalidValue;
+        if (!p->tri) {
+            const int hb = (p->hb_rows > 0 && p->hb_rows < BM) ? p->hb_rows : BM;
+            if (!make_map(&maps.ah, p->A, p->d, p->rows, p->B, p->lda, p->a_batch, hb))
+                return cudaErrorInvalidValue;
+        }
         segs[nseg++] = *p;
     }
     if (nseg == 0) return cudaSuccess;
     if (nseg == 1) { maps.a[1] = maps.a[0]; maps.b[1] = maps.b[0]; segs[1] = segs[0]; segs[1].B = 0; }
+    if (segs[0].tri && nseg == 1) maps.ah = maps.a[0];
     NormJob nj;
     memset(&nj, 0, sizeof(nj));
     if (norms != nullptr) nj = *norms;
+    GatherJob gj;
+    memset(&gj, 0, sizeof(gj));
+    if (gather != nullptr) gj = *gather;
     const bool fused = nseg == 2;
     prof_begin(ctx, fused ? K_GRAM_TC_CASCADE : (segs[0].tri ? K_GRAM_TC_TRI : K_GRAM_TC_CROSS), s);
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3(2 * ctx->tc2_pairs);
     cfg.blockDim = dim3(NUM_THREADS);
-    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.dynamicSmemBytes = SMEM_PAIR_BYTES;
     cfg.stream = s;
     cudaLaunchAttribute attr[3];
     int na = 0;
     attr[na].id = cudaLaunchAttributeClusterDimension;
     attr[na].val.clusterDim.x = 2; attr[na].val.clusterDim.y = 1; attr[na].val.clusterDim.z = 1;
     ++na;
-    if (fused && ctx->cooperative) {
+    // CTAs wait on results of other CTAs (triangle before cross epilogues, the gather before
+    // everything): all of them have to be resident
+    if ((fused || gj.X != nullptr) && ctx->cooperative) {
         attr[na].id = cudaLaunchAttributeCooperative;
         attr[na].val.cooperative = 1;
         ++na;
@@ -532,10 +823,21 @@ cudaError_t launch_gram_tc2(ada_ctx* ctx, const GramProblem* tri, const GramProb
     }
     cfg.attrs = attr;
     cfg.numAttrs = na;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, k_gram_tc2, maps, segs[0], segs[1], nseg, nj, ctx->tile_ctr,
+    cudaError_t e = cudaLaunchKernelEx(&cfg, k_gram_tc2, maps, segs[0], segs[1], nseg, nj, gj, ctx->tile_ctr,
                                        ctx->status);
     prof_end(ctx, s);
     return e;
 }
 
 }  // namespace ada
+
+#ifdef ADA_TRACE
+extern "C" int ada_trace_read(unsigned long long* host, int clear) {
+    if (cudaMemcpyFromSymbol(host, ada::g_trace, sizeof(ada::g_trace)) != cudaSuccess) return 1;
+    if (clear) {
+        static unsigned long long zeros[160 * 64];
+        if (cudaMemcpyToSymbol(ada::g_trace, zeros, sizeof(zeros)) != cudaSuccess) return 2;
+    }
+    return 0;
+}
+#endif

@@ -249,7 +249,10 @@ static __device__ __forceinline__ void norm_rows(const NormJob& job, int w, int 
     const int nvec = job.d >> 3;
     const __nv_bfloat16* X = reinterpret_cast<const __nv_bfloat16*>(job.X);
     for (int64_t row = w; row < job.n_rows; row += nw) {
-        const uint4* src = reinterpret_cast<const uint4*>(X + row * job.ldx);
+        const int64_t off = job.rows_per_seq > 0
+            ? (row / job.rows_per_seq) * job.batch + (row % job.rows_per_seq) * job.ldx
+            : row * job.ldx;
+        const uint4* src = reinterpret_cast<const uint4*>(X + off);
         // sixteen (then eight) independent 128-bit loads in flight per lane: these few warps
         // have to cover the memory latency that a dedicated kernel would hide with occupancy
         float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;

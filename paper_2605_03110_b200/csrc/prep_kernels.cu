@@ -451,6 +451,7 @@ struct CompactArgs {
     float thr;
     int32_t *keep_idx, *keep_cnt, *add_idx, *add_cnt, *rem_idx, *rem_cnt;
     float *gamma_a, *gamma_b;    // full: gamma | cascade: gamma_rep, gamma_cross (optional)
+    const float* row_scale;      // cascade: 1/||x_t|| still to be applied to g_tok, or NULL
     // adaptive threshold (Section 8.1)
     const float* thr_seq;        // [B] thresholds of this step, or NULL = thr
     const int32_t* r_in;         // [B] inherited counts (Eq. 6 denominator)
@@ -513,6 +514,7 @@ __global__ void __launch_bounds__(1024) k_compact(const CompactArgs a) {
     // independent loads first, the position-indexed gather second
     const int pos = (cascade && in) ? a.role[o + t] : 0;
     const unsigned gt = in ? a.g_tok[o + t] : 0u;
+    const float rs = (in && a.row_scale != nullptr) ? a.row_scale[o + t] : 1.0f;
     const unsigned gp = pos > 0 ? a.g_rep[o + pos - 1] : 0u;
     bool keep = false, add = false, rem = false;
     if (in) {
@@ -524,7 +526,8 @@ __global__ void __launch_bounds__(1024) k_compact(const CompactArgs a) {
             a.g_rep[o + pos - 1] = 0u;
             a.role[o + t] = 0;
         } else {                          // Definition 1 / line 9
-            gb = __uint_as_float(gt);
+            // (an untouched entry is a maximum over nothing: 0 whatever the row's norm)
+            gb = gt != 0u ? __uint_as_float(gt) * rs : 0.f;
             keep = gb < thr;
             add = cascade && keep;
         }
@@ -605,6 +608,7 @@ __global__ void __launch_bounds__(1024) k_compact(const CompactArgs a) {
             *a.done_ctr = 0u;
             a.dep_ctr[0] = 0u;
             a.dep_ctr[1] = 0u;   // norm warps' counter of the Gram launch
+            a.dep_ctr[3] = 0u;   // in-launch gather counter
         }
     }
 }
@@ -673,7 +677,7 @@ cudaError_t launch_compact_full(ada_ctx* ctx, int B, int T, float thr, int32_t* 
     a.agg_stride = ctx->agg_stride; a.T = T; a.thr = thr;
     a.keep_idx = rep_idx; a.keep_cnt = rep_cnt;
     a.add_idx = nullptr; a.add_cnt = nullptr; a.rem_idx = nullptr; a.rem_cnt = nullptr;
-    a.gamma_a = gamma; a.gamma_b = nullptr;
+    a.gamma_a = gamma; a.gamma_b = nullptr; a.row_scale = nullptr;
     a.thr_seq = nullptr; a.r_in = nullptr;
     memset(&a.tu, 0, sizeof(a.tu));
     return launch_compact(ctx, K_COMPACT_FULL, a, B, s);
@@ -682,7 +686,8 @@ cudaError_t launch_compact_full(ada_ctx* ctx, int B, int T, float thr, int32_t* 
 cudaError_t launch_compact_cascade(ada_ctx* ctx, int B, int T, float thr, int32_t* rep_out,
                                    int32_t* rep_out_cnt, int32_t* add_idx, int32_t* add_cnt,
                                    int32_t* rem_idx, int32_t* rem_cnt, float* gamma_rep,
-                                   float* gamma_cross, const TauUpdate& tu, cudaStream_t s) {
+                                   float* gamma_cross, const TauUpdate& tu, bool row_scale,
+                                   cudaStream_t s) {
     CompactArgs a;
     a.g_tok = ctx->g_tok; a.g_rep = ctx->g_rep; a.role = ctx->role;
     a.agg = ctx->agg; a.done_ctr = ctx->done_ctr; a.dep_ctr = ctx->tile_ctr; a.status = ctx->status;
@@ -690,6 +695,7 @@ cudaError_t launch_compact_cascade(ada_ctx* ctx, int B, int T, float thr, int32_
     a.keep_idx = rep_out; a.keep_cnt = rep_out_cnt;
     a.add_idx = add_idx; a.add_cnt = add_cnt; a.rem_idx = rem_idx; a.rem_cnt = rem_cnt;
     a.gamma_a = gamma_rep; a.gamma_b = gamma_cross;
+    a.row_scale = row_scale ? ctx->inv_norm : nullptr;
     a.thr_seq = tu.tau_state != nullptr ? ctx->thr_seq : nullptr;
     a.r_in = ctx->r_eff;
     a.tu = tu;
