@@ -230,6 +230,7 @@ def sweep(args):
     print("|---|---|---|---|---|---|---|---|---|---|---|")
     for T in wl.SWEEP_T:
         ctx = ada.ada_create(1, T, 4096, ada.ADA_BF16)
+        ada.ada_set_engine(ctx, args.engine)
         for q in wl.SWEEP_Q:
             cfg = wl.sweep_config(T, q)
             X0, X1 = [torch.from_numpy(lb.X.view(np.int16)).view(torch.bfloat16).to(dev)
@@ -413,7 +414,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=4, choices=[1, 2, 3, 4])
     ap.add_argument("--layers", type=int, default=0, help="override L (0 = the configuration's)")
-    ap.add_argument("--engine", type=int, default=0, help="0 auto, 1 force FFMA Gram")
+    ap.add_argument("--engine", type=int, default=0,
+                    help="0 auto, 1 force the FFMA Gram, 2 the one-CTA tcgen05 kernel, 3 the pair-CTA one")
     ap.add_argument("--ref-layers", type=int, default=4)
     ap.add_argument("--ref-warmup", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -62,9 +62,10 @@ bool use_split(const ada_ctx* ctx, ada_dtype dt) {
 // the pair-CTA form of the tensor-core kernel, or the one-CTA form?
 bool use_pair(const ada_ctx* ctx, int64_t B, int64_t T, int64_t d) {
     if (ctx->engine == ADA_ENGINE_TCGEN05_PAIR) return true;
-    // The pair kernel pays off once there are several 256-row tiles per SM pair and a long
-    // contraction; small problems are covered better by the finer one-CTA tiles.
-    return ctx->engine == ADA_ENGINE_AUTO && B * T >= 8192 && d >= 2048;
+    // The pair kernel pays off from a few thousand rows and a long contraction on (measured on
+    // the crossover sweep: at T = 4096, d = 4096 both calls are faster on it, at T = 2048 they
+    // are not); small problems are covered better by the finer one-CTA tiles.
+    return ctx->engine == ADA_ENGINE_AUTO && B * T >= 4096 && d >= 2048;
 }
 
 // tensor-core launch of one or two segments, in the one-CTA or the pair-CTA form

@@ -234,6 +234,13 @@ __device__ __forceinline__ void gather_rows(const GatherJob& gj, int g, int nw, 
     const int nvec = gj.d >> 3;
     int b = 0;
     int64_t item = g;
+    // this warp's first entry is most often entry g of sequence 0: fetch it (and its
+    // predecessor) beside the count instead of after it
+    int32_t first_idx = 0, first_prev = -1;
+    if (g < gj.T) {
+        first_idx = __ldg(gj.rep_in + g);
+        if (g > 0) first_prev = __ldg(gj.rep_in + g - 1);
+    }
     while (b < gj.B) {
         int cnt = gj.rep_in_cnt[b];
         if (cnt < 0 || cnt > gj.T) {
@@ -245,9 +252,10 @@ __device__ __forceinline__ void gather_rows(const GatherJob& gj, int g, int nw, 
         const int i = (int)item;
         item += nw;                                   // this warp's next entry (maybe in a later sequence)
         const int32_t* list = gj.rep_in + (int64_t)b * gj.T;
-        const int32_t idx = list[i];
+        const bool spec = b == 0 && i == g;
+        const int32_t idx = spec ? first_idx : list[i];
         bool ok = idx >= 0 && idx < gj.T;
-        if (ok && i > 0) ok = list[i - 1] < idx;
+        if (ok && i > 0) ok = (spec ? first_prev : list[i - 1]) < idx;
         const int64_t prow = (int64_t)b * gj.T + i;
         if (!ok) {
             if (lane == 0) { atomicOr(status, ST_BAD_INDEX); gj.inv_rep[prow] = 0.f; }
@@ -365,7 +373,9 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
     const int tiles0 = sh.tiles0, total = sh.tiles0 + sh.tiles1;
     const int hrows = sh.hrows;                          // rows per CTA of a cross tile
     const bool smem_norms = sh.one_col_tile != 0;        // row norms out of the tiles in shared memory
-    const unsigned gather_total = (unsigned)(gridDim.x * NORM_WARPS);
+    // the helper warps AND the epilogue warps (idle until the first tile is done) share the gather
+    constexpr int GATHER_WARPS = NORM_WARPS + 4;
+    const unsigned gather_total = (unsigned)(gridDim.x * GATHER_WARPS);
     const bool has_gather = gather.X != nullptr;
     Piece pc;
     if (threadIdx.x == 0) TRACE(1);
@@ -496,6 +506,9 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
         bool norm_ok = norms.X == nullptr;           // row norms computed by this launch's norm warps
         bool gather_ok = !has_gather;
         const unsigned norm_total = (unsigned)(gridDim.x * NORM_WARPS);
+        if (has_gather)               // Algorithm 1 lines 1-2, shared with the helper warps
+            gather_rows(gather, blockIdx.x * GATHER_WARPS + NORM_WARPS + (warp - 2), gridDim.x * GATHER_WARPS,
+                        lane, dep_ctr + 3, status);
         // the accumulator goes back to the leader's barrier
         const unsigned empty_addr[2] = {map_to_cta(smem_u32(&sh.tmem_empty[0]), 0),
                                         map_to_cta(smem_u32(&sh.tmem_empty[1]), 0)};
@@ -624,7 +637,7 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
             norm_rows(norms, blockIdx.x * NORM_WARPS + (warp - 6), gridDim.x * NORM_WARPS, lane,
                       dep_ctr + 1, status);
         if (has_gather)               // Algorithm 1 lines 1-2
-            gather_rows(gather, blockIdx.x * NORM_WARPS + (warp - 6), gridDim.x * NORM_WARPS, lane,
+            gather_rows(gather, blockIdx.x * GATHER_WARPS + (warp - 6), gridDim.x * GATHER_WARPS, lane,
                         dep_ctr + 3, status);
         if (warp == 6 && lane == 0) TRACE(2);
         const GramProblem& cx = (nseg > 1) ? seg1 : seg0;
