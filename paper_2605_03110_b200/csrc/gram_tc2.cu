@@ -208,89 +208,6 @@ struct GramMaps {
     CUtensorMap ah;          // left operand of the cross segment in boxes of hb_rows rows
 };
 
-// bounded wait of ONE thread until a global counter reaches `target`
-__device__ __forceinline__ bool wait_counter_1(const unsigned* counter, unsigned target,
-                                               volatile int* abort_flag, int where) {
-    const unsigned long long t0 = global_ns();
-    unsigned seen;
-    while (true) {
-        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
-        if (seen >= target) return true;
-        if (*abort_flag != 0) return false;
-        if (global_ns() - t0 > WAIT_LIMIT_NS) { *abort_flag = where; return false; }
-        __nanosleep(64);
-    }
-}
-
-// Algorithm 1 lines 1-2, by the helper warps of every CTA (warp `g` of `nw`): entry i of
-// sequence b is checked (in range, strictly above entry i-1), role[token] = i + 1, the raw row
-// goes to Xrep[b, i] and its inverse norm to inv_rep[b, i]; a rejected entry gets inverse norm
-// 0 (its column then counts for nothing) and raises the status.  Ends with one arrival per warp
-// on `counter`.
-__device__ __forceinline__ void gather_rows(const GatherJob& gj, int g, int nw, int lane,
-                                            unsigned* counter, unsigned* status) {
-    const __nv_bfloat16* X = reinterpret_cast<const __nv_bfloat16*>(gj.X);
-    __nv_bfloat16* Xrep = reinterpret_cast<__nv_bfloat16*>(gj.Xrep);
-    const int nvec = gj.d >> 3;
-    int b = 0;
-    int64_t item = g;
-    // this warp's first entry is most often entry g of sequence 0: fetch it (and its
-    // predecessor) beside the count instead of after it
-    int32_t first_idx = 0, first_prev = -1;
-    if (g < gj.T) {
-        first_idx = __ldg(gj.rep_in + g);
-        if (g > 0) first_prev = __ldg(gj.rep_in + g - 1);
-    }
-    while (b < gj.B) {
-        int cnt = gj.rep_in_cnt[b];
-        if (cnt < 0 || cnt > gj.T) {
-            if (g == 0 && lane == 0) atomicOr(status, ST_BAD_COUNT);
-            cnt = cnt < 0 ? 0 : gj.T;
-        }
-        if (g == 0 && lane == 0) gj.r_eff[b] = cnt;
-        if (item >= cnt) { item -= cnt; ++b; continue; }
-        const int i = (int)item;
-        item += nw;                                   // this warp's next entry (maybe in a later sequence)
-        const int32_t* list = gj.rep_in + (int64_t)b * gj.T;
-        const bool spec = b == 0 && i == g;
-        const int32_t idx = spec ? first_idx : list[i];
-        bool ok = idx >= 0 && idx < gj.T;
-        if (ok && i > 0) ok = (spec ? first_prev : list[i - 1]) < idx;
-        const int64_t prow = (int64_t)b * gj.T + i;
-        if (!ok) {
-            if (lane == 0) { atomicOr(status, ST_BAD_INDEX); gj.inv_rep[prow] = 0.f; }
-            continue;
-        }
-        const uint4* src = reinterpret_cast<const uint4*>(X + (int64_t)b * gj.xb + (int64_t)idx * gj.ldx);
-        uint4* dst = reinterpret_cast<uint4*>(Xrep + prow * (int64_t)gj.d);
-        float ss = 0.f;
-        int v = lane;
-        for (; v + 480 < nvec; v += 512) {            // sixteen loads in flight per lane
-            uint4 x[16];
-#pragma unroll
-            for (int q = 0; q < 16; ++q) x[q] = __ldg(src + v + 32 * q);
-#pragma unroll
-            for (int q = 0; q < 16; ++q) { ss += sumsq_bf16x8(x[q]); dst[v + 32 * q] = x[q]; }
-        }
-        for (; v < nvec; v += 32) {
-            const uint4 x = __ldg(src + v);
-            ss += sumsq_bf16x8(x);
-            dst[v] = x;
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-        if (lane == 0) {
-            gj.inv_rep[prow] = (ss <= 3.0e38f && ss > 0.f) ? 1.0f / sqrtf(ss) : 0.f;
-            gj.role[(int64_t)b * gj.T + idx] = i + 1;
-        }
-    }
-    // the rows just written are read by TMA (async proxy) from other CTAs
-    asm volatile("fence.proxy.async.global;" ::: "memory");
-    __threadfence();
-    __syncwarp();
-    if (lane == 0) atomicAdd(counter, 1u);
-}
-
 // ---------------------------------------------------------------- the kernel
 struct alignas(16) SharedPair {
     unsigned long long full[MAX_STAGES];
