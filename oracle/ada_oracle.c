@@ -24,6 +24,10 @@
  *     variant for which Proposition 3's proof goes through).
  *   - tokens removed at line 5 are not re-examined as additions (line 6 uses
  *     the complement of the inherited set).
+ *   - Eq. 2 (attention on the representative set) is taken as printed: every
+ *     representative attends to every representative; `causal` != 0 restricts
+ *     row i to the representatives at or before it in token order (what a
+ *     causal language model's attention would keep).
  *
  * Pinned by tests/test_oracle_*.py (worked examples, closed forms, brute
  * force, invariants, an independent numpy statement, label-level prediction).
@@ -289,4 +293,56 @@ double ada_oracle_tau_update(double tau, double rho, double target, double gain,
 double ada_oracle_turnover(int64_t n_add, int64_t n_rem, int64_t r) {
     if (r == 0) return NAN;
     return (double)(n_add + n_rem) / (double)r;
+}
+
+/*
+ * Attention on the representative set (Section 2.3, Eq. 2) for one sequence of T tokens
+ * and h heads.  Q, K, V: [T][h][d_h].  For head j, with rho_0 < ... < rho_{r-1} the
+ * representatives:
+ *     S_ik   = q_{rho_i} . k_{rho_k} / sqrt(d_h)
+ *     P_i.   = softmax over k of S_i.          (causal: only k <= i)
+ *     A_i    = sum_k P_ik v_{rho_k}
+ * out[rho_i][j][:] = A_i; and, when `nearest` is given, a token t outside the set takes
+ * the output of its nearest representative: out[t][j][:] = out[nearest[t]][j][:]
+ * (Section 2.3).  Rows that receive nothing are set to 0.  Returns 0.
+ */
+int ada_oracle_attention_reps(const double* Q, const double* K, const double* V, int64_t T,
+                              int64_t h, int64_t d_h, const int32_t* rep, int64_t r,
+                              const int32_t* nearest, int causal, double* out) {
+    const int64_t row = h * d_h;
+    memset(out, 0, (size_t)(T * row) * sizeof(double));
+    const double scale = 1.0 / sqrt((double)d_h);
+#pragma omp parallel for schedule(dynamic, 4)
+    for (int64_t ij = 0; ij < r * h; ++ij) {
+        const int64_t i = ij / h, j = ij % h;
+        const double* q = Q + (int64_t)rep[i] * row + j * d_h;
+        double* p = (double*)malloc((size_t)(r > 0 ? r : 1) * sizeof(double));
+        const int64_t kmax = causal ? i + 1 : r;
+        double m = -INFINITY;
+        for (int64_t k = 0; k < kmax; ++k) {
+            const double* kk = K + (int64_t)rep[k] * row + j * d_h;
+            double s = 0.0;
+            for (int64_t c = 0; c < d_h; ++c) s += q[c] * kk[c];
+            p[k] = s * scale;
+            if (p[k] > m) m = p[k];
+        }
+        double z = 0.0;
+        for (int64_t k = 0; k < kmax; ++k) { p[k] = exp(p[k] - m); z += p[k]; }
+        double* o = out + (int64_t)rep[i] * row + j * d_h;
+        for (int64_t k = 0; k < kmax; ++k) {
+            const double w = p[k] / z;
+            const double* v = V + (int64_t)rep[k] * row + j * d_h;
+            for (int64_t c = 0; c < d_h; ++c) o[c] += w * v[c];
+        }
+        free(p);
+    }
+    if (nearest != NULL) {
+        /* representatives map to themselves; -1 (empty set) leaves the row at 0 */
+#pragma omp parallel for schedule(static)
+        for (int64_t t = 0; t < T; ++t) {
+            const int32_t s = nearest[t];
+            if (s >= 0 && s != t) memcpy(out + t * row, out + (int64_t)s * row, (size_t)row * sizeof(double));
+        }
+    }
+    return 0;
 }

@@ -53,6 +53,8 @@ def _load():
         lib.ada_oracle_jaccard.restype = C.c_double
         lib.ada_oracle_turnover.argtypes = [i64, i64, i64]
         lib.ada_oracle_turnover.restype = C.c_double
+        lib.ada_oracle_attention_reps.argtypes = [dp, dp, dp, i64, i64, i64, ip, i64, ip, C.c_int, dp]
+        lib.ada_oracle_attention_reps.restype = C.c_int
         lib.ada_oracle_tau_update.argtypes = [C.c_double] * 6
         lib.ada_oracle_tau_update.restype = C.c_double
         _lib = lib
@@ -166,6 +168,26 @@ def nearest(X, rep):
     if _load().ada_oracle_nearest(_dp(X), T, d, _ip(rep), rep.size, _ip(out), _dp(g)) != 0:
         raise MemoryError
     return out, g
+
+
+def attention_reps(Q, K, V, rep, nearest_idx=None, causal: bool = False) -> np.ndarray:
+    """Eq. 2 on the representative rows of Q, K, V (each T x h x d_h), expanded to all tokens
+    through `nearest_idx` when given (Section 2.3).  Returns out float64 [T, h, d_h]."""
+    Q, K, V = (np.ascontiguousarray(a, dtype=np.float64) for a in (Q, K, V))
+    T, h, d_h = Q.shape
+    assert K.shape == Q.shape and V.shape == Q.shape
+    rep = np.ascontiguousarray(rep, dtype=np.int32)
+    if rep.size and (np.any(np.diff(rep) <= 0) or rep[0] < 0 or rep[-1] >= T):
+        raise ValueError("representative set must be strictly ascending and inside [0, T)")
+    out = np.empty((T, h, d_h), dtype=np.float64)
+    near_p = None
+    if nearest_idx is not None:
+        near = np.ascontiguousarray(nearest_idx, dtype=np.int32)
+        assert near.size == T
+        near_p = _ip(near)
+    _load().ada_oracle_attention_reps(_dp(Q), _dp(K), _dp(V), T, h, d_h, _ip(rep), rep.size, near_p,
+                                      int(bool(causal)), _dp(out))
+    return out
 
 
 def op_count(cascade: bool, T: int, d: int, r: int = 0) -> int:
