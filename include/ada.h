@@ -232,6 +232,34 @@ ada_status ada_nearest_rep(ada_ctx* ctx, const void* X, int64_t B, int64_t T, in
                            const int32_t* rep_cnt, int32_t* nearest_idx, float* nearest_gamma,
                            void* stream);
 
+/*
+ * Attention on the representative set (Section 2.3, Eq. 2):
+ *     Attn_R = softmax(Q_R K_R^T / sqrt(d_h)) V_R        (an r x r problem per head)
+ * with Q_R, K_R, V_R the rows of Q, K, V at the representatives, and the expansion stated with
+ * it: a token outside R takes the attention output of its nearest representative.
+ *   Q, K, V      bf16, ONE sequence of T tokens, h heads side by side in a token's row: head j
+ *                of token t starts at X[t * ld + j * d_h] (ld >= h * d_h); d_h a multiple of 16,
+ *                at most 128; otherwise ADA_ERR_UNSUPPORTED (also for ADA_F32 contexts/inputs)
+ *   rep_idx/cnt  R as an ascending list (device), e.g. the output of a selection call
+ *   nearest_idx  optional, T entries (device), e.g. from ada_nearest_rep on the same R: token t
+ *                receives out[nearest_idx[t]] (a representative maps to itself; -1 gives zeros).
+ *                NULL: only the representatives' rows of `out` are written
+ *   out          fp32, T rows of h * d_h with row stride ldo: out[rho_i] = Attn_R row i
+ *   flags        0: Eq. 2 as printed, every representative attends to every representative;
+ *                ADA_ATTN_CAUSAL: row i only to the representatives at or before it in token
+ *                order (the mask a causal language model applies; the paper's equation has none)
+ * Both contractions run on the tensor cores (tcgen05, accumulators in TMEM), the probabilities
+ * are rounded to bf16 between them, the softmax statistics are fp32.  The gathered copies of
+ * Q_R, K_R and V_R^T live in a buffer of the context allocated on the first call (3 x T x h x
+ * d_h bf16): make that call before capturing into a CUDA graph.  The context must have been
+ * created with maxT >= T and maxd >= h * d_h.  Enqueues on `stream`, never synchronises.
+ */
+#define ADA_ATTN_CAUSAL 1u
+ada_status ada_attention_reps(ada_ctx* ctx, const void* Q, const void* K, const void* V, int64_t T,
+                              int64_t h, int64_t d_h, int64_t ld, ada_dtype dt, const int32_t* rep_idx,
+                              const int32_t* rep_cnt, const int32_t* nearest_idx, float* out,
+                              int64_t ldo, uint32_t flags, void* stream);
+
 /* Same operations with HOST buffers: inputs are copied to the device (staging
  * buffers owned by the context, allocated on first use), the device-pointer
  * call above runs, results are copied back, all on `stream`, and the call

@@ -19,6 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libada.so")
 ADA_OK = 0
 ADA_F32, ADA_BF16 = 0, 1
 ADA_CROSS_CAUSAL = 1
+ADA_ATTN_CAUSAL = 1
 ADA_ENGINE_AUTO, ADA_ENGINE_FFMA, ADA_ENGINE_TCGEN05, ADA_ENGINE_TCGEN05_PAIR = 0, 1, 2, 3
 
 SYMBOLS = [
@@ -27,7 +28,7 @@ SYMBOLS = [
     "ada_device_status", "ada_profile_enable", "ada_profile_read", "ada_status_string",
     "ada_select_full_noalloc", "ada_set_cooperative", "ada_selftest_wait_timeout", "ada_nearest_rep",
     "ada_select_full_heads", "ada_cascade_step_heads", "ada_set_dependent_launch",
-    "ada_cascade_step_adaptive",
+    "ada_cascade_step_adaptive", "ada_attention_reps",
 ]
 ADA_NOALLOC_MAX_T = 16384
 
@@ -73,6 +74,8 @@ def lib() -> C.CDLL:
         L.ada_select_full_heads.argtypes = L.ada_select_full.argtypes
         L.ada_cascade_step_heads.argtypes = L.ada_cascade_step.argtypes
         L.ada_nearest_rep.argtypes = [vp, vp, i64, i64, i64, i64, C.c_int, i32p, i32p, i32p, fp, vp]
+        L.ada_attention_reps.argtypes = [vp, vp, vp, vp, i64, i64, i64, i64, C.c_int, i32p, i32p, i32p, fp,
+                                         i64, C.c_uint32, vp]
         L.ada_select_full_host.argtypes = [vp, vp, i64, i64, i64, C.c_int, C.c_double, i32p, i32p, fp, vp]
         L.ada_cascade_step_host.argtypes = [vp, vp, i64, i64, i64, C.c_int, C.c_double,
                                             i32p, i32p, i32p, i32p, i32p, i32p, i32p, i32p, fp, fp,
@@ -324,6 +327,25 @@ def ada_nearest_rep(ctx: Context, X: torch.Tensor, rep_idx: torch.Tensor, rep_cn
                                  rep_cnt.data_ptr(), near.data_ptr(), _ptr(g), _stream(stream)),
            "ada_nearest_rep")
     return near, g
+
+
+def ada_attention_reps(ctx: Context, Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor,
+                       rep_idx: torch.Tensor, rep_cnt: torch.Tensor, nearest_idx=None, out=None,
+                       flags: int = 0, stream=None) -> torch.Tensor:
+    """Section 2.3, Eq. 2: attention on the representative rows of Q, K, V (each T x h x d_h,
+    bf16), expanded to every token through nearest_idx when given.  Returns out fp32 [T, h, d_h]
+    (rows that receive nothing are left as they are: zeros in a fresh tensor)."""
+    T, h, d_h, ld = _shape_heads(Q)
+    for X in (K, V):
+        if X.shape != Q.shape or X.stride() != Q.stride():
+            raise ValueError("Q, K, V must share shape and strides")
+    if out is None:
+        out = torch.zeros((T, h, d_h), dtype=torch.float32, device=Q.device)
+    _check(lib().ada_attention_reps(ctx.h, Q.data_ptr(), K.data_ptr(), V.data_ptr(), T, h, d_h, ld,
+                                    dtype_of(Q), rep_idx.data_ptr(), rep_cnt.data_ptr(),
+                                    _ptr(nearest_idx), out.data_ptr(), out.stride(0), flags,
+                                    _stream(stream)), "ada_attention_reps")
+    return out
 
 
 def ada_select_full_host(ctx: Context, X: torch.Tensor, tau: float, rep_idx: torch.Tensor,

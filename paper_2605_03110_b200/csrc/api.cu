@@ -157,6 +157,7 @@ ada_status ada_create(ada_ctx** out, int device, int64_t maxB, int64_t maxT, int
     ctx->es = dt == ADA_F32 ? 4 : 2;
     ctx->engine = ADA_ENGINE_AUTO;
     ctx->stage = nullptr; ctx->stage_bytes = 0; ctx->host_stream = nullptr;
+    ctx->attn_ws = nullptr; ctx->attn_ws_bytes = 0;
     ctx->tc_attr_set = false;
     ctx->cooperative = true;
     ctx->dep_launch = true;
@@ -220,6 +221,7 @@ ada_status ada_destroy(ada_ctx* ctx) {
         cudaEventDestroy(ctx->prof.ev1[i]);
     }
     if (ctx->stage) cudaFree(ctx->stage);
+    if (ctx->attn_ws) cudaFree(ctx->attn_ws);
     if (ctx->host_stream) cudaStreamDestroy(ctx->host_stream);
     cudaFree(ctx->ws);
     delete ctx;
@@ -537,6 +539,29 @@ ada_status ada_nearest_rep(ada_ctx* ctx, const void* X, int64_t B, int64_t T, in
     q.causal = 0;
     CU(launch_gram_tc(ctx, nullptr, &q, nullptr, s));
     CU(launch_nearest_finish(ctx, (int)B, (int)T, rep_idx, nearest_idx, nearest_gamma, s));
+    return ADA_OK;
+}
+
+ada_status ada_attention_reps(ada_ctx* ctx, const void* Q, const void* K, const void* V, int64_t T,
+                              int64_t h, int64_t d_h, int64_t ld, ada_dtype dt, const int32_t* rep_idx,
+                              const int32_t* rep_cnt, const int32_t* nearest_idx, float* out,
+                              int64_t ldo, uint32_t flags, void* stream) {
+    if (ctx == nullptr || Q == nullptr || K == nullptr || V == nullptr || rep_idx == nullptr ||
+        rep_cnt == nullptr || out == nullptr)
+        return ADA_ERR_INVALID_ARG;
+    if (T < 1 || h < 1 || d_h < 1 || ld < h * d_h || ldo < h * d_h || (flags & ~ADA_ATTN_CAUSAL) != 0)
+        return ADA_ERR_INVALID_ARG;
+    if (dt != ADA_F32 && dt != ADA_BF16) return ADA_ERR_INVALID_ARG;
+    // bf16 operands on the tensor cores; head widths the two contractions' tiles cover
+    if (dt != ADA_BF16 || ctx->dt != ADA_BF16 || d_h % 16 != 0 || d_h > 128 || !gram_tc_available())
+        return ADA_ERR_UNSUPPORTED;
+    if (T > ctx->maxT || h * d_h > ctx->maxd) return ADA_ERR_WORKSPACE;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(out) || (ld * 2) % 16 != 0 ||
+        (ldo * 4) % 16 != 0)
+        return ADA_ERR_UNSUPPORTED;
+    DeviceGuard guard(ctx->device);
+    CU(launch_attention_reps(ctx, Q, K, V, (int)T, (int)h, (int)d_h, ld, rep_idx, rep_cnt, nearest_idx, out,
+                             ldo, (flags & ADA_ATTN_CAUSAL) ? 1 : 0, static_cast<cudaStream_t>(stream)));
     return ADA_OK;
 }
 

@@ -159,6 +159,9 @@ struct ada_ctx {
     // fp32 contexts: three-term bf16 splits laid out for one contraction of length 6d
     void *splitXA, *splitXB;   // [maxB*maxT][6 maxd] of X
     void *splitRA, *splitRB;   // same, of the gathered representative rows
+    // gathered Q_R, K_R, V_R^T of the attention on the representative set (allocated on first use)
+    char* attn_ws;
+    size_t attn_ws_bytes;
     // staging for the *_host entry points (allocated on first use)
     char* stage;
     size_t stage_bytes;
@@ -242,6 +245,12 @@ cudaError_t launch_gram_tc(ada_ctx* ctx, const GramProblem* tri, const GramProbl
                            const NormJob* norms, cudaStream_t s);
 bool gram_tc_available();
 cudaError_t launch_selftest_wait(ada_ctx* ctx, int limit_ms, cudaStream_t s);
+
+// attn_reps.cu (Eq. 2 on the representative rows, both contractions on tcgen05)
+cudaError_t launch_attention_reps(ada_ctx* ctx, const void* Q, const void* K, const void* V, int T, int h,
+                                  int d_h, int64_t ld, const int32_t* rep_idx, const int32_t* rep_cnt,
+                                  const int32_t* nearest_idx, float* out, int64_t ldo, int causal,
+                                  cudaStream_t s);
 
 // gram_tc2.cu (bf16, tcgen05.cta_group::2: two CTAs per 256-row tile)
 cudaError_t launch_gram_tc2(ada_ctx* ctx, const GramProblem* tri, const GramProblem* cross,

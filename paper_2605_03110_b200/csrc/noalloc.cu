@@ -63,6 +63,8 @@ ada_status setup_device(int device, PerDevice** out) {
         c.tc2_attr_set = false;
         c.tc2_pairs = 0;
         c.ws = nullptr;
+        c.attn_ws = nullptr;
+        c.attn_ws_bytes = 0;
         c.stage = nullptr;
         c.stage_bytes = 0;
         c.host_stream = nullptr;
