@@ -324,6 +324,75 @@ def hbm_point(ada, dev, T, q, peaks, args):
             "l2": "256 MiB write before every call"}
 
 
+def overlap_bench(args, cfg):
+    """Section 8.4: the selection of layer l+1 on one stream while the nearest-representative map
+    and the attention on the representatives (Eq. 2) of layer l run on another.  The layers of
+    `cfg` stand in for Q, K, V (h heads of d/h); serial order on one stream against the two-stream
+    order, CUDA events around the whole chain, inputs resident in HBM.  Prints a table."""
+    import torch
+    from paper_2605_03110_b200 import binding as ada
+    from paper_2605_03110_b200.pipeline import SelectionAttentionPipeline
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    h = args.heads or 32
+    T, d, L = cfg.T, cfg.d, cfg.L
+    d_h = d // h
+    layers = [torch.from_numpy(lb.X[0].view(np.int16)).view(torch.bfloat16).to(dev).view(T, h, d_h)
+              for lb in wl.generate_layers(cfg, seed=0)]
+    outs = [torch.zeros((T, h, d_h), dtype=torch.float32, device=dev) for _ in range(2)]
+    pipe = SelectionAttentionPipeline(T, h, d_h, cfg.tau, dev)
+    out_of = lambda l: outs[l & 1]
+
+    def timed(fn):
+        for _ in range(max(2, args.warmup)):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / args.steps
+
+    st = torch.cuda.current_stream()
+
+    def selection_only():
+        for l in range(L):
+            pipe._select(l, layers[l], st)
+
+    def consumers_only():
+        for l in range(L):
+            pipe._consume(l, layers[l], out_of(l), st)
+
+    ms_sel = timed(selection_only)
+    ms_con = timed(consumers_only)            # on the sets the last selection pass left behind
+    ms_serial = timed(lambda: pipe.run(layers, [out_of(l) for l in range(L)], overlap=False))
+    ms_over = timed(lambda: pipe.run(layers, [out_of(l) for l in range(L)], overlap=True))
+    r_last = int(pipe.sets[(L - 1) % len(pipe.sets)].rep_out_cnt[0])
+    # the attention call alone, on the last layer's set (gather + Eq. 2 + expansion)
+    last = pipe.sets[(L - 1) % len(pipe.sets)]
+    X = layers[L - 1]
+    ms_att = timed(lambda: ada.ada_attention_reps(pipe.con, X, X, X, last.rep_out[0], last.rep_out_cnt,
+                                                  nearest_idx=pipe.near[0], out=outs[0]))
+    ms_att_reps = timed(lambda: ada.ada_attention_reps(pipe.con, X, X, X, last.rep_out[0], last.rep_out_cnt,
+                                                       out=outs[0]))
+    assert ada.ada_device_status(pipe.sel)[0] == 0 and ada.ada_device_status(pipe.con)[0] == 0
+    pipe.close()
+    print(f"workload configs[{cfg.cfg_id - 1}] {cfg.name}: T={T} d={d} L={L}, {h} heads of {d_h}; r at the last "
+          f"layer {r_last}; {args.steps} eager passes per figure (launches from Python)")
+    print("| chain | ms per L layers |")
+    print("|---|---|")
+    print(f"| selection alone (full + {L - 1} cascade steps) | {ms_sel:.3f} |")
+    print(f"| consumers alone (nearest-representative map + attention on the representatives, {L} layers) | {ms_con:.3f} |")
+    print(f"| both, one stream | {ms_serial:.3f} |")
+    print(f"| both, two streams (selection of layer l+1 beside the consumers of layer l) | {ms_over:.3f} |")
+    gf = 2 * 2.0 * r_last * r_last * d_h * h / 1e9
+    print(f"attention on the representatives alone, r = {r_last}: {ms_att_reps * 1e3:.1f} us without the expansion "
+          f"({gf:.1f} GFLOP in the two contractions of Eq. 2 -> {gf / ms_att_reps:.0f} TFLOP/s), "
+          f"{ms_att * 1e3:.1f} us with it ({T * d * 4 / 1e6:.0f} MB of fp32 output rows)")
+
+
 def heads_bench(args, cfg):
     """Per-head selection (Section 8.5) on the layers of `cfg` read as (T, h, d/h): the whole
     L-layer cascade pipeline with one representative set per head, beside the shared-set pipeline
@@ -426,6 +495,9 @@ def main():
     ap.add_argument("--sweep", action="store_true",
                     help="crossover sweep (configs[4]): full selection vs one cascade step per (T, r/T); "
                          "prints a table instead of the JSON line")
+    ap.add_argument("--overlap", action="store_true",
+                    help="selection / attention pipelining on two streams (Section 8.4) on --workload 3 or 4 "
+                         "(--heads h, default 32); prints a table instead of the JSON line")
     ap.add_argument("--causal", action="store_true",
                     help="cascade steps with ADA_CROSS_CAUSAL (line 8 restricted to s < t)")
     ap.add_argument("--no-cooperative", action="store_true",
@@ -439,6 +511,10 @@ def main():
                          "pipeline on --workload 3 or 4; prints a table instead of the JSON line")
     args = ap.parse_args()
 
+    if args.overlap:
+        cfg = wl.CONFIGS[args.workload]
+        overlap_bench(args, wl.scaled(cfg, L=args.layers) if args.layers else cfg)
+        return
     if args.heads:
         cfg = wl.CONFIGS[args.workload]
         heads_bench(args, wl.scaled(cfg, L=args.layers) if args.layers else cfg)

@@ -149,3 +149,35 @@ def test_error_paths(ada):
     with pytest.raises(TypeError):
         ada.ada_attention_reps(ctx, q.half(), q.half(), q.half(), idx, cnt)
     ada.ada_destroy(ctx)
+
+
+def test_two_stream_pipeline_matches_the_serial_order(ada):
+    """Section 8.4: selection of layer l+1 on one stream while layer l's nearest-representative map
+    and attention run on another; the results are those of the serial order, bit for bit."""
+    from paper_2605_03110_b200.pipeline import SelectionAttentionPipeline
+    cfg = wl.scaled(wl.CONFIGS[3], T=1024, d=1024, L=5, P=100, rho=0.05)
+    dev = torch.device("cuda", 0)
+    T, h, d_h = cfg.T, 8, cfg.d // 8
+    layers = [torch.from_numpy(lb.X[0].view(np.int16)).view(torch.bfloat16).to(dev).view(T, h, d_h)
+              for lb in wl.generate_layers(cfg, seed=0)]
+    pipe = SelectionAttentionPipeline(T, h, d_h, cfg.tau, dev)
+    res = []
+    for overlap in (False, True, True):
+        outs = [torch.zeros((T, h, d_h), dtype=torch.float32, device=dev) for _ in layers]
+        pipe.run(layers, outs, overlap=overlap)
+        torch.cuda.synchronize()
+        res.append(outs)
+    for a, b, c in zip(*res):
+        assert torch.equal(a, b) and torch.equal(a, c)
+        assert float(a.abs().max()) > 0.0
+    assert ada.ada_device_status(pipe.sel)[0] == 0 and ada.ada_device_status(pipe.con)[0] == 0
+    # against the oracle at the last layer: the chain of sets, then Eq. 2 with the device's map
+    R = None
+    for l, lb in enumerate(wl.generate_layers(cfg, seed=0)):
+        X64 = wl.as_f64(lb.X[0])
+        R = oracle.select_full(X64, cfg.tau)[0] if l == 0 else oracle.cascade_step(X64, cfg.tau, R).rep
+    near = pipe.near[0].cpu().numpy()
+    Xh = X64.reshape(T, h, d_h)
+    ref = oracle.attention_reps(Xh, Xh, Xh, R, nearest_idx=near)
+    assert np.max(np.abs(res[1][-1].cpu().numpy() - ref)) <= 2.0 ** -8 * float(np.max(np.abs(X64)))
+    pipe.close()
