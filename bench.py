@@ -268,6 +268,8 @@ def hbm_point(ada, dev, T, q, peaks, args):
     X0, X1 = [torch.from_numpy(lb.X.view(np.int16)).view(torch.bfloat16).to(dev)
               for lb in wl.generate_layers(cfg, seed=0)]
     ctx = ada.ada_create(1, T, cfg.d, ada.ADA_BF16, device=dev.index or 0)
+    if args.no_cooperative:
+        ada.ada_set_cooperative(ctx, False)
     idx, cnt, _ = ada.ada_select_full(ctx, X0, cfg.tau, want_gamma=False)
     out = ada.CascadeOut(1, T, dev, want_gamma=False)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
@@ -495,6 +497,8 @@ def main():
     ap.add_argument("--sweep", action="store_true",
                     help="crossover sweep (configs[4]): full selection vs one cascade step per (T, r/T); "
                          "prints a table instead of the JSON line")
+    ap.add_argument("--hbm-only", action="store_true",
+                    help="only the two HBM-bound cross-Gram points (one JSON line each)")
     ap.add_argument("--overlap", action="store_true",
                     help="selection / attention pipelining on two streams (Section 8.4) on --workload 3 or 4 "
                          "(--heads h, default 32); prints a table instead of the JSON line")
@@ -511,6 +515,13 @@ def main():
                          "pipeline on --workload 3 or 4; prints a table instead of the JSON line")
     args = ap.parse_args()
 
+    if args.hbm_only:
+        import torch
+        from paper_2605_03110_b200 import binding as ada
+        torch.cuda.set_device(0)
+        for Tq in (16384, 8192):
+            print(json.dumps(hbm_point(ada, torch.device("cuda", 0), Tq, 0.01, measured_peaks(), args)))
+        return
     if args.overlap:
         cfg = wl.CONFIGS[args.workload]
         overlap_bench(args, wl.scaled(cfg, L=args.layers) if args.layers else cfg)
