@@ -177,6 +177,9 @@ ada_status ada_create(ada_ctx** out, int device, int64_t maxB, int64_t maxT, int
     const size_t o_inv = take(n_tok * 4), o_invr = take(n_tok * 4);
     const size_t o_reff = take((size_t)maxB * 4), o_stat = take(32), o_thr = take((size_t)maxB * 4);
     const size_t o_xrep = take(n_tok * (size_t)maxd * ctx->es + 1024);
+    // bf16: the rows outside a large inherited set, copied out for the cross step (Algorithm 1 line 6)
+    const size_t o_ntok = take(dt == ADA_BF16 ? n_tok * 4 : 0);
+    const size_t o_xnon = take(dt == ADA_BF16 ? n_tok * (size_t)maxd * 2 + 1024 : 0);
     const size_t split_bytes = dt == ADA_F32 ? n_tok * (size_t)maxd * 12 + 1024 : 0;
     const size_t o_sxa = take(split_bytes), o_sxb = take(split_bytes), o_sra = take(split_bytes),
                  o_srb = take(split_bytes);
@@ -199,6 +202,8 @@ ada_status ada_create(ada_ctx** out, int device, int64_t maxB, int64_t maxT, int
     ctx->agg_stride = agg_stride;
     ctx->near_key = reinterpret_cast<unsigned long long*>(ctx->ws + o_near);
     ctx->Xrep = ctx->ws + o_xrep;
+    ctx->Xnon = dt == ADA_BF16 ? ctx->ws + o_xnon : nullptr;
+    ctx->non_tok = dt == ADA_BF16 ? reinterpret_cast<int32_t*>(ctx->ws + o_ntok) : nullptr;
     ctx->splitXA = split_bytes ? ctx->ws + o_sxa : nullptr;
     ctx->splitXB = split_bytes ? ctx->ws + o_sxb : nullptr;
     ctx->splitRA = split_bytes ? ctx->ws + o_sra : nullptr;
@@ -388,6 +393,7 @@ static ada_status cascade_impl(ada_ctx* ctx, const void* X, int64_t B, int64_t T
     gj.rep_in = rep_in; gj.rep_in_cnt = rep_in_cnt;
     gj.role = ctx->role; gj.r_eff = ctx->r_eff; gj.Xrep = ctx->Xrep; gj.inv_rep = ctx->inv_rep;
     gj.T = (int)T; gj.d = (int)d; gj.B = (int)B;
+    gj.Xnon = ctx->Xnon; gj.non_tok = ctx->non_tok; gj.inv_norm = ctx->inv_norm;
     if (split)   // 1/||x|| of all rows; bf16 terms of X and of the gathered rows
         CU(launch_split(ctx, X, (int)B, (int)T, (int)d, ldx, xb, true, s));
     // lines 3-4: r x r Gram among inherited reps, max over earlier ones

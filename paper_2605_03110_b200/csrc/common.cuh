@@ -101,6 +101,11 @@ struct GatherJob {
     void* Xrep;               // [B*T][d]
     float* inv_rep;           // [B*T] by position
     int T, d, B;
+    // line 6's row set as a matrix of its own, made when the inherited set is large (see
+    // gather_rows): rows outside the set in token order, their token indices, 1/||x_t|| by token
+    void* Xnon;               // [B*T][d], or NULL: never
+    int32_t* non_tok;         // [B*T]
+    float* inv_norm;          // [B*T]
 };
 
 // Row norms computed inside a tensor-core Gram launch by four extra warps per CTA
@@ -156,6 +161,8 @@ struct ada_ctx {
     int agg_stride;
     unsigned long long* near_key;  // [maxB*maxT] packed (value, ~column) of the nearest representative
     void* Xrep;          // [maxB*maxT*maxd] gathered representative rows (raw values)
+    void* Xnon;          // [maxB*maxT*maxd] bf16 contexts: the rows outside a large inherited set
+    int32_t* non_tok;    // [maxB*maxT] their token indices
     // fp32 contexts: three-term bf16 splits laid out for one contraction of length 6d
     void *splitXA, *splitXB;   // [maxB*maxT][6 maxd] of X
     void *splitRA, *splitRB;   // same, of the gathered representative rows

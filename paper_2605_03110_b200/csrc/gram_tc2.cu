@@ -126,8 +126,13 @@ __device__ __forceinline__ void cross_cols(const GramProblem& p, int n, int& nct
     if (nct == 0 && p.inv_out != nullptr && n == 0) nct = 1;
     w = nct > 0 ? max(32, (((n + nct - 1) / nct) + 31) & ~31) : 0;    // each CTA holds w/2 columns: keep w/2 a multiple of 16
 }
+// rows of the cross segment's left operand for a sequence with n inherited tokens: all of
+// X, or only the tokens outside the inherited set when those were copied out (compact)
+__device__ __forceinline__ int cross_rows(const GramProblem& p, int n, bool compact) {
+    return compact ? p.rows - n : p.rows;
+}
 // hrows: rows of the left operand per CTA in cross tiles (128, or fewer in the streaming form)
-__device__ __forceinline__ int seg_tiles(const GramProblem& p, int hrows) {
+__device__ __forceinline__ int seg_tiles(const GramProblem& p, int hrows, bool compact) {
     int total = 0;
     for (int b = 0; b < p.B; ++b) {
         const int n = seq_n(p, b);
@@ -135,19 +140,19 @@ __device__ __forceinline__ int seg_tiles(const GramProblem& p, int hrows) {
         else {
             int nct, w;
             cross_cols(p, n, nct, w);
-            total += ((p.rows + 2 * hrows - 1) / (2 * hrows)) * nct;
+            total += ((cross_rows(p, n, compact) + 2 * hrows - 1) / (2 * hrows)) * nct;
         }
     }
     return total;
 }
-__device__ __forceinline__ bool decode_tile(const GramProblem& p, int hrows, int id, Piece& t) {
+__device__ __forceinline__ bool decode_tile(const GramProblem& p, int hrows, bool compact, int id, Piece& t) {
     for (int b = 0; b < p.B; ++b) {
         const int n = seq_n(p, b);
         int cnt = 0, nct = 0, w = 0;
         if (p.tri) cnt = n > 0 ? tri_tiles(n) : 0;
         else {
             cross_cols(p, n, nct, w);
-            cnt = ((p.rows + 2 * hrows - 1) / (2 * hrows)) * nct;
+            cnt = ((cross_rows(p, n, compact) + 2 * hrows - 1) / (2 * hrows)) * nct;
         }
         if (id >= cnt) { id -= cnt; continue; }
         t.b = b;
@@ -164,7 +169,7 @@ __device__ __forceinline__ bool decode_tile(const GramProblem& p, int hrows, int
         } else {
             t.row0 = (id / nct) * 2 * hrows;
             t.col0 = (id % nct) * w;
-            t.m = p.rows;
+            t.m = cross_rows(p, n, compact);
             nc = min(n - t.col0, w);
         }
         t.ncols = max(32, (nc + 31) & ~31);
@@ -198,14 +203,17 @@ __device__ __forceinline__ bool norm_duty(const GramProblem& p, const Piece& pc,
 // tile's last row has no admissible (row, column) pair: every role skips it, so neither
 // its loads nor its MMAs are issued.  Column tokens ascend with the column index.  (A tile
 // that has to yield row norms is never skipped.)
-__device__ __forceinline__ bool dead_tile(const GramProblem& p, const Piece& pc, int hrows, bool from_smem) {
+__device__ __forceinline__ bool dead_tile(const GramProblem& p, const Piece& pc, int hrows, bool from_smem,
+                                          bool compact) {
     if (p.tri || !p.causal || p.col_token == nullptr || pc.n <= 0 || norm_duty(p, pc, from_smem)) return false;
+    if (compact) return false;     // rows are compacted there: a row index is not a token index
     return p.col_token[(int64_t)pc.b * p.cap + pc.col0] >= pc.row0 + 2 * hrows;
 }
 
 struct GramMaps {
     CUtensorMap a[2], b[2];
     CUtensorMap ah;          // left operand of the cross segment in boxes of hb_rows rows
+    CUtensorMap an;          // the rows outside a large inherited set (Xnon), 128-row boxes
 };
 
 // ---------------------------------------------------------------- the kernel
@@ -218,7 +226,7 @@ struct alignas(16) SharedPair {
     unsigned long long drain;
     unsigned tmem_base;
     int abort_flag;
-    int tiles0, tiles1, hrows, one_col_tile;
+    int tiles0, tiles1, hrows, one_col_tile, compact;
     unsigned norm_cnt[MAX_STAGES];             // norm warps done with a stage
     // per epilogue warp, so that staging needs no barrier across warps
     alignas(16) float col_scale[4][BN];
@@ -277,10 +285,19 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
         if (one)
             for (int b = 0; b < cx.B; ++b) one = one && seq_n(cx, b) <= BN;
         if (one && cx.hb_rows > 0 && cx.hb_rows < BM) hrows = cx.hb_rows;
+        // a large inherited set (two fifths of the tokens or more, in every sequence) of a long
+        // sequence: the rows outside it are copied out by the gather and the cross tiles run over
+        // those only.  (Measured on the crossover sweep at r/T = 0.5: 1052 -> 699 us at T = 16384,
+        // 250 -> 217 us at T = 8192, but 87 -> 97 us at T = 4096, where the copy costs more than
+        // the saved tiles.)
+        bool compact = !cx.tri && !one && gather.X != nullptr && gather.Xnon != nullptr && cx.rows >= 8192;
+        if (compact)
+            for (int b = 0; b < cx.B; ++b) compact = compact && 5 * (int64_t)seq_n(cx, b) >= 2 * (int64_t)cx.rows;
         sh.hrows = hrows;
         sh.one_col_tile = one ? 1 : 0;
-        sh.tiles0 = seg_tiles(seg0, hrows);
-        sh.tiles1 = nseg > 1 ? seg_tiles(seg1, hrows) : 0;
+        sh.compact = compact ? 1 : 0;
+        sh.tiles0 = seg_tiles(seg0, hrows, compact);
+        sh.tiles1 = nseg > 1 ? seg_tiles(seg1, hrows, compact) : 0;
     }
     tcgen05_fence_before();
     __syncthreads();
@@ -290,6 +307,7 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
     const int tiles0 = sh.tiles0, total = sh.tiles0 + sh.tiles1;
     const int hrows = sh.hrows;                          // rows per CTA of a cross tile
     const bool smem_norms = sh.one_col_tile != 0;        // row norms out of the tiles in shared memory
+    const bool compact = sh.compact != 0;                // cross tiles over the copied-out rows (Xnon)
     // the helper warps AND the epilogue warps (idle until the first tile is done) share the gather
     constexpr int GATHER_WARPS = NORM_WARPS + 4;
     const unsigned gather_total = (unsigned)(gridDim.x * GATHER_WARPS);
@@ -312,8 +330,8 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
             for (int id = pair; ok && id < total; id += npairs) {
                 const int sg = id < tiles0 ? 0 : 1;
                 const GramProblem& p = sg ? seg1 : seg0;
-                if (!decode_tile(p, hrows, id - (sg ? tiles0 : 0), pc)) break;
-                if (dead_tile(p, pc, hrows, smem_norms)) continue;   // causal cross tile with no admissible pair
+                if (!decode_tile(p, hrows, compact, id - (sg ? tiles0 : 0), pc)) break;
+                if (dead_tile(p, pc, hrows, smem_norms, compact)) continue;   // causal cross tile with no admissible pair
                 const int num_kb = (p.d + BKS - 1) / BKS;
                 const int half = pc.ncols >> 1;
                 const int nbox = (half + BOX_N - 1) / BOX_N;
@@ -322,7 +340,7 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
                 const int subb = sub_bytes_pair(a_bytes, pc.ncols);
                 const int sb = KSUB * subb;
                 const unsigned tx = (unsigned)(KSUB * (arows * 128 + nbox * BOX_BYTES));
-                const CUtensorMap* amap = (!p.tri && hrows != BM) ? &maps.ah : &maps.a[sg];
+                const CUtensorMap* amap = p.tri ? &maps.a[sg] : (compact ? &maps.an : (hrows != BM ? &maps.ah : &maps.a[sg]));
                 if (sb != cur_sb) {
                     for (int q = 0; q < cur_nst && ok; ++q)
                         if ((used >> q) & 1u)
@@ -370,8 +388,8 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
             for (int id = pair; ok && id < total; id += npairs) {
                 const int sg = id < tiles0 ? 0 : 1;
                 const GramProblem& p = sg ? seg1 : seg0;
-                if (!decode_tile(p, hrows, id - (sg ? tiles0 : 0), pc)) break;
-                if (dead_tile(p, pc, hrows, smem_norms)) continue;   // causal cross tile with no admissible pair
+                if (!decode_tile(p, hrows, compact, id - (sg ? tiles0 : 0), pc)) break;
+                if (dead_tile(p, pc, hrows, smem_norms, compact)) continue;   // causal cross tile with no admissible pair
                 const int num_kb = (p.d + BKS - 1) / BKS;
                 const int a_bytes = a_bytes_of(p.tri ? BM : hrows);
                 const int subb = sub_bytes_pair(a_bytes, pc.ncols);
@@ -425,7 +443,7 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
         const unsigned norm_total = (unsigned)(gridDim.x * NORM_WARPS);
         if (has_gather)               // Algorithm 1 lines 1-2, shared with the helper warps
             gather_rows(gather, blockIdx.x * GATHER_WARPS + NORM_WARPS + (warp - 2), gridDim.x * GATHER_WARPS,
-                        lane, dep_ctr + 3, status);
+                        lane, dep_ctr + 3, status, compact);
         // the accumulator goes back to the leader's barrier
         const unsigned empty_addr[2] = {map_to_cta(smem_u32(&sh.tmem_empty[0]), 0),
                                         map_to_cta(smem_u32(&sh.tmem_empty[1]), 0)};
@@ -433,8 +451,8 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
         for (int id = pair; id < total; id += npairs) {
             const int sg = id < tiles0 ? 0 : 1;
             const GramProblem& p = sg ? seg1 : seg0;
-            if (!decode_tile(p, hrows, id - (sg ? tiles0 : 0), pc)) break;
-            if (dead_tile(p, pc, hrows, smem_norms)) continue;   // causal cross tile with no admissible pair
+            if (!decode_tile(p, hrows, compact, id - (sg ? tiles0 : 0), pc)) break;
+            if (dead_tile(p, pc, hrows, smem_norms, compact)) continue;   // causal cross tile with no admissible pair
             const unsigned acc = tile_it & 1u, acc_ph = (tile_it >> 1) & 1u;
             ++tile_it;
             const int64_t o = (int64_t)pc.b * p.cap;
@@ -496,6 +514,8 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
             const int row_base = pc.row0 + (int)rank * arows;
             const int row = row_base + lrow;
             const bool row_live = lrow < arows && row < pc.m;
+            // the token this row belongs to: the row index itself, except over the copied-out rows
+            const int tokrow = (compact && !p.tri && row_live) ? __ldcg(gather.non_tok + o + row) : row;
             const bool defer = !p.tri && p.defer_row != 0;   // the row's own factor is applied later
             // inherited reps are not candidates (with a deferred factor the compaction ignores them)
             const bool skip = row_live && !p.tri && !defer && p.row_role[o + row] != 0;
@@ -523,7 +543,7 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
                         const float x = fabsf(v[j]) * cs[c0 + j];
-                        if (ct[c0 + j] < row) mx = fmaxf(mx, x);
+                        if (ct[c0 + j] < tokrow) mx = fmaxf(mx, x);
                     }
                 }
             }
@@ -538,7 +558,7 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
                 if (!skip) {
                     if (!defer && !inv_early) inv_row = __ldcg(p.inv_a + o + row);
                     mx *= inv_row;
-                    if (mx > 0.f) atomicMax(p.out + o + row, __float_as_uint(mx));
+                    if (mx > 0.f) atomicMax(p.out + o + tokrow, __float_as_uint(mx));
                 }
             }
             if (sg == 0 && nseg > 1) {
@@ -555,10 +575,10 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
                       dep_ctr + 1, status);
         if (has_gather)               // Algorithm 1 lines 1-2
             gather_rows(gather, blockIdx.x * GATHER_WARPS + (warp - 6), gridDim.x * GATHER_WARPS, lane,
-                        dep_ctr + 3, status);
+                        dep_ctr + 3, status, compact);
         if (warp == 6 && lane == 0) TRACE(2);
         const GramProblem& cx = (nseg > 1) ? seg1 : seg0;
-        if (!cx.tri && cx.inv_out != nullptr && !smem_norms) {
+        if (!cx.tri && cx.inv_out != nullptr && !smem_norms && !compact) {
             // several column tiles: 1/||x_t|| of every row with plain loads, behind the main loops
             // (nothing in this launch waits for them: the row factor is applied by the compaction)
             NormJob nj;
@@ -577,8 +597,8 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
             for (int id = pair; ok && id < total; id += npairs) {
                 const int sg = id < tiles0 ? 0 : 1;
                 const GramProblem& p = sg ? seg1 : seg0;
-                if (!decode_tile(p, hrows, id - (sg ? tiles0 : 0), pc)) break;
-                if (dead_tile(p, pc, hrows, smem_norms)) continue;
+                if (!decode_tile(p, hrows, compact, id - (sg ? tiles0 : 0), pc)) break;
+                if (dead_tile(p, pc, hrows, smem_norms, compact)) continue;
                 const int num_kb = (p.d + BKS - 1) / BKS;
                 const int arows = p.tri ? BM : hrows;
                 const int a_bytes = a_bytes_of(arows);
@@ -720,6 +740,10 @@ cudaError_t launch_gram_tc2(ada_ctx* ctx, const GramProblem* tri, const GramProb
     if (nseg == 0) return cudaSuccess;
     if (nseg == 1) { maps.a[1] = maps.a[0]; maps.b[1] = maps.b[0]; segs[1] = segs[0]; segs[1].B = 0; }
     if (segs[0].tri && nseg == 1) maps.ah = maps.a[0];
+    maps.an = maps.ah;
+    if (gather != nullptr && gather->Xnon != nullptr && cross != nullptr &&
+        !make_map(&maps.an, gather->Xnon, cross->d, cross->rows, cross->B, cross->d, (int64_t)cross->cap * cross->d, BM))
+        return cudaErrorInvalidValue;
     NormJob nj;
     memset(&nj, 0, sizeof(nj));
     if (norms != nullptr) nj = *norms;

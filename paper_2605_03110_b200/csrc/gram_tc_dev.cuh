@@ -346,10 +346,39 @@ static __device__ __forceinline__ bool wait_counter_1(const unsigned* counter, u
 // goes to Xrep[b, i] and its inverse norm to inv_rep[b, i]; a rejected entry gets inverse norm
 // 0 (its column then counts for nothing) and raises the status.  Ends with one arrival per warp
 // on `counter`.
+// one warp: copy a row of nvec 16-byte vectors, return its sum of squares (all lanes)
+static __device__ __forceinline__ float copy_row_sumsq(const uint4* __restrict__ src, uint4* __restrict__ dst,
+                                                       int nvec, int lane) {
+    float ss = 0.f;
+    int v = lane;
+    for (; v + 480 < nvec; v += 512) {            // sixteen loads in flight per lane
+        uint4 x[16];
+#pragma unroll
+        for (int q = 0; q < 16; ++q) x[q] = __ldg(src + v + 32 * q);
+#pragma unroll
+        for (int q = 0; q < 16; ++q) { ss += sumsq_bf16x8(x[q]); dst[v + 32 * q] = x[q]; }
+    }
+    for (; v < nvec; v += 32) {
+        const uint4 x = __ldg(src + v);
+        ss += sumsq_bf16x8(x);
+        dst[v] = x;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    return ss;
+}
+
+// `compact`: also Algorithm 1 line 6's row set as a matrix of its own.  Line 6 builds the
+// cross-Gram from the (T - r) tokens OUTSIDE the inherited set; when the set is large, streaming
+// all T rows and masking the inherited ones wastes r/T of the loads and MMAs, so the rows
+// between consecutive inherited tokens are copied, in order, to Xnon (row t goes to t minus the
+// number of inherited tokens before it), with their token index in non_tok and 1/||x_t|| in
+// inv_norm.  A warp takes one gap between two list entries at a time.
 static __device__ __forceinline__ void gather_rows(const GatherJob& gj, int g, int nw, int lane,
-                                            unsigned* counter, unsigned* status) {
+                                            unsigned* counter, unsigned* status, bool compact) {
     const __nv_bfloat16* X = reinterpret_cast<const __nv_bfloat16*>(gj.X);
     __nv_bfloat16* Xrep = reinterpret_cast<__nv_bfloat16*>(gj.Xrep);
+    __nv_bfloat16* Xnon = reinterpret_cast<__nv_bfloat16*>(gj.Xnon);
     const int nvec = gj.d >> 3;
     int b = 0;
     int64_t item = g;
@@ -367,10 +396,34 @@ static __device__ __forceinline__ void gather_rows(const GatherJob& gj, int g, i
             cnt = cnt < 0 ? 0 : gj.T;
         }
         if (g == 0 && lane == 0) gj.r_eff[b] = cnt;
-        if (item >= cnt) { item -= cnt; ++b; continue; }
+        const int n_items = compact ? 2 * cnt + 1 : cnt;     // list entries, then the gaps around them
+        if (item >= n_items) { item -= n_items; ++b; continue; }
         const int i = (int)item;
-        item += nw;                                   // this warp's next entry (maybe in a later sequence)
+        item += nw;                                   // this warp's next item (maybe in a later sequence)
         const int32_t* list = gj.rep_in + (int64_t)b * gj.T;
+        if (i >= cnt) {
+            // gap number gp: the tokens after entry gp - 1 and before entry gp
+            const int gp = i - cnt;
+            int lo = gp > 0 ? list[gp - 1] + 1 : 0;
+            int hi = gp < cnt ? list[gp] : gj.T;
+            lo = max(lo, 0); hi = min(hi, gj.T);      // (a bad list is reported by the entries' check)
+            for (int t = lo; t < hi; ++t) {
+                const int dstrow = t - gp;
+                if (dstrow < 0 || dstrow >= gj.T) continue;
+                const uint4* src = reinterpret_cast<const uint4*>(X + (int64_t)b * gj.xb + (int64_t)t * gj.ldx);
+                uint4* dst = reinterpret_cast<uint4*>(Xnon + ((int64_t)b * gj.T + dstrow) * (int64_t)gj.d);
+                const float ss = copy_row_sumsq(src, dst, nvec, lane);
+                if (lane == 0) {
+                    float inv = 0.f;
+                    if (!(ss <= 3.0e38f)) atomicOr(status, ST_NONFINITE);
+                    else if (ss > 0.f) inv = 1.0f / sqrtf(ss);
+                    else atomicAdd(status + 1, 1u);
+                    gj.inv_norm[(int64_t)b * gj.T + t] = inv;
+                    gj.non_tok[(int64_t)b * gj.T + dstrow] = t;
+                }
+            }
+            continue;
+        }
         const bool spec = b == 0 && i == g;
         const int32_t idx = spec ? first_idx : list[i];
         bool ok = idx >= 0 && idx < gj.T;
@@ -382,22 +435,7 @@ static __device__ __forceinline__ void gather_rows(const GatherJob& gj, int g, i
         }
         const uint4* src = reinterpret_cast<const uint4*>(X + (int64_t)b * gj.xb + (int64_t)idx * gj.ldx);
         uint4* dst = reinterpret_cast<uint4*>(Xrep + prow * (int64_t)gj.d);
-        float ss = 0.f;
-        int v = lane;
-        for (; v + 480 < nvec; v += 512) {            // sixteen loads in flight per lane
-            uint4 x[16];
-#pragma unroll
-            for (int q = 0; q < 16; ++q) x[q] = __ldg(src + v + 32 * q);
-#pragma unroll
-            for (int q = 0; q < 16; ++q) { ss += sumsq_bf16x8(x[q]); dst[v + 32 * q] = x[q]; }
-        }
-        for (; v < nvec; v += 32) {
-            const uint4 x = __ldg(src + v);
-            ss += sumsq_bf16x8(x);
-            dst[v] = x;
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        const float ss = copy_row_sumsq(src, dst, nvec, lane);
         if (lane == 0) {
             gj.inv_rep[prow] = (ss <= 3.0e38f && ss > 0.f) ? 1.0f / sqrtf(ss) : 0.f;
             gj.role[(int64_t)b * gj.T + idx] = i + 1;

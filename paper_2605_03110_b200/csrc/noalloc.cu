@@ -83,6 +83,8 @@ ada_status setup_device(int device, PerDevice** out) {
         c.r_eff = nullptr;
         c.thr_seq = nullptr;
         c.Xrep = nullptr;
+        c.Xnon = nullptr;
+        c.non_tok = nullptr;
         c.near_key = nullptr;
         c.splitXA = c.splitXB = c.splitRA = c.splitRB = nullptr;
         pd.setup_status = ADA_OK;
