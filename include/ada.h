@@ -103,6 +103,15 @@ ada_status ada_set_engine(ada_ctx* ctx, ada_engine e);
  * launches.  Default: on. */
 ada_status ada_set_cooperative(ada_ctx* ctx, int on);
 
+/* Algorithm 1 line 6 forms the cross-Gram from the tokens OUTSIDE the inherited set.  On the
+ * pair-CTA kernel, when the inherited set holds two fifths of a sequence's tokens or more, the
+ * rows outside it are copied out in token order inside the launch and the cross tiles run over
+ * those rows only, instead of streaming all T rows and discarding the inherited ones -- for
+ * sequences of at least `min_rows` tokens (default 8192: below that the copy was measured to
+ * cost more than the tiles it saves).  Results do not depend on it.  min_rows >= 1;
+ * a huge value turns it off. */
+ada_status ada_set_row_compaction(ada_ctx* ctx, int64_t min_rows);
+
 /* Programmatic dependent launch of the library's kernels (on by default).  When on, every
  * kernel is launched with the stream-serialization attribute and begins with a grid-dependency
  * wait, so that its blocks can be placed, and its set-up that reads nothing (barriers, TMEM

@@ -28,7 +28,7 @@ SYMBOLS = [
     "ada_device_status", "ada_profile_enable", "ada_profile_read", "ada_status_string",
     "ada_select_full_noalloc", "ada_set_cooperative", "ada_selftest_wait_timeout", "ada_nearest_rep",
     "ada_select_full_heads", "ada_cascade_step_heads", "ada_set_dependent_launch",
-    "ada_cascade_step_adaptive", "ada_attention_reps",
+    "ada_cascade_step_adaptive", "ada_attention_reps", "ada_set_row_compaction",
 ]
 ADA_NOALLOC_MAX_T = 16384
 
@@ -61,6 +61,7 @@ def lib() -> C.CDLL:
         L.ada_set_engine.argtypes = [vp, C.c_int]
         L.ada_set_cooperative.argtypes = [vp, C.c_int]
         L.ada_set_dependent_launch.argtypes = [vp, C.c_int]
+        L.ada_set_row_compaction.argtypes = [vp, i64]
         L.ada_selftest_wait_timeout.argtypes = [vp, C.c_int, vp]
         L.ada_normalize.argtypes = [vp, vp, i64, i64, i64, i64, C.c_int, vp, fp, i32p, i32p, vp, vp]
         L.ada_select_full.argtypes = [vp, vp, i64, i64, i64, i64, C.c_int, C.c_double, i32p, i32p,
@@ -168,6 +169,11 @@ def ada_set_engine(ctx: Context, engine: int) -> None:
 
 def ada_set_cooperative(ctx: Context, on: bool) -> None:
     _check(lib().ada_set_cooperative(ctx.h, int(bool(on))), "ada_set_cooperative")
+
+
+def ada_set_row_compaction(ctx: Context, min_rows: int) -> None:
+    """Sequence length from which a large inherited set's complement is copied out for the cross step."""
+    _check(lib().ada_set_row_compaction(ctx.h, int(min_rows)), "ada_set_row_compaction")
 
 
 def ada_set_dependent_launch(ctx: Context, on: bool) -> None:

@@ -163,6 +163,7 @@ ada_status ada_create(ada_ctx** out, int device, int64_t maxB, int64_t maxT, int
     ctx->dep_launch = true;
     ctx->tc2_attr_set = false;
     ctx->tc2_pairs = 0;
+    ctx->compact_min_rows = 8192;
     cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
 
     const size_t n_tok = (size_t)maxB * (size_t)maxT;
@@ -241,6 +242,12 @@ ada_status ada_set_engine(ada_ctx* ctx, ada_engine e) {
     if ((e == ADA_ENGINE_TCGEN05 || e == ADA_ENGINE_TCGEN05_PAIR) && !gram_tc_available())
         return ADA_ERR_UNSUPPORTED;
     ctx->engine = e;
+    return ADA_OK;
+}
+
+ada_status ada_set_row_compaction(ada_ctx* ctx, int64_t min_rows) {
+    if (ctx == nullptr || min_rows < 1) return ADA_ERR_INVALID_ARG;
+    ctx->compact_min_rows = min_rows > 0x7fffffff ? 0x7fffffff : (int)min_rows;
     return ADA_OK;
 }
 
@@ -394,6 +401,7 @@ static ada_status cascade_impl(ada_ctx* ctx, const void* X, int64_t B, int64_t T
     gj.role = ctx->role; gj.r_eff = ctx->r_eff; gj.Xrep = ctx->Xrep; gj.inv_rep = ctx->inv_rep;
     gj.T = (int)T; gj.d = (int)d; gj.B = (int)B;
     gj.Xnon = ctx->Xnon; gj.non_tok = ctx->non_tok; gj.inv_norm = ctx->inv_norm;
+    gj.compact_min_rows = ctx->compact_min_rows;
     if (split)   // 1/||x|| of all rows; bf16 terms of X and of the gathered rows
         CU(launch_split(ctx, X, (int)B, (int)T, (int)d, ldx, xb, true, s));
     // lines 3-4: r x r Gram among inherited reps, max over earlier ones

@@ -106,6 +106,7 @@ struct GatherJob {
     void* Xnon;               // [B*T][d], or NULL: never
     int32_t* non_tok;         // [B*T]
     float* inv_norm;          // [B*T]
+    int compact_min_rows;     // sequences shorter than this never use it
 };
 
 // Row norms computed inside a tensor-core Gram launch by four extra warps per CTA
@@ -143,6 +144,7 @@ struct ada_ctx {
     bool tc_attr_set;
     bool cooperative;    // fused launches use the cooperative attribute
     bool dep_launch;     // kernels are launched with programmatic stream serialization
+    int compact_min_rows;  // sequence length from which a large inherited set's complement is copied out
     bool tc2_attr_set;   // pair-CTA kernel configured
     int tc2_pairs;       // clusters of two that fit on the device at once
     // device workspace

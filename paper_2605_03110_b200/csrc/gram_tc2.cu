@@ -290,7 +290,7 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
         // those only.  (Measured on the crossover sweep at r/T = 0.5: 1052 -> 699 us at T = 16384,
         // 250 -> 217 us at T = 8192, but 87 -> 97 us at T = 4096, where the copy costs more than
         // the saved tiles.)
-        bool compact = !cx.tri && !one && gather.X != nullptr && gather.Xnon != nullptr && cx.rows >= 8192;
+        bool compact = !cx.tri && !one && gather.X != nullptr && gather.Xnon != nullptr && cx.rows >= gather.compact_min_rows;
         if (compact)
             for (int b = 0; b < cx.B; ++b) compact = compact && 5 * (int64_t)seq_n(cx, b) >= 2 * (int64_t)cx.rows;
         sh.hrows = hrows;

@@ -60,6 +60,7 @@ ada_status setup_device(int device, PerDevice** out) {
         c.tc_attr_set = false;
         c.cooperative = true;
         c.dep_launch = false;          // plain stream order between this call's launches
+        c.compact_min_rows = 0x7fffffff;
         c.tc2_attr_set = false;
         c.tc2_pairs = 0;
         c.ws = nullptr;

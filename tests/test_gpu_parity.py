@@ -589,3 +589,55 @@ def test_dependent_launch_on_and_off_give_identical_results(ada, cfg_id):
     assert len(res[0]) == len(res[1])
     for a, b in zip(*res):
         assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("T,d", [(130, 72), (257, 768), (600, 8), (1500, 256)])
+def test_row_compaction_of_the_cross_step_small_shapes(ada, T, d):
+    """Algorithm 1 line 6 over the copied-out rows (pair kernel, forced on at any length):
+    inherited sets of two fifths of the tokens and more, literal and causal, against the oracle."""
+    from parity import check_cascade
+    ctx = ada.ada_create(1, T, d, ada.ADA_BF16)
+    ada.ada_set_engine(ctx, ada.ADA_ENGINE_TCGEN05_PAIR)
+    ada.ada_set_row_compaction(ctx, 1)
+    X = clustered(T, d, 4000 + T + d, "bf16")
+    rng = np.random.default_rng(T + d)
+    sets = [list(range(T)), list(range(0, T, 2)), list(range(1, T, 2)), list(range(T // 2, T)),
+            list(range(0, T // 2 + 1)), sorted(rng.choice(T, (T * 3) // 5, replace=False).tolist()),
+            list(range(0, T, 3))]                      # the last one is below the threshold: streamed
+    for R in sets:
+        for causal in (False, True):
+            check_cascade(ctx, X, TAU, [R], causal=causal)
+    ada.ada_destroy(ctx)
+
+
+def test_row_compaction_batched_and_on_and_off_agree(ada):
+    """Several sequences with different large sets in one call; the lists and gammas with the
+    row compaction on and off are identical bit for bit (it changes which rows are loaded, not
+    what is computed for them)."""
+    from parity import check_cascade, to_device
+    cfg = wl.scaled(wl.CONFIGS[2], B=3, T=700, d=264, L=2)
+    Xs, _ = wl.generate_all(cfg)
+    rng = np.random.default_rng(9)
+    Rs = [sorted(rng.choice(cfg.T, n, replace=False).tolist()) for n in (300, 699, 420)]
+    outs = []
+    for min_rows in (1, 1 << 30):
+        ctx = ada.ada_create(3, cfg.T, cfg.d, ada.ADA_BF16)
+        ada.ada_set_engine(ctx, ada.ADA_ENGINE_TCGEN05_PAIR)
+        ada.ada_set_row_compaction(ctx, min_rows)
+        check_cascade(ctx, Xs[1], cfg.tau, Rs)
+        rin = np.zeros((3, cfg.T), dtype=np.int32)
+        for b, r in enumerate(Rs):
+            rin[b, :len(r)] = r
+        o = ada.ada_cascade_step(ctx, to_device(Xs[1]), cfg.tau, torch.from_numpy(rin).cuda(),
+                                 torch.tensor([len(r) for r in Rs], dtype=torch.int32).cuda())
+        outs.append([o.rep_out.clone(), o.rep_out_cnt.clone(), o.add_cnt.clone(), o.rem_cnt.clone(),
+                     o.gamma_rep.clone(), o.gamma_cross.clone()])
+        assert ada.ada_device_status(ctx)[0] == 0
+        ada.ada_destroy(ctx)
+    for a, b in zip(*outs[:2]):
+        if a.dtype == torch.int32 and a.dim() == 2:      # list capacity beyond the counts is unspecified
+            for s in range(3):
+                n = int(outs[0][1][s])
+                assert torch.equal(a[s, :n], b[s, :n])
+        else:
+            assert torch.equal(a, b)
