@@ -37,8 +37,8 @@ UNIT = "tokens*layers/s"
 # same kernel on the same workload (one launch each), printed as `traffic_static` with their
 # origin beside them.  Keyed by (kernel, workload).
 NCU_TRAFFIC_BYTES = {
-    # fused cascade launch on configs[3]: mean of the captured layers 1 (76.9 MB) and 30 (108.4 MB)
-    ("gram_tc_cascade", 4): 92.65e6,
+    # cascade launch on configs[3]: mean of the captured layers 1 (77.2 MB) and 30 (104.3 MB)
+    ("gram_tc_cascade", 4): 90.75e6,
     # fused cascade launches of layers 1-2 on the smaller workloads
     ("gram_tc_cascade", 1): 9.53e6,
     ("gram_tc_cascade", 2): 28.9e6,

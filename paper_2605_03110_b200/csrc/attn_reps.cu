@@ -115,6 +115,11 @@ k_attn_reps(const __grid_constant__ AttnMaps maps, int T, int d_h, int h,
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int head = blockIdx.y, q0 = blockIdx.x * AQ;
 
+    // The grid is sized for T because r lives on the device: a CTA whose query rows lie past r
+    // leaves before it sets anything up (no barriers, no TMEM).
+    grid_dep_wait();
+    const int n = clamp_count(rep_cnt, T);
+    if (q0 >= n) return;
     if (threadIdx.x == 0) {
         mbar_init(&sh.q_full, 1);
         for (int i = 0; i < 2; ++i) {
@@ -132,13 +137,11 @@ k_attn_reps(const __grid_constant__ AttnMaps maps, int T, int d_h, int h,
                      ::"r"(smem_u32(&sh.tmem_base)), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    grid_dep_wait();
-    const int n = clamp_count(rep_cnt, T);
     tcgen05_fence_before();
     __syncthreads();
     tcgen05_fence_after();
     const unsigned tmem_base = sh.tmem_base;
-    const bool active = q0 < n;                        // uniform over the CTA
+    const bool active = true;
     int nkv = (n + AKV - 1) / AKV;
     if (causal) nkv = min(nkv, (int)blockIdx.x + 1);   // keys at or before the tile's last row
     const int nkb = (d_h + BK - 1) / BK;               // 64-element K blocks of the first contraction
