@@ -209,7 +209,8 @@ ada_status ada_create(ada_ctx** out, int device, int64_t maxB, int64_t maxT, int
     ctx->splitXB = split_bytes ? ctx->ws + o_sxb : nullptr;
     ctx->splitRA = split_bytes ? ctx->ws + o_sra : nullptr;
     ctx->splitRB = split_bytes ? ctx->ws + o_srb : nullptr;
-    if (cudaMemset(ctx->ws, 0, o_xrep) != cudaSuccess) {
+    if (cudaMemset(ctx->ws, 0, o_xrep) != cudaSuccess ||
+        (dt == ADA_BF16 && cudaMemset(ctx->ws + o_ntok, 0, n_tok * 4) != cudaSuccess)) {
         cudaFree(ctx->ws);
         delete ctx;
         return ADA_ERR_CUDA;

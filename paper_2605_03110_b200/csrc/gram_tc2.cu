@@ -513,9 +513,15 @@ k_gram_tc2(const __grid_constant__ GramMaps maps, const __grid_constant__ GramPr
             const int lrow = quad * 32 + lane;
             const int row_base = pc.row0 + (int)rank * arows;
             const int row = row_base + lrow;
-            const bool row_live = lrow < arows && row < pc.m;
+            bool row_live = lrow < arows && row < pc.m;
             // the token this row belongs to: the row index itself, except over the copied-out rows
-            const int tokrow = (compact && !p.tri && row_live) ? __ldcg(gather.non_tok + o + row) : row;
+            // (an entry the gather did not write -- possible only with a rejected list -- is
+            // never used as an index)
+            int tokrow = row;
+            if (compact && !p.tri && row_live) {
+                tokrow = __ldcg(gather.non_tok + o + row);
+                if ((unsigned)tokrow >= (unsigned)p.cap) { tokrow = row; row_live = false; }
+            }
             const bool defer = !p.tri && p.defer_row != 0;   // the row's own factor is applied later
             // inherited reps are not candidates (with a deferred factor the compaction ignores them)
             const bool skip = row_live && !p.tri && !defer && p.row_role[o + row] != 0;

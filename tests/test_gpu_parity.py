@@ -641,3 +641,26 @@ def test_row_compaction_batched_and_on_and_off_agree(ada):
                 assert torch.equal(a[s, :n], b[s, :n])
         else:
             assert torch.equal(a, b)
+
+
+def test_rejected_list_on_the_pair_kernel_with_row_compaction(ada):
+    """A list that is not ascending is reported and leaves everything in bounds, also where the
+    launch copies the rows outside the set (their positions then make no sense); the context
+    works afterwards."""
+    from parity import check_cascade
+    T, d = 192, 64
+    ctx = ada.ada_create(1, T, d, ada.ADA_BF16)
+    ada.ada_set_engine(ctx, ada.ADA_ENGINE_TCGEN05_PAIR)
+    ada.ada_set_row_compaction(ctx, 1)
+    X = clustered(T, d, 77, "bf16")
+    Xd = torch.from_numpy(X.view(np.int16)).view(torch.bfloat16).cuda()
+    bad = torch.zeros((1, T), dtype=torch.int32)
+    bad[0, :120] = torch.arange(150, 30, -1, dtype=torch.int32)      # descending
+    ada.ada_cascade_step(ctx, Xd, TAU, bad.cuda(), torch.tensor([120], dtype=torch.int32).cuda())
+    assert ada.ada_device_status(ctx)[0] == 5
+    bad[0, :120] = torch.arange(0, 120, dtype=torch.int32)
+    bad[0, 60] = 5000                                                 # out of range
+    ada.ada_cascade_step(ctx, Xd, TAU, bad.cuda(), torch.tensor([120], dtype=torch.int32).cuda())
+    assert ada.ada_device_status(ctx)[0] == 5
+    check_cascade(ctx, X, TAU, [list(range(0, T, 2))])
+    ada.ada_destroy(ctx)
