@@ -737,6 +737,12 @@ def main():
     if bound == "tensor" and cfg.dtype == "bf16":
         roofline["frac_sustained"] = achieved / peaks["bf16_sustained"]
         roofline["frac_burst"] = achieved / peaks["bf16_burst"]
+        # the whole timed step (every launch of the path, graph replay): all algorithmic flops of a
+        # step over ms_per_step -- free of the per-launch event brackets of the figure above
+        step_tf = sum(flops.values()) / (ms_step * 1e-3) / 1e12
+        roofline["whole_step"] = {"achieved": step_tf, "unit": "TFLOP/s",
+                                  "frac_burst": step_tf / peaks["bf16_burst"],
+                                  "frac_sustained": step_tf / peaks["bf16_sustained"]}
 
     # ---- sustained: the same graph replayed for at least a second (a 1 kW part settles to lower
     # clocks under load; the K-step figure above is the short-run one) ----
