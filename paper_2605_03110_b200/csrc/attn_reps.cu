@@ -8,11 +8,12 @@
 //   k_attn_reps     one CTA per (128 query rows, head).  Both contractions run on tcgen05:
 //                   S = Q K^T into TMEM (two 128 x 128 fp32 buffers), softmax by four warps
 //                   straight out of TMEM (one row per thread, so maxima and sums are
-//                   thread-local), P rounded to bf16 into shared memory in the 128-byte
-//                   swizzled K-major layout, O += P V^T into a third TMEM accumulator.  The
-//                   softmax is two-pass (first the row maxima and sums over all key tiles, then
-//                   the normalised probabilities), which costs a second Q K^T but needs no
-//                   rescaling of the accumulator; r is a few thousand at most.
+//                   thread-local), P rounded to bf16 into shared memory (two buffers) in the
+//                   128-byte swizzled K-major layout, O += P V^T into a third TMEM accumulator.
+//                   One pass over the key tiles: probabilities are taken against a per-row
+//                   reference maximum that is raised (and the accumulator rescaled, in TMEM) only
+//                   when the running maximum has moved by more than 8 powers of two, which after
+//                   the first tile is rare; the division by the row sum happens at the output.
 //   k_attn_expand   out[t] = out[nearest[t]] for the tokens outside R
 // Every wait is bounded (see gram_tc_dev.cuh).
 #include "gram_tc_dev.cuh"
@@ -21,21 +22,32 @@ namespace ada {
 
 using namespace tc;
 
+// Time stamps for in-kernel timelines (development builds only: -DADA_TRACE): the first 16 query
+// tiles of head 0.
+#ifdef ADA_TRACE
+__device__ unsigned long long g_atrace[16 * 32];
+#define ATRACE(slot) do { if (blockIdx.y == 0 && blockIdx.x < 16) g_atrace[blockIdx.x * 32 + (slot)] = tc::global_ns(); } while (0)
+#else
+#define ATRACE(slot) do { } while (0)
+#endif
+
 namespace {
 
 constexpr int AQ = 128;                 // query rows per CTA (TMEM lanes)
 constexpr int AKV = 128;                // keys per tile
 constexpr int KB_BYTES = 128 * BK * 2;  // one 64-element K block of a 128-row tile: 16 KiB
-constexpr int ATT_THREADS = 192;        // TMA producer, MMA issuer, four softmax warps
+constexpr int ATT_THREADS = 320;        // TMA producer, MMA issuer, eight softmax warps
 
 struct alignas(16) AttnShared {
     unsigned long long q_full, k_full[2], k_empty[2], v_full[2], v_empty[2];
-    unsigned long long s_full[2], s_empty[2], p_full, p_empty, o_full;
+    unsigned long long s_full[2], s_empty[2], p_full[2], p_empty[2], o_full;
+    unsigned long long x_put[4], x_got[4];   // per 32-row group: the two warps of a row exchange a value
     unsigned tmem_base;
     int abort_flag;
+    float xval[2][128];                      // [column half][row]
 };
-// Q (2 K blocks) | K ring 2 x 2 | V^T ring 2 x 2 | P (2 K blocks)
-constexpr int ATT_SMEM = (2 + 4 + 4 + 2) * KB_BYTES + (int)sizeof(AttnShared) + 1024;
+// Q (2 K blocks) | K ring 2 x 2 | V^T ring 2 x 2 | P 2 x 2
+constexpr int ATT_SMEM = (2 + 4 + 4 + 4) * KB_BYTES + (int)sizeof(AttnShared) + 1024;
 static_assert(ATT_SMEM <= 227 * 1024, "shared memory budget");
 
 struct AttnMaps {
@@ -99,6 +111,80 @@ k_attn_gather(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restri
 }
 
 // ---------------------------------------------------------------- attention
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ void tmem_st32(unsigned taddr, const float (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};\n\t"
+        "tcgen05.wait::st.sync.aligned;"
+        ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
+          "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])),
+          "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])),
+          "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+          "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])),
+          "r"(__float_as_uint(v[15])), "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])),
+          "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])), "r"(__float_as_uint(v[20])),
+          "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])),
+          "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])),
+          "r"(__float_as_uint(v[27])), "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])),
+          "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+        : "memory");
+}
+// The four softmax warps run one per scheduler with nothing to hide latency behind, so the
+// per-element code is kept to a max, an fma, an ex2, an add and half a convert, in
+// independent chains; the mask is applied only on tiles that need one.
+// 32 raw scores of one row: (mask,) maximum.  lim: how many of the 32 columns are admissible
+// (columns ascend, so both the end of the set and the causal bound cut a suffix)
+template <bool MASKED>
+__device__ __forceinline__ float tile_max32(unsigned (&r)[32], int lim, float cm) {
+    float m0 = cm, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+    for (int q = 0; q < 32; q += 4) {
+        if (MASKED) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (q + e >= lim) r[q + e] = 0xff800000u;   // -inf
+        }
+        m0 = fmaxf(m0, __uint_as_float(r[q]));
+        m1 = fmaxf(m1, __uint_as_float(r[q + 1]));
+        m2 = fmaxf(m2, __uint_as_float(r[q + 2]));
+        m3 = fmaxf(m3, __uint_as_float(r[q + 3]));
+    }
+    return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+}
+// p = 2^(s * sc - mref) for 32 raw scores, as bf16 into the row's 64 bytes of the swizzled P tile;
+// returns their sum
+__device__ __forceinline__ float exp_store(const unsigned (&r)[32], float sc, float mref, unsigned char* rowp,
+                                           int cc0, int row) {
+    unsigned w[16];
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+    for (int q = 0; q < 32; q += 4) {
+        const float p0 = ex2_approx(fmaf(__uint_as_float(r[q]), sc, -mref));
+        const float p1 = ex2_approx(fmaf(__uint_as_float(r[q + 1]), sc, -mref));
+        const float p2 = ex2_approx(fmaf(__uint_as_float(r[q + 2]), sc, -mref));
+        const float p3 = ex2_approx(fmaf(__uint_as_float(r[q + 3]), sc, -mref));
+        s0 += p0; s1 += p1; s2 += p2; s3 += p3;
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(p0, p1), hi = __floats2bfloat162_rn(p2, p3);
+        w[q >> 1] = *reinterpret_cast<const unsigned*>(&lo);
+        w[(q >> 1) + 1] = *reinterpret_cast<const unsigned*>(&hi);
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+        *reinterpret_cast<uint4*>(rowp + (((cc0 + q) ^ (row & 7)) << 4)) =
+            make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
+    return (s0 + s1) + (s2 + s3);
+}
+
+// How far a row's reference maximum may lag behind its true running maximum (in powers of two)
+// before the accumulator is rescaled: the probabilities of a tile are 2^(s - m_ref) <= 2^LAG.
+constexpr float ATT_LAG = 8.0f;
+
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 k_attn_reps(const __grid_constant__ AttnMaps maps, int T, int d_h, int h,
             const int32_t* __restrict__ rep_idx, const int32_t* __restrict__ rep_cnt,
@@ -109,8 +195,8 @@ k_attn_reps(const __grid_constant__ AttnMaps maps, int T, int d_h, int h,
     unsigned char* qs = smem;                          // Q tile: nkb K blocks
     unsigned char* ks = smem + 2 * KB_BYTES;           // K ring: 2 slots x 2 K blocks
     unsigned char* vs = smem + 6 * KB_BYTES;           // V^T ring: 2 slots x 2 K blocks of d_h rows
-    unsigned char* ps = smem + 10 * KB_BYTES;          // P: 2 K blocks
-    AttnShared& sh = *reinterpret_cast<AttnShared*>(smem + 12 * KB_BYTES);
+    unsigned char* ps = smem + 10 * KB_BYTES;          // P: 2 buffers x 2 K blocks
+    AttnShared& sh = *reinterpret_cast<AttnShared*>(smem + 14 * KB_BYTES);
     volatile int* abort_flag = &sh.abort_flag;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int head = blockIdx.y, q0 = blockIdx.x * AQ;
@@ -120,14 +206,17 @@ k_attn_reps(const __grid_constant__ AttnMaps maps, int T, int d_h, int h,
     grid_dep_wait();
     const int n = clamp_count(rep_cnt, T);
     if (q0 >= n) return;
+    if (threadIdx.x == 0) ATRACE(0);
     if (threadIdx.x == 0) {
         mbar_init(&sh.q_full, 1);
         for (int i = 0; i < 2; ++i) {
             mbar_init(&sh.k_full[i], 1); mbar_init(&sh.k_empty[i], 1);
             mbar_init(&sh.v_full[i], 1); mbar_init(&sh.v_empty[i], 1);
-            mbar_init(&sh.s_full[i], 1); mbar_init(&sh.s_empty[i], 4);
+            mbar_init(&sh.s_full[i], 1); mbar_init(&sh.s_empty[i], 8);
+            mbar_init(&sh.p_full[i], 8); mbar_init(&sh.p_empty[i], 1);
         }
-        mbar_init(&sh.p_full, 4); mbar_init(&sh.p_empty, 1); mbar_init(&sh.o_full, 1);
+        for (int i = 0; i < 4; ++i) { mbar_init(&sh.x_put[i], 2); mbar_init(&sh.x_got[i], 2); }
+        mbar_init(&sh.o_full, 1);
         sh.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -141,195 +230,213 @@ k_attn_reps(const __grid_constant__ AttnMaps maps, int T, int d_h, int h,
     __syncthreads();
     tcgen05_fence_after();
     const unsigned tmem_base = sh.tmem_base;
-    const bool active = true;
+    if (threadIdx.x == 0) ATRACE(1);
     int nkv = (n + AKV - 1) / AKV;
     if (causal) nkv = min(nkv, (int)blockIdx.x + 1);   // keys at or before the tile's last row
     const int nkb = (d_h + BK - 1) / BK;               // 64-element K blocks of the first contraction
     const int v_kb_bytes = d_h * BK * 2;               // one K block (64 keys) of the V^T tile
+    // Buffer b = j & 1 of every ring serves the key tiles j = b, b + 2, ...: tile j is its
+    // (j >> 1)-th use, which fixes the parity of every wait below.
 
-    if (active && warp == 0) {
+    if (warp == 0) {
         // ------------------------------------------------ TMA producer
         if (lane == 0) {
             bool ok = true;
             mbar_expect_tx(&sh.q_full, (unsigned)(nkb * KB_BYTES));
             for (int kb = 0; kb < nkb; ++kb) tma_load_3d(&maps.q, &sh.q_full, qs + kb * KB_BYTES, kb * BK, q0, head);
-            unsigned kfill = 0, vfill = 0;             // per slot: parity of the number of fills
-            int kit = 0;
-            for (int pass = 0; pass < 2 && ok; ++pass) {
-                for (int j = 0; j < nkv && ok; ++j, ++kit) {
-                    const int s = kit & 1;
-                    if (!mbar_wait(&sh.k_empty[s], ((kfill >> s) & 1u) ^ 1u, abort_flag, 31)) { ok = false; break; }
-                    mbar_expect_tx(&sh.k_full[s], (unsigned)(nkb * KB_BYTES));
-                    for (int kb = 0; kb < nkb; ++kb)
-                        tma_load_3d(&maps.k, &sh.k_full[s], ks + (s * 2 + kb) * KB_BYTES, kb * BK, j * AKV, head);
-                    kfill ^= 1u << s;
-                    if (pass == 1) {
-                        const int v = j & 1;
-                        if (!mbar_wait(&sh.v_empty[v], ((vfill >> v) & 1u) ^ 1u, abort_flag, 32)) { ok = false; break; }
-                        mbar_expect_tx(&sh.v_full[v], (unsigned)(2 * v_kb_bytes));
-                        for (int u = 0; u < 2; ++u)
-                            tma_load_3d(&maps.v, &sh.v_full[v], vs + v * 2 * KB_BYTES + u * v_kb_bytes,
-                                        j * AKV + u * BK, 0, head);
-                        vfill ^= 1u << v;
-                    }
-                }
+            for (int j = 0; j < nkv && ok; ++j) {
+                const int s = j & 1;
+                const unsigned prev = (((unsigned)j >> 1) & 1u) ^ 1u;
+                if (!mbar_wait(&sh.k_empty[s], prev, abort_flag, 31)) { ok = false; break; }
+                mbar_expect_tx(&sh.k_full[s], (unsigned)(nkb * KB_BYTES));
+                for (int kb = 0; kb < nkb; ++kb)
+                    tma_load_3d(&maps.k, &sh.k_full[s], ks + (s * 2 + kb) * KB_BYTES, kb * BK, j * AKV, head);
+                if (!mbar_wait(&sh.v_empty[s], prev, abort_flag, 32)) { ok = false; break; }
+                mbar_expect_tx(&sh.v_full[s], (unsigned)(2 * v_kb_bytes));
+                for (int u = 0; u < 2; ++u)
+                    tma_load_3d(&maps.v, &sh.v_full[s], vs + s * 2 * KB_BYTES + u * v_kb_bytes, j * AKV + u * BK, 0,
+                                head);
             }
-            // every copy has to land before the CTA may exit: a slot's release implies it
-            for (int s = 0; s < 2; ++s) {
-                if (kit > s) {
-                    const unsigned long long t0 = global_ns();
-                    while (!mbar_try(&sh.k_empty[s], ((kfill >> s) & 1u) ^ 1u))
-                        if (*abort_flag != 0 || global_ns() - t0 > WAIT_LIMIT_NS / 2) { *abort_flag = 33; break; }
-                }
-                if (nkv > s) {
-                    const unsigned long long t0 = global_ns();
-                    while (!mbar_try(&sh.v_empty[s], ((vfill >> s) & 1u) ^ 1u))
-                        if (*abort_flag != 0 || global_ns() - t0 > WAIT_LIMIT_NS / 2) { *abort_flag = 34; break; }
-                }
+            // every copy has to land before the CTA may exit: a slot's last release implies it
+            for (int s = 0; s < 2 && ok; ++s) {
+                if (nkv <= s) continue;
+                const int last = ((nkv - 1 - s) >> 1) * 2 + s;         // last tile that used slot s
+                const unsigned ph = ((unsigned)last >> 1) & 1u;
+                const unsigned long long t0 = global_ns();
+                while (!(mbar_try(&sh.k_empty[s], ph) && mbar_try(&sh.v_empty[s], ph)))
+                    if (*abort_flag != 0 || global_ns() - t0 > WAIT_LIMIT_NS / 2) { *abort_flag = 33; break; }
             }
         }
-    } else if (active && warp == 1) {
+    } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer
         if (lane == 0) {
             bool ok = mbar_wait(&sh.q_full, 0u, abort_flag, 35);
-            unsigned kuse = 0, suse = 0;               // parities per slot / buffer
-            int kit = 0, sit = 0;
             const unsigned idesc1 = instr_desc(AKV);
             const unsigned idesc2 = instr_desc(d_h);
-            // S[buf] = Q K_j^T
-            auto issue_s = [&]() {
-                const int s = kit & 1, b = sit & 1;
-                if (!mbar_wait(&sh.k_full[s], (kuse >> s) & 1u, abort_flag, 36)) { ok = false; return; }
-                if (!mbar_wait(&sh.s_empty[b], ((suse >> b) & 1u) ^ 1u, abort_flag, 37)) { ok = false; return; }
+            // S[j & 1] = Q K_j^T
+            auto issue_s = [&](int j) {
+                const int b = j & 1;
+                const unsigned ph = ((unsigned)j >> 1) & 1u;
+                if (!mbar_wait(&sh.k_full[b], ph, abort_flag, 36)) { ok = false; return; }
+                if (!mbar_wait(&sh.s_empty[b], ph ^ 1u, abort_flag, 37)) { ok = false; return; }
                 tcgen05_fence_after();
                 for (int kb = 0; kb < nkb; ++kb) {
                     const unsigned long long adesc = smem_desc_sw128(smem_u32(qs + kb * KB_BYTES));
-                    const unsigned long long bdesc = smem_desc_sw128(smem_u32(ks + (s * 2 + kb) * KB_BYTES));
+                    const unsigned long long bdesc = smem_desc_sw128(smem_u32(ks + (b * 2 + kb) * KB_BYTES));
                     const int steps = min(BK, d_h - kb * BK) / UMMA_K;
                     for (int k = 0; k < steps; ++k)
                         umma_bf16(tmem_base + b * AKV, adesc + 2 * k, bdesc + 2 * k, idesc1, (kb | k) != 0);
                 }
-                umma_commit(&sh.k_empty[s]);
+                umma_commit(&sh.k_empty[b]);
                 umma_commit(&sh.s_full[b]);
-                kuse ^= 1u << s; suse ^= 1u << b;
-                ++kit; ++sit;
             };
-            for (int j = 0; j < nkv && ok; ++j) issue_s();          // pass 1: statistics only
-            if (ok) issue_s();                                       // pass 2, tile 0
-            unsigned vuse = 0;
+            if (ok) issue_s(0);
             for (int j = 0; j < nkv && ok; ++j) {
-                if (j + 1 < nkv) issue_s();                          // keeps one S tile ahead of the softmax
+                if (j + 1 < nkv) issue_s(j + 1);                     // one score tile ahead of the softmax
                 if (!ok) break;
-                const int v = j & 1;
-                if (!mbar_wait(&sh.p_full, (unsigned)(j & 1), abort_flag, 38)) { ok = false; break; }
-                if (!mbar_wait(&sh.v_full[v], (vuse >> v) & 1u, abort_flag, 39)) { ok = false; break; }
+                const int b = j & 1;
+                const unsigned ph = ((unsigned)j >> 1) & 1u;
+                if (!mbar_wait(&sh.p_full[b], ph, abort_flag, 38)) { ok = false; break; }
+                if (!mbar_wait(&sh.v_full[b], ph, abort_flag, 39)) { ok = false; break; }
                 tcgen05_fence_after();
-                for (int u = 0; u < 2; ++u) {                        // O += P V_j
-                    const unsigned long long adesc = smem_desc_sw128(smem_u32(ps + u * KB_BYTES));
-                    const unsigned long long bdesc = smem_desc_sw128(smem_u32(vs + v * 2 * KB_BYTES + u * v_kb_bytes));
+                for (int u = 0; u < 2; ++u) {                        // O += P_j V_j
+                    const unsigned long long adesc = smem_desc_sw128(smem_u32(ps + (b * 2 + u) * KB_BYTES));
+                    const unsigned long long bdesc = smem_desc_sw128(smem_u32(vs + b * 2 * KB_BYTES + u * v_kb_bytes));
                     for (int k = 0; k < BK / UMMA_K; ++k)
                         umma_bf16(tmem_base + 2 * AKV, adesc + 2 * k, bdesc + 2 * k, idesc2, (j | u | k) != 0);
                 }
-                umma_commit(&sh.v_empty[v]);
-                umma_commit(&sh.p_empty);
-                vuse ^= 1u << v;
+                umma_commit(&sh.v_empty[b]);
+                umma_commit(&sh.p_empty[b]);
             }
             if (ok) umma_commit(&sh.o_full);
             else { /* the softmax warps time out on their own */ }
         }
-    } else if (active && warp >= 2) {
-        // ------------------------------------------------ softmax and output (warps 2..5)
+    } else {
+        // ------------------------------------------------ softmax and output (warps 2..9)
+        // One pass over the key tiles.  A row keeps a reference maximum m_ref that is raised only
+        // when the running maximum exceeds it by more than ATT_LAG; the tile's probabilities are
+        // 2^(s - m_ref) (at most 2^ATT_LAG, unnormalised), their sum goes into l, and O and l are
+        // rescaled by 2^(m_old - m_new) on the rare tile where m_ref moves -- after the MMAs
+        // that still add to O have retired.  The result O / l does not depend on m_ref.
+        // Two warps share a group of 32 rows (a warp reaches the TMEM lanes 32 (warp % 4) ..):
+        // warps 2..5 take the first 64 columns of every tile, warps 6..9 the other 64, and the
+        // two exchange their maxima (and at the end their sums) through shared memory.
         const int quad = warp & 3;
+        const int half = (warp - 2) >> 2;
         const int i = quad * 32 + lane;                // this thread's row of the tile
         const int qrow = q0 + i;                       // position in the representative list
         const unsigned tlane = tmem_base + ((unsigned)(quad * 32) << 16);
         const float sc = 1.4426950408889634f / sqrtf((float)d_h);   // log2(e) / sqrt(d_h)
-        float m = -INFINITY, l = 0.f;
-        unsigned suse = 0;
-        int sit = 0;
+        float m_ref = -INFINITY, l = 0.f;
         bool ok = true;
-        // pass 1: row maximum and sum of exponentials over all key tiles
-        for (int j = 0; j < nkv && ok; ++j, ++sit) {
-            const int b = sit & 1;
-            const bool got = mbar_wait(&sh.s_full[b], (suse >> b) & 1u, abort_flag, 40);
+        unsigned xn = 0;                               // exchanges so far
+        // both warps of a row give `mine`, each gets the other's
+        auto exchange = [&](float mine, float& other) -> bool {
+            bool g = xn == 0 || mbar_wait(&sh.x_got[quad], (xn - 1) & 1u, abort_flag, 45);   // my last value was read
+            if (!__all_sync(0xffffffffu, g)) return false;
+            sh.xval[half][i] = mine;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.x_put[quad]);
+            g = mbar_wait(&sh.x_put[quad], xn & 1u, abort_flag, 46);
+            if (!__all_sync(0xffffffffu, g)) return false;
+            other = sh.xval[half ^ 1][i];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.x_got[quad]);
+            ++xn;
+            return true;
+        };
+        for (int j = 0; j < nkv && ok; ++j) {
+            const int b = j & 1;
+            const unsigned ph = ((unsigned)j >> 1) & 1u;
+            bool got = mbar_wait(&sh.s_full[b], ph, abort_flag, 40);
             if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
+            if (j == 0 && threadIdx.x == 64) ATRACE(2);
+            if (j == 2 && threadIdx.x == 64) ATRACE(20);
             tcgen05_fence_after();
-            for (int c0 = 0; c0 < AKV; c0 += 32) {
-                float v[32];
-                tmem_ld32(tlane + b * AKV + c0, v);
-                float cm = -INFINITY;
-#pragma unroll
-                for (int q = 0; q < 32; ++q) {
-                    const int col = j * AKV + c0 + q;
-                    const bool valid = col < n && (!causal || col <= qrow);
-                    v[q] = valid ? v[q] * sc : -INFINITY;
-                    cm = fmaxf(cm, v[q]);
-                }
-                if (cm > -INFINITY) {
-                    const float mn = fmaxf(m, cm);
-                    float add = 0.f;
-#pragma unroll
-                    for (int q = 0; q < 32; ++q) add += exp2f(v[q] - mn);
-                    l = l * exp2f(m - mn) + add;
-                    m = mn;
-                }
-            }
+            unsigned r0[32], r1[32];                   // the row's 64 scores stay in registers
+            tmem_ld32_issue(tlane + b * AKV + half * 64, r0);
+            tmem_ld32_issue(tlane + b * AKV + half * 64 + 32, r1);
+            tmem_ld_wait(r0); tmem_ld_wait(r1);
+            if (j == 2 && threadIdx.x == 64) ATRACE(21);
             tcgen05_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sh.s_empty[b]);
-            suse ^= 1u << b;
-        }
-        // pass 2: P = exp2(S - m) / l as bf16 into shared memory, K-major with the 128-byte swizzle
-        const float inv_l = l > 0.f ? 1.0f / l : 0.f;
-        for (int j = 0; j < nkv && ok; ++j, ++sit) {
-            const int b = sit & 1;
-            bool got = mbar_wait(&sh.s_full[b], (suse >> b) & 1u, abort_flag, 41);
-            // the previous tile's P has been consumed by its MMAs
-            got = got && mbar_wait(&sh.p_empty, (unsigned)((j & 1) ^ 1), abort_flag, 42);
-            if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
-            tcgen05_fence_after();
-            for (int c0 = 0; c0 < AKV; c0 += 32) {
-                float v[32];
-                tmem_ld32(tlane + b * AKV + c0, v);
-                unsigned w[16];
-#pragma unroll
-                for (int q = 0; q < 32; q += 2) {
-                    const int col = j * AKV + c0 + q;
-                    const bool v0 = col < n && (!causal || col <= qrow);
-                    const bool v1 = col + 1 < n && (!causal || col + 1 <= qrow);
-                    const float p0 = v0 ? exp2f(v[q] * sc - m) * inv_l : 0.f;
-                    const float p1 = v1 ? exp2f(v[q + 1] * sc - m) * inv_l : 0.f;
-                    const __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-                    w[q >> 1] = *reinterpret_cast<const unsigned*>(&pk);
-                }
-                unsigned char* rowp = ps + (c0 >> 6) * KB_BYTES + i * 128;
-                const int cc0 = (c0 & 63) >> 3;        // first 16-byte chunk of these 32 columns
-#pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    *reinterpret_cast<uint4*>(rowp + (((cc0 + q) ^ (i & 7)) << 4)) =
-                        make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
+            if (lane == 0) mbar_arrive(&sh.s_empty[b]);        // the score buffer is free for tile j + 2
+            // columns past r, and under the causal mask the keys after the query, count as -inf
+            const int c0 = j * AKV + half * 64;
+            const bool masked = (j * AKV + AKV > n) || (causal && j * AKV + AKV - 1 > q0);
+            float cm = -INFINITY;                              // of the raw scores
+            if (masked) {
+                const int lim = min(n, causal ? qrow + 1 : n) - c0;
+                cm = tile_max32<true>(r0, lim, cm);
+                cm = tile_max32<true>(r1, lim - 32, cm);
+            } else {
+                cm = tile_max32<false>(r0, 32, cm);
+                cm = tile_max32<false>(r1, 32, cm);
             }
+            float cm_other;
+            if (!exchange(cm, cm_other)) { ok = false; break; }
+            cm = fmaxf(cm, cm_other) * sc;                     // sc > 0: the maximum of the scaled scores
+            if (j == 2 && threadIdx.x == 64) ATRACE(22);
+            const float m_new = fmaxf(m_ref, cm);
+            const bool raise = m_new > m_ref + ATT_LAG;        // also true for the first finite maximum
+            if (j == 0) {
+                m_ref = m_new;                                 // nothing accumulated yet
+            } else if (__any_sync(0xffffffffu, raise)) {
+                // O is about to change under the accumulating MMAs: wait until tile j-1's have retired.
+                // (Both warps of a row see the same maxima and take the same decision; each
+                // rescales every other 32-column chunk of O.)
+                got = mbar_wait(&sh.p_empty[(j - 1) & 1], ((unsigned)(j - 1) >> 1) & 1u, abort_flag, 44);
+                if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
+                tcgen05_fence_after();
+                const float f = raise ? ex2_approx(m_ref - m_new) : 1.0f;   // 0 for a row without a finite score so far
+                for (int o0 = half * 32; o0 < d_h; o0 += 64) {
+                    float v[32];
+                    tmem_ld32(tlane + 2 * AKV + o0, v);
+#pragma unroll
+                    for (int q = 0; q < 32; ++q) v[q] *= f;
+                    tmem_st32(tlane + 2 * AKV + o0, v);
+                }
+                tcgen05_fence_before();
+                l *= f;
+                if (raise) m_ref = m_new;
+            }
+            // the MMAs of tile j-2 have consumed this P buffer
+            got = mbar_wait(&sh.p_empty[b], ph ^ 1u, abort_flag, 42);
+            if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
+            if (j == 2 && threadIdx.x == 64) ATRACE(23);
+            const float mref = m_ref > -INFINITY ? m_ref : 0.f;   // all scores -inf so far: every p is 0
+            unsigned char* prow = ps + (b * 2 + half) * KB_BYTES + i * 128;
+            float sum = exp_store(r0, sc, mref, prow, 0, i);
+            sum += exp_store(r1, sc, mref, prow, 4, i);
+            l += sum;
+            if (j == 2 && threadIdx.x == 64) ATRACE(24);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the MMA reads P through the async proxy
             tcgen05_fence_before();
             __syncwarp();
-            if (lane == 0) { mbar_arrive(&sh.p_full); mbar_arrive(&sh.s_empty[b]); }
-            suse ^= 1u << b;
+            if (lane == 0) mbar_arrive(&sh.p_full[b]);
+            if (threadIdx.x == 64) ATRACE(3 + min(j, 12));
         }
         // output rows of this tile's representatives, at their token positions
+        float l_other = 0.f;
+        if (ok && !exchange(l, l_other)) ok = false;
         if (ok) {
             const bool got = mbar_wait(&sh.o_full, 0u, abort_flag, 43);
             if (__all_sync(0xffffffffu, got)) {
+                if (threadIdx.x == 64) ATRACE(16);
                 tcgen05_fence_after();
+                const float lt = l + l_other;
+                const float inv_l = lt > 0.f ? 1.0f / lt : 0.f;
                 const int tok = qrow < n ? rep_idx[qrow] : -1;
                 float* dst = (tok >= 0 && tok < T) ? out + (int64_t)tok * ldo + (int64_t)head * d_h : nullptr;
-                for (int c0 = 0; c0 < d_h; c0 += 32) {
+                for (int o0 = half * 32; o0 < d_h; o0 += 64) {
                     float v[32];
-                    tmem_ld32(tlane + 2 * AKV + c0, v);
+                    tmem_ld32(tlane + 2 * AKV + o0, v);
                     if (dst != nullptr) {
 #pragma unroll
                         for (int q = 0; q < 32; q += 4)
-                            if (c0 + q < d_h)
-                                *reinterpret_cast<float4*>(dst + c0 + q) = make_float4(v[q], v[q + 1], v[q + 2], v[q + 3]);
+                            if (o0 + q < d_h)
+                                *reinterpret_cast<float4*>(dst + o0 + q) =
+                                    make_float4(v[q] * inv_l, v[q + 1] * inv_l, v[q + 2] * inv_l, v[q + 3] * inv_l);
                     }
                 }
             }
@@ -345,6 +452,7 @@ k_attn_reps(const __grid_constant__ AttnMaps maps, int T, int d_h, int h,
         atomicOr(status, ST_TIMEOUT);
         status[2] = 200u + (unsigned)sh.abort_flag;
     }
+    if (threadIdx.x == 0) ATRACE(17);
 }
 
 // ---------------------------------------------------------------- expansion (Section 2.3)
@@ -404,3 +512,14 @@ cudaError_t launch_attention_reps(ada_ctx* ctx, const void* Q, const void* K, co
 }
 
 }  // namespace ada
+
+#ifdef ADA_TRACE
+extern "C" int ada_trace_read_attn(unsigned long long* host, int clear) {
+    if (cudaMemcpyFromSymbol(host, ada::g_atrace, sizeof(ada::g_atrace)) != cudaSuccess) return 1;
+    if (clear) {
+        static unsigned long long zeros[16 * 32];
+        if (cudaMemcpyToSymbol(ada::g_atrace, zeros, sizeof(zeros)) != cudaSuccess) return 2;
+    }
+    return 0;
+}
+#endif
