@@ -41,10 +41,9 @@ constexpr int ATT_THREADS = 320;        // TMA producer, MMA issuer, eight softm
 struct alignas(16) AttnShared {
     unsigned long long q_full, k_full[2], k_empty[2], v_full[2], v_empty[2];
     unsigned long long s_full[2], s_empty[2], p_full[2], p_empty[2], o_full;
-    unsigned long long x_put[4], x_got[4];   // per 32-row group: the two warps of a row exchange a value
+    unsigned long long x_put[4];             // per 32-row group: the two warps of a row exchange their statistics
     unsigned tmem_base;
     int abort_flag;
-    float xval[2][128];                      // [column half][row]
 };
 // Q (2 K blocks) | K ring 2 x 2 | V^T ring 2 x 2 | P 2 x 2
 constexpr int ATT_SMEM = (2 + 4 + 4 + 4) * KB_BYTES + (int)sizeof(AttnShared) + 1024;
@@ -135,7 +134,7 @@ __device__ __forceinline__ void tmem_st32(unsigned taddr, const float (&v)[32]) 
           "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
         : "memory");
 }
-// The four softmax warps run one per scheduler with nothing to hide latency behind, so the
+// The softmax warps run one or two per scheduler with little to hide latency behind, so the
 // per-element code is kept to a max, an fma, an ex2, an add and half a convert, in
 // independent chains; the mask is applied only on tiles that need one.
 // 32 raw scores of one row: (mask,) maximum.  lim: how many of the 32 columns are admissible
@@ -212,10 +211,10 @@ k_attn_reps(const __grid_constant__ AttnMaps maps, int T, int d_h, int h,
         for (int i = 0; i < 2; ++i) {
             mbar_init(&sh.k_full[i], 1); mbar_init(&sh.k_empty[i], 1);
             mbar_init(&sh.v_full[i], 1); mbar_init(&sh.v_empty[i], 1);
-            mbar_init(&sh.s_full[i], 1); mbar_init(&sh.s_empty[i], 8);
-            mbar_init(&sh.p_full[i], 8); mbar_init(&sh.p_empty[i], 1);
+            mbar_init(&sh.s_full[i], 1); mbar_init(&sh.s_empty[i], 4);
+            mbar_init(&sh.p_full[i], 4); mbar_init(&sh.p_empty[i], 1);
         }
-        for (int i = 0; i < 4; ++i) { mbar_init(&sh.x_put[i], 2); mbar_init(&sh.x_got[i], 2); }
+        for (int i = 0; i < 4; ++i) mbar_init(&sh.x_put[i], 2);
         mbar_init(&sh.o_full, 1);
         sh.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -299,11 +298,12 @@ k_attn_reps(const __grid_constant__ AttnMaps maps, int T, int d_h, int h,
                 if (!mbar_wait(&sh.p_full[b], ph, abort_flag, 38)) { ok = false; break; }
                 if (!mbar_wait(&sh.v_full[b], ph, abort_flag, 39)) { ok = false; break; }
                 tcgen05_fence_after();
-                for (int u = 0; u < 2; ++u) {                        // O += P_j V_j
+                for (int u = 0; u < 2; ++u) {                        // O[j & 1] += P_j V_j
                     const unsigned long long adesc = smem_desc_sw128(smem_u32(ps + (b * 2 + u) * KB_BYTES));
                     const unsigned long long bdesc = smem_desc_sw128(smem_u32(vs + b * 2 * KB_BYTES + u * v_kb_bytes));
                     for (int k = 0; k < BK / UMMA_K; ++k)
-                        umma_bf16(tmem_base + 2 * AKV, adesc + 2 * k, bdesc + 2 * k, idesc2, (j | u | k) != 0);
+                        umma_bf16(tmem_base + (2 + b) * AKV, adesc + 2 * k, bdesc + 2 * k, idesc2,
+                                  ((j >> 1) | u | k) != 0);
                 }
                 umma_commit(&sh.v_empty[b]);
                 umma_commit(&sh.p_empty[b]);
@@ -316,127 +316,139 @@ k_attn_reps(const __grid_constant__ AttnMaps maps, int T, int d_h, int h,
         // One pass over the key tiles.  A row keeps a reference maximum m_ref that is raised only
         // when the running maximum exceeds it by more than ATT_LAG; the tile's probabilities are
         // 2^(s - m_ref) (at most 2^ATT_LAG, unnormalised), their sum goes into l, and O and l are
-        // rescaled by 2^(m_old - m_new) on the rare tile where m_ref moves -- after the MMAs
-        // that still add to O have retired.  The result O / l does not depend on m_ref.
-        // Two warps share a group of 32 rows (a warp reaches the TMEM lanes 32 (warp % 4) ..):
-        // warps 2..5 take the first 64 columns of every tile, warps 6..9 the other 64, and the
-        // two exchange their maxima (and at the end their sums) through shared memory.
+        // rescaled by 2^(m_old - m_new) on the rare tile where m_ref moves.  O / l does not
+        // depend on m_ref.
+        // Two sets of four warps (a warp reaches the TMEM lanes 32 (warp % 4) ..) take ALTERNATE
+        // key tiles: warps 2..5 the even ones, warps 6..9 the odd ones, each set with its own score
+        // buffer, P buffer, accumulator and (m_ref, l), so that one set's exponentials overlap the
+        // other's loads and maxima with nothing exchanged per tile.  The two partial results are
+        // merged at the output like two halves of any split softmax.
         const int quad = warp & 3;
-        const int half = (warp - 2) >> 2;
+        const int half = (warp - 2) >> 2;              // = parity of this set's key tiles = its buffers
         const int i = quad * 32 + lane;                // this thread's row of the tile
         const int qrow = q0 + i;                       // position in the representative list
         const unsigned tlane = tmem_base + ((unsigned)(quad * 32) << 16);
+        const unsigned t_s = tlane + half * AKV, t_o = tlane + (2 + half) * AKV;
         const float sc = 1.4426950408889634f / sqrtf((float)d_h);   // log2(e) / sqrt(d_h)
+        const int lim_abs = min(n, causal ? qrow + 1 : n);          // admissible keys of this row: [0, lim_abs)
         float m_ref = -INFINITY, l = 0.f;
         bool ok = true;
-        unsigned xn = 0;                               // exchanges so far
-        // both warps of a row give `mine`, each gets the other's
-        auto exchange = [&](float mine, float& other) -> bool {
-            bool g = xn == 0 || mbar_wait(&sh.x_got[quad], (xn - 1) & 1u, abort_flag, 45);   // my last value was read
-            if (!__all_sync(0xffffffffu, g)) return false;
-            sh.xval[half][i] = mine;
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sh.x_put[quad]);
-            g = mbar_wait(&sh.x_put[quad], xn & 1u, abort_flag, 46);
-            if (!__all_sync(0xffffffffu, g)) return false;
-            other = sh.xval[half ^ 1][i];
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sh.x_got[quad]);
-            ++xn;
-            return true;
-        };
-        for (int j = 0; j < nkv && ok; ++j) {
-            const int b = j & 1;
+        for (int j = half; j < nkv && ok; j += 2) {
             const unsigned ph = ((unsigned)j >> 1) & 1u;
-            bool got = mbar_wait(&sh.s_full[b], ph, abort_flag, 40);
+            bool got = mbar_wait(&sh.s_full[half], ph, abort_flag, 40);
             if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
             if (j == 0 && threadIdx.x == 64) ATRACE(2);
             if (j == 2 && threadIdx.x == 64) ATRACE(20);
             tcgen05_fence_after();
-            unsigned r0[32], r1[32];                   // the row's 64 scores stay in registers
-            tmem_ld32_issue(tlane + b * AKV + half * 64, r0);
-            tmem_ld32_issue(tlane + b * AKV + half * 64 + 32, r1);
-            tmem_ld_wait(r0); tmem_ld_wait(r1);
-            if (j == 2 && threadIdx.x == 64) ATRACE(21);
-            tcgen05_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sh.s_empty[b]);        // the score buffer is free for tile j + 2
             // columns past r, and under the causal mask the keys after the query, count as -inf
-            const int c0 = j * AKV + half * 64;
-            const bool masked = (j * AKV + AKV > n) || (causal && j * AKV + AKV - 1 > q0);
-            float cm = -INFINITY;                              // of the raw scores
-            if (masked) {
-                const int lim = min(n, causal ? qrow + 1 : n) - c0;
-                cm = tile_max32<true>(r0, lim, cm);
-                cm = tile_max32<true>(r1, lim - 32, cm);
-            } else {
-                cm = tile_max32<false>(r0, 32, cm);
-                cm = tile_max32<false>(r1, 32, cm);
+            const int c0 = j * AKV;
+            const bool masked = (c0 + AKV > n) || (causal && c0 + AKV - 1 > q0);
+            // sweep 1: the row maximum of the raw scores
+            float cm = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < AKV; c += 64) {
+                unsigned r0[32], r1[32];
+                tmem_ld32_issue(t_s + c, r0);
+                tmem_ld32_issue(t_s + c + 32, r1);
+                tmem_ld_wait(r0); tmem_ld_wait(r1);
+                if (masked) {
+                    cm = tile_max32<true>(r0, lim_abs - (c0 + c), cm);
+                    cm = tile_max32<true>(r1, lim_abs - (c0 + c + 32), cm);
+                } else {
+                    cm = tile_max32<false>(r0, 32, cm);
+                    cm = tile_max32<false>(r1, 32, cm);
+                }
             }
-            float cm_other;
-            if (!exchange(cm, cm_other)) { ok = false; break; }
-            cm = fmaxf(cm, cm_other) * sc;                     // sc > 0: the maximum of the scaled scores
-            if (j == 2 && threadIdx.x == 64) ATRACE(22);
+            cm *= sc;                                          // sc > 0: the maximum of the scaled scores
+            if (j == 2 && threadIdx.x == 64) ATRACE(21);
             const float m_new = fmaxf(m_ref, cm);
             const bool raise = m_new > m_ref + ATT_LAG;        // also true for the first finite maximum
-            if (j == 0) {
+            // the MMAs of this set's previous tile have retired: its P buffer is free and nothing
+            // is adding to its accumulator
+            got = mbar_wait(&sh.p_empty[half], ph ^ 1u, abort_flag, 42);
+            if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
+            if (j < 2) {
                 m_ref = m_new;                                 // nothing accumulated yet
             } else if (__any_sync(0xffffffffu, raise)) {
-                // O is about to change under the accumulating MMAs: wait until tile j-1's have retired.
-                // (Both warps of a row see the same maxima and take the same decision; each
-                // rescales every other 32-column chunk of O.)
-                got = mbar_wait(&sh.p_empty[(j - 1) & 1], ((unsigned)(j - 1) >> 1) & 1u, abort_flag, 44);
-                if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
                 tcgen05_fence_after();
                 const float f = raise ? ex2_approx(m_ref - m_new) : 1.0f;   // 0 for a row without a finite score so far
-                for (int o0 = half * 32; o0 < d_h; o0 += 64) {
+                for (int o0 = 0; o0 < d_h; o0 += 32) {
                     float v[32];
-                    tmem_ld32(tlane + 2 * AKV + o0, v);
+                    tmem_ld32(t_o + o0, v);
 #pragma unroll
                     for (int q = 0; q < 32; ++q) v[q] *= f;
-                    tmem_st32(tlane + 2 * AKV + o0, v);
+                    tmem_st32(t_o + o0, v);
                 }
-                tcgen05_fence_before();
                 l *= f;
                 if (raise) m_ref = m_new;
             }
-            // the MMAs of tile j-2 have consumed this P buffer
-            got = mbar_wait(&sh.p_empty[b], ph ^ 1u, abort_flag, 42);
-            if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
-            if (j == 2 && threadIdx.x == 64) ATRACE(23);
+            if (j == 2 && threadIdx.x == 64) ATRACE(22);
+            // sweep 2: the probabilities
             const float mref = m_ref > -INFINITY ? m_ref : 0.f;   // all scores -inf so far: every p is 0
-            unsigned char* prow = ps + (b * 2 + half) * KB_BYTES + i * 128;
-            float sum = exp_store(r0, sc, mref, prow, 0, i);
-            sum += exp_store(r1, sc, mref, prow, 4, i);
+            unsigned char* prow = ps + half * 2 * KB_BYTES + i * 128;
+            float sum = 0.f;
+#pragma unroll
+            for (int c = 0; c < AKV; c += 64) {
+                unsigned r0[32], r1[32];
+                tmem_ld32_issue(t_s + c, r0);
+                tmem_ld32_issue(t_s + c + 32, r1);
+                tmem_ld_wait(r0); tmem_ld_wait(r1);
+                if (masked) {
+                    tile_max32<true>(r0, lim_abs - (c0 + c), 0.f);
+                    tile_max32<true>(r1, lim_abs - (c0 + c + 32), 0.f);
+                }
+                sum += exp_store(r0, sc, mref, prow + (c >> 6) * KB_BYTES, 0, i);
+                sum += exp_store(r1, sc, mref, prow + (c >> 6) * KB_BYTES, 4, i);
+            }
             l += sum;
-            if (j == 2 && threadIdx.x == 64) ATRACE(24);
+            if (j == 2 && threadIdx.x == 64) ATRACE(23);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the MMA reads P through the async proxy
             tcgen05_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sh.p_full[b]);
+            if (lane == 0) { mbar_arrive(&sh.s_empty[half]); mbar_arrive(&sh.p_full[half]); }
             if (threadIdx.x == 64) ATRACE(3 + min(j, 12));
         }
         // output rows of this tile's representatives, at their token positions
-        float l_other = 0.f;
-        if (ok && !exchange(l, l_other)) ok = false;
         if (ok) {
-            const bool got = mbar_wait(&sh.o_full, 0u, abort_flag, 43);
+            bool got = mbar_wait(&sh.o_full, 0u, abort_flag, 43);
             if (__all_sync(0xffffffffu, got)) {
                 if (threadIdx.x == 64) ATRACE(16);
                 tcgen05_fence_after();
-                const float lt = l + l_other;
-                const float inv_l = lt > 0.f ? 1.0f / lt : 0.f;
-                const int tok = qrow < n ? rep_idx[qrow] : -1;
-                float* dst = (tok >= 0 && tok < T) ? out + (int64_t)tok * ldo + (int64_t)head * d_h : nullptr;
-                for (int o0 = half * 32; o0 < d_h; o0 += 64) {
-                    float v[32];
-                    tmem_ld32(tlane + 2 * AKV + o0, v);
-                    if (dst != nullptr) {
+                // the two sets' statistics meet in the (now idle) P region
+                float2* xs = reinterpret_cast<float2*>(ps);
+                xs[half * AQ + i] = make_float2(m_ref, l);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.x_put[quad]);
+                got = mbar_wait(&sh.x_put[quad], 0u, abort_flag, 45);
+                if (__all_sync(0xffffffffu, got)) {
+                    const float2 other = xs[(half ^ 1) * AQ + i];
+                    const float m = fmaxf(m_ref, other.x);
+                    const float f_own = m_ref > -INFINITY ? ex2_approx(m_ref - m) : 0.f;
+                    const float f_oth = other.x > -INFINITY ? ex2_approx(other.x - m) : 0.f;
+                    const float lt = l * f_own + other.y * f_oth;
+                    const float inv_l = lt > 0.f ? 1.0f / lt : 0.f;
+                    const float fa = (half == 0 ? f_own : f_oth) * inv_l;      // factor of the even tiles' accumulator
+                    const float fb = (half == 0 ? f_oth : f_own) * inv_l;
+                    const bool use_b = nkv > 1;                                  // was the odd accumulator ever written
+                    const int tok = qrow < n ? rep_idx[qrow] : -1;
+                    float* dst = (tok >= 0 && tok < T) ? out + (int64_t)tok * ldo + (int64_t)head * d_h : nullptr;
+                    for (int o0 = half * 32; o0 < d_h; o0 += 64) {
+                        float va[32], vb[32];
+                        tmem_ld32(tlane + 2 * AKV + o0, va);
+                        if (use_b) tmem_ld32(tlane + 3 * AKV + o0, vb);
+                        if (dst != nullptr) {
 #pragma unroll
-                        for (int q = 0; q < 32; q += 4)
-                            if (o0 + q < d_h)
-                                *reinterpret_cast<float4*>(dst + o0 + q) =
-                                    make_float4(v[q] * inv_l, v[q + 1] * inv_l, v[q + 2] * inv_l, v[q + 3] * inv_l);
+                            for (int q = 0; q < 32; q += 4) {
+                                if (o0 + q < d_h) {
+                                    float4 w = make_float4(va[q] * fa, va[q + 1] * fa, va[q + 2] * fa, va[q + 3] * fa);
+                                    if (use_b) {
+                                        w.x = fmaf(vb[q], fb, w.x); w.y = fmaf(vb[q + 1], fb, w.y);
+                                        w.z = fmaf(vb[q + 2], fb, w.z); w.w = fmaf(vb[q + 3], fb, w.w);
+                                    }
+                                    *reinterpret_cast<float4*>(dst + o0 + q) = w;
+                                }
+                            }
+                        }
                     }
                 }
             }
