@@ -39,14 +39,16 @@ constexpr int KB_BYTES = 128 * BK * 2;  // one 64-element K block of a 128-row t
 constexpr int ATT_THREADS = 320;        // TMA producer, MMA issuer, eight softmax warps
 
 struct alignas(16) AttnShared {
-    unsigned long long q_full, k_full[2], k_empty[2], v_full[2], v_empty[2];
-    unsigned long long s_full[2], s_empty[2], p_full[2], p_empty[2], o_full;
+    unsigned long long q_full, q_empty, k_full[2], k_empty[2], v_full[2], v_empty[2];
+    unsigned long long s_full[2], s_empty[2], p_full[2], p_empty[2], o_full, o_empty;
     unsigned long long x_put[4];             // per 32-row group: the two warps of a row exchange their statistics
     unsigned tmem_base;
     int abort_flag;
+    float2 xstat[2][AQ];                     // (m_ref, l) of each warp set, by row
 };
-// Q (2 K blocks) | K ring 2 x 2 | V^T ring 2 x 2 | P 2 x 2
-constexpr int ATT_SMEM = (2 + 4 + 4 + 4) * KB_BYTES + (int)sizeof(AttnShared) + 1024;
+// Q (2 K blocks) | K ring 2 x 2 | V^T ring 2 x 2 | P 2 x 2.  The dynamic shared memory is declared
+// 1024-byte aligned (the swizzled tiles need it); the kernel checks the address it gets.
+constexpr int ATT_SMEM = (2 + 4 + 4 + 4) * KB_BYTES + (int)sizeof(AttnShared);
 static_assert(ATT_SMEM <= 227 * 1024, "shared memory budget");
 
 struct AttnMaps {
@@ -188,9 +190,7 @@ __global__ void __launch_bounds__(ATT_THREADS, 1)
 k_attn_reps(const __grid_constant__ AttnMaps maps, int T, int d_h, int h,
             const int32_t* __restrict__ rep_idx, const int32_t* __restrict__ rep_cnt,
             float* __restrict__ out, int64_t ldo, int causal, unsigned* __restrict__ status) {
-    extern __shared__ unsigned char smem_raw[];
-    unsigned char* smem = reinterpret_cast<unsigned char*>(
-        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    extern __shared__ __align__(1024) unsigned char smem[];
     unsigned char* qs = smem;                          // Q tile: nkb K blocks
     unsigned char* ks = smem + 2 * KB_BYTES;           // K ring: 2 slots x 2 K blocks
     unsigned char* vs = smem + 6 * KB_BYTES;           // V^T ring: 2 slots x 2 K blocks of d_h rows
@@ -198,16 +198,24 @@ k_attn_reps(const __grid_constant__ AttnMaps maps, int T, int d_h, int h,
     AttnShared& sh = *reinterpret_cast<AttnShared*>(smem + 14 * KB_BYTES);
     volatile int* abort_flag = &sh.abort_flag;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int head = blockIdx.y, q0 = blockIdx.x * AQ;
 
-    // The grid is sized for T because r lives on the device: a CTA whose query rows lie past r
-    // leaves before it sets anything up (no barriers, no TMEM).
+    // Persistent CTAs: the work items are (128 query rows, head) pairs, nq * h of them with
+    // nq = ceil(r / 128) known only on the device; CTA c takes items c, c + gridDim.x, ...
+    // Barriers, TMEM and the rings live across items (a buffer's uses are counted on, so every
+    // wait's parity follows from a running count), and the next item's Q, first keys and first
+    // score tiles are under way while the softmax warps still write the previous item's rows.
     grid_dep_wait();
     const int n = clamp_count(rep_cnt, T);
-    if (q0 >= n) return;
+    const int nq = (n + AQ - 1) / AQ;
+    const int total = nq * h;
+    if ((int)blockIdx.x >= total) return;              // before anything is set up
+    if ((smem_u32(smem) & 1023u) != 0u) {              // the tiles would not be where the swizzle assumes
+        if (threadIdx.x == 0) { atomicOr(status, ST_TIMEOUT); status[2] = 299u; }
+        return;
+    }
     if (threadIdx.x == 0) ATRACE(0);
     if (threadIdx.x == 0) {
-        mbar_init(&sh.q_full, 1);
+        mbar_init(&sh.q_full, 1); mbar_init(&sh.q_empty, 1);
         for (int i = 0; i < 2; ++i) {
             mbar_init(&sh.k_full[i], 1); mbar_init(&sh.k_empty[i], 1);
             mbar_init(&sh.v_full[i], 1); mbar_init(&sh.v_empty[i], 1);
@@ -215,7 +223,7 @@ k_attn_reps(const __grid_constant__ AttnMaps maps, int T, int d_h, int h,
             mbar_init(&sh.p_full[i], 4); mbar_init(&sh.p_empty[i], 1);
         }
         for (int i = 0; i < 4; ++i) mbar_init(&sh.x_put[i], 2);
-        mbar_init(&sh.o_full, 1);
+        mbar_init(&sh.o_full, 1); mbar_init(&sh.o_empty, 8);
         sh.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -230,37 +238,46 @@ k_attn_reps(const __grid_constant__ AttnMaps maps, int T, int d_h, int h,
     tcgen05_fence_after();
     const unsigned tmem_base = sh.tmem_base;
     if (threadIdx.x == 0) ATRACE(1);
-    int nkv = (n + AKV - 1) / AKV;
-    if (causal) nkv = min(nkv, (int)blockIdx.x + 1);   // keys at or before the tile's last row
+    const int nkv_all = (n + AKV - 1) / AKV;
     const int nkb = (d_h + BK - 1) / BK;               // 64-element K blocks of the first contraction
     const int v_kb_bytes = d_h * BK * 2;               // one K block (64 keys) of the V^T tile
-    // Buffer b = j & 1 of every ring serves the key tiles j = b, b + 2, ...: tile j is its
-    // (j >> 1)-th use, which fixes the parity of every wait below.
+    // Buffer b = j & 1 of every ring serves the key tiles j = b, b + 2, ... of an item; with
+    // base[b] uses in the CTA's earlier items, tile j is use number base[b] + (j >> 1).
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
         if (lane == 0) {
             bool ok = true;
-            mbar_expect_tx(&sh.q_full, (unsigned)(nkb * KB_BYTES));
-            for (int kb = 0; kb < nkb; ++kb) tma_load_3d(&maps.q, &sh.q_full, qs + kb * KB_BYTES, kb * BK, q0, head);
-            for (int j = 0; j < nkv && ok; ++j) {
-                const int s = j & 1;
-                const unsigned prev = (((unsigned)j >> 1) & 1u) ^ 1u;
-                if (!mbar_wait(&sh.k_empty[s], prev, abort_flag, 31)) { ok = false; break; }
-                mbar_expect_tx(&sh.k_full[s], (unsigned)(nkb * KB_BYTES));
+            unsigned base[2] = {0u, 0u};
+            int k = 0;
+            for (int item = blockIdx.x; item < total && ok; item += gridDim.x, ++k) {
+                const int qt = item % nq, head = item / nq, q0 = qt * AQ;
+                const int nkv = causal ? min(nkv_all, qt + 1) : nkv_all;   // keys at or before the tile's last row
+                // the previous item's Q K^T MMAs have read Q
+                if (k > 0 && !mbar_wait(&sh.q_empty, (unsigned)(k - 1) & 1u, abort_flag, 30)) { ok = false; break; }
+                mbar_expect_tx(&sh.q_full, (unsigned)(nkb * KB_BYTES));
                 for (int kb = 0; kb < nkb; ++kb)
-                    tma_load_3d(&maps.k, &sh.k_full[s], ks + (s * 2 + kb) * KB_BYTES, kb * BK, j * AKV, head);
-                if (!mbar_wait(&sh.v_empty[s], prev, abort_flag, 32)) { ok = false; break; }
-                mbar_expect_tx(&sh.v_full[s], (unsigned)(2 * v_kb_bytes));
-                for (int u = 0; u < 2; ++u)
-                    tma_load_3d(&maps.v, &sh.v_full[s], vs + s * 2 * KB_BYTES + u * v_kb_bytes, j * AKV + u * BK, 0,
-                                head);
+                    tma_load_3d(&maps.q, &sh.q_full, qs + kb * KB_BYTES, kb * BK, q0, head);
+                for (int j = 0; j < nkv && ok; ++j) {
+                    const int s = j & 1;
+                    const unsigned prev = ((base[s] + ((unsigned)j >> 1)) & 1u) ^ 1u;
+                    if (!mbar_wait(&sh.k_empty[s], prev, abort_flag, 31)) { ok = false; break; }
+                    mbar_expect_tx(&sh.k_full[s], (unsigned)(nkb * KB_BYTES));
+                    for (int kb = 0; kb < nkb; ++kb)
+                        tma_load_3d(&maps.k, &sh.k_full[s], ks + (s * 2 + kb) * KB_BYTES, kb * BK, j * AKV, head);
+                    if (!mbar_wait(&sh.v_empty[s], prev, abort_flag, 32)) { ok = false; break; }
+                    mbar_expect_tx(&sh.v_full[s], (unsigned)(2 * v_kb_bytes));
+                    for (int u = 0; u < 2; ++u)
+                        tma_load_3d(&maps.v, &sh.v_full[s], vs + s * 2 * KB_BYTES + u * v_kb_bytes, j * AKV + u * BK,
+                                    0, head);
+                }
+                base[0] += (unsigned)(nkv + 1) >> 1;
+                base[1] += (unsigned)nkv >> 1;
             }
             // every copy has to land before the CTA may exit: a slot's last release implies it
             for (int s = 0; s < 2 && ok; ++s) {
-                if (nkv <= s) continue;
-                const int last = ((nkv - 1 - s) >> 1) * 2 + s;         // last tile that used slot s
-                const unsigned ph = ((unsigned)last >> 1) & 1u;
+                if (base[s] == 0u) continue;
+                const unsigned ph = (base[s] - 1u) & 1u;
                 const unsigned long long t0 = global_ns();
                 while (!(mbar_try(&sh.k_empty[s], ph) && mbar_try(&sh.v_empty[s], ph)))
                     if (*abort_flag != 0 || global_ns() - t0 > WAIT_LIMIT_NS / 2) { *abort_flag = 33; break; }
@@ -269,47 +286,59 @@ k_attn_reps(const __grid_constant__ AttnMaps maps, int T, int d_h, int h,
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer
         if (lane == 0) {
-            bool ok = mbar_wait(&sh.q_full, 0u, abort_flag, 35);
+            bool ok = true;
+            unsigned base[2] = {0u, 0u};
             const unsigned idesc1 = instr_desc(AKV);
             const unsigned idesc2 = instr_desc(d_h);
-            // S[j & 1] = Q K_j^T
-            auto issue_s = [&](int j) {
-                const int b = j & 1;
-                const unsigned ph = ((unsigned)j >> 1) & 1u;
-                if (!mbar_wait(&sh.k_full[b], ph, abort_flag, 36)) { ok = false; return; }
-                if (!mbar_wait(&sh.s_empty[b], ph ^ 1u, abort_flag, 37)) { ok = false; return; }
-                tcgen05_fence_after();
-                for (int kb = 0; kb < nkb; ++kb) {
-                    const unsigned long long adesc = smem_desc_sw128(smem_u32(qs + kb * KB_BYTES));
-                    const unsigned long long bdesc = smem_desc_sw128(smem_u32(ks + (b * 2 + kb) * KB_BYTES));
-                    const int steps = min(BK, d_h - kb * BK) / UMMA_K;
-                    for (int k = 0; k < steps; ++k)
-                        umma_bf16(tmem_base + b * AKV, adesc + 2 * k, bdesc + 2 * k, idesc1, (kb | k) != 0);
+            int k = 0;
+            for (int item = blockIdx.x; item < total && ok; item += gridDim.x, ++k) {
+                const int qt = item % nq;
+                const int nkv = causal ? min(nkv_all, qt + 1) : nkv_all;
+                if (!mbar_wait(&sh.q_full, (unsigned)k & 1u, abort_flag, 35)) { ok = false; break; }
+                // S[j & 1] = Q K_j^T
+                auto issue_s = [&](int j) {
+                    const int b = j & 1;
+                    const unsigned ph = (base[b] + ((unsigned)j >> 1)) & 1u;
+                    if (!mbar_wait(&sh.k_full[b], ph, abort_flag, 36)) { ok = false; return; }
+                    if (!mbar_wait(&sh.s_empty[b], ph ^ 1u, abort_flag, 37)) { ok = false; return; }
+                    tcgen05_fence_after();
+                    for (int kb = 0; kb < nkb; ++kb) {
+                        const unsigned long long adesc = smem_desc_sw128(smem_u32(qs + kb * KB_BYTES));
+                        const unsigned long long bdesc = smem_desc_sw128(smem_u32(ks + (b * 2 + kb) * KB_BYTES));
+                        const int steps = min(BK, d_h - kb * BK) / UMMA_K;
+                        for (int q = 0; q < steps; ++q)
+                            umma_bf16(tmem_base + b * AKV, adesc + 2 * q, bdesc + 2 * q, idesc1, (kb | q) != 0);
+                    }
+                    umma_commit(&sh.k_empty[b]);
+                    umma_commit(&sh.s_full[b]);
+                    if (j == nkv - 1) umma_commit(&sh.q_empty);          // Q may be replaced
+                };
+                issue_s(0);
+                for (int j = 0; j < nkv && ok; ++j) {
+                    if (j + 1 < nkv) issue_s(j + 1);                     // each warp set one score tile ahead
+                    if (!ok) break;
+                    const int b = j & 1;
+                    const unsigned ph = (base[b] + ((unsigned)j >> 1)) & 1u;
+                    if (!mbar_wait(&sh.p_full[b], ph, abort_flag, 38)) { ok = false; break; }
+                    if (!mbar_wait(&sh.v_full[b], ph, abort_flag, 39)) { ok = false; break; }
+                    // the accumulators are overwritten: the previous item's rows have been read out
+                    if (j == 0 && k > 0 && !mbar_wait(&sh.o_empty, (unsigned)(k - 1) & 1u, abort_flag, 47)) { ok = false; break; }
+                    tcgen05_fence_after();
+                    for (int u = 0; u < 2; ++u) {                        // O[j & 1] += P_j V_j
+                        const unsigned long long adesc = smem_desc_sw128(smem_u32(ps + (b * 2 + u) * KB_BYTES));
+                        const unsigned long long bdesc = smem_desc_sw128(smem_u32(vs + b * 2 * KB_BYTES + u * v_kb_bytes));
+                        for (int q = 0; q < BK / UMMA_K; ++q)
+                            umma_bf16(tmem_base + (2 + b) * AKV, adesc + 2 * q, bdesc + 2 * q, idesc2,
+                                      ((j >> 1) | u | q) != 0);
+                    }
+                    umma_commit(&sh.v_empty[b]);
+                    umma_commit(&sh.p_empty[b]);
                 }
-                umma_commit(&sh.k_empty[b]);
-                umma_commit(&sh.s_full[b]);
-            };
-            if (ok) issue_s(0);
-            for (int j = 0; j < nkv && ok; ++j) {
-                if (j + 1 < nkv) issue_s(j + 1);                     // one score tile ahead of the softmax
-                if (!ok) break;
-                const int b = j & 1;
-                const unsigned ph = ((unsigned)j >> 1) & 1u;
-                if (!mbar_wait(&sh.p_full[b], ph, abort_flag, 38)) { ok = false; break; }
-                if (!mbar_wait(&sh.v_full[b], ph, abort_flag, 39)) { ok = false; break; }
-                tcgen05_fence_after();
-                for (int u = 0; u < 2; ++u) {                        // O[j & 1] += P_j V_j
-                    const unsigned long long adesc = smem_desc_sw128(smem_u32(ps + (b * 2 + u) * KB_BYTES));
-                    const unsigned long long bdesc = smem_desc_sw128(smem_u32(vs + b * 2 * KB_BYTES + u * v_kb_bytes));
-                    for (int k = 0; k < BK / UMMA_K; ++k)
-                        umma_bf16(tmem_base + (2 + b) * AKV, adesc + 2 * k, bdesc + 2 * k, idesc2,
-                                  ((j >> 1) | u | k) != 0);
-                }
-                umma_commit(&sh.v_empty[b]);
-                umma_commit(&sh.p_empty[b]);
+                if (ok) umma_commit(&sh.o_full);
+                base[0] += (unsigned)(nkv + 1) >> 1;
+                base[1] += (unsigned)nkv >> 1;
             }
-            if (ok) umma_commit(&sh.o_full);
-            else { /* the softmax warps time out on their own */ }
+            /* on failure the softmax warps time out on their own */
         }
     } else {
         // ------------------------------------------------ softmax and output (warps 2..9)
@@ -326,132 +355,143 @@ k_attn_reps(const __grid_constant__ AttnMaps maps, int T, int d_h, int h,
         const int quad = warp & 3;
         const int half = (warp - 2) >> 2;              // = parity of this set's key tiles = its buffers
         const int i = quad * 32 + lane;                // this thread's row of the tile
-        const int qrow = q0 + i;                       // position in the representative list
         const unsigned tlane = tmem_base + ((unsigned)(quad * 32) << 16);
         const unsigned t_s = tlane + half * AKV, t_o = tlane + (2 + half) * AKV;
         const float sc = 1.4426950408889634f / sqrtf((float)d_h);   // log2(e) / sqrt(d_h)
-        const int lim_abs = min(n, causal ? qrow + 1 : n);          // admissible keys of this row: [0, lim_abs)
-        float m_ref = -INFINITY, l = 0.f;
         bool ok = true;
-        for (int j = half; j < nkv && ok; j += 2) {
-            const unsigned ph = ((unsigned)j >> 1) & 1u;
-            bool got = mbar_wait(&sh.s_full[half], ph, abort_flag, 40);
-            if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
-            if (j == 0 && threadIdx.x == 64) ATRACE(2);
-            if (j == 2 && threadIdx.x == 64) ATRACE(20);
-            tcgen05_fence_after();
-            // columns past r, and under the causal mask the keys after the query, count as -inf
-            const int c0 = j * AKV;
-            const bool masked = (c0 + AKV > n) || (causal && c0 + AKV - 1 > q0);
-            // sweep 1: the row maximum of the raw scores
-            float cm = -INFINITY;
-#pragma unroll
-            for (int c = 0; c < AKV; c += 64) {
-                unsigned r0[32], r1[32];
-                tmem_ld32_issue(t_s + c, r0);
-                tmem_ld32_issue(t_s + c + 32, r1);
-                tmem_ld_wait(r0); tmem_ld_wait(r1);
-                if (masked) {
-                    cm = tile_max32<true>(r0, lim_abs - (c0 + c), cm);
-                    cm = tile_max32<true>(r1, lim_abs - (c0 + c + 32), cm);
-                } else {
-                    cm = tile_max32<false>(r0, 32, cm);
-                    cm = tile_max32<false>(r1, 32, cm);
-                }
-            }
-            cm *= sc;                                          // sc > 0: the maximum of the scaled scores
-            if (j == 2 && threadIdx.x == 64) ATRACE(21);
-            const float m_new = fmaxf(m_ref, cm);
-            const bool raise = m_new > m_ref + ATT_LAG;        // also true for the first finite maximum
-            // the MMAs of this set's previous tile have retired: its P buffer is free and nothing
-            // is adding to its accumulator
-            got = mbar_wait(&sh.p_empty[half], ph ^ 1u, abort_flag, 42);
-            if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
-            if (j < 2) {
-                m_ref = m_new;                                 // nothing accumulated yet
-            } else if (__any_sync(0xffffffffu, raise)) {
+        unsigned base = 0u;                            // uses of this set's buffers in earlier items
+        int k = 0;
+        for (int item = blockIdx.x; item < total && ok; item += gridDim.x, ++k) {
+            const int qt = item % nq, head = item / nq, q0 = qt * AQ;
+            const int nkv = causal ? min(nkv_all, qt + 1) : nkv_all;
+            const int qrow = q0 + i;                                    // position in the representative list
+            const int lim_abs = min(n, causal ? qrow + 1 : n);          // admissible keys of this row: [0, lim_abs)
+            float m_ref = -INFINITY, l = 0.f;
+            for (int j = half; j < nkv && ok; j += 2) {
+                const unsigned ph = (base + ((unsigned)j >> 1)) & 1u;
+                bool got = mbar_wait(&sh.s_full[half], ph, abort_flag, 40);
+                if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
+                if (k == 0 && j == 0 && threadIdx.x == 64) ATRACE(2);
+                if (k == 0 && j == 2 && threadIdx.x == 64) ATRACE(20);
                 tcgen05_fence_after();
-                const float f = raise ? ex2_approx(m_ref - m_new) : 1.0f;   // 0 for a row without a finite score so far
-                for (int o0 = 0; o0 < d_h; o0 += 32) {
-                    float v[32];
-                    tmem_ld32(t_o + o0, v);
+                // columns past r, and under the causal mask the keys after the query, count as -inf
+                const int c0 = j * AKV;
+                const bool masked = (c0 + AKV > n) || (causal && c0 + AKV - 1 > q0);
+                // sweep 1: the row maximum of the raw scores
+                float cm = -INFINITY;
 #pragma unroll
-                    for (int q = 0; q < 32; ++q) v[q] *= f;
-                    tmem_st32(t_o + o0, v);
+                for (int c = 0; c < AKV; c += 64) {
+                    unsigned r0[32], r1[32];
+                    tmem_ld32_issue(t_s + c, r0);
+                    tmem_ld32_issue(t_s + c + 32, r1);
+                    tmem_ld_wait(r0); tmem_ld_wait(r1);
+                    if (masked) {
+                        cm = tile_max32<true>(r0, lim_abs - (c0 + c), cm);
+                        cm = tile_max32<true>(r1, lim_abs - (c0 + c + 32), cm);
+                    } else {
+                        cm = tile_max32<false>(r0, 32, cm);
+                        cm = tile_max32<false>(r1, 32, cm);
+                    }
                 }
-                l *= f;
-                if (raise) m_ref = m_new;
-            }
-            if (j == 2 && threadIdx.x == 64) ATRACE(22);
-            // sweep 2: the probabilities
-            const float mref = m_ref > -INFINITY ? m_ref : 0.f;   // all scores -inf so far: every p is 0
-            unsigned char* prow = ps + half * 2 * KB_BYTES + i * 128;
-            float sum = 0.f;
+                cm *= sc;                                          // sc > 0: the maximum of the scaled scores
+                if (k == 0 && j == 2 && threadIdx.x == 64) ATRACE(21);
+                const float m_new = fmaxf(m_ref, cm);
+                const bool raise = m_new > m_ref + ATT_LAG;        // also true for the first finite maximum
+                // the MMAs of this set's previous tile have retired: its P buffer is free and nothing
+                // is adding to its accumulator
+                got = mbar_wait(&sh.p_empty[half], ph ^ 1u, abort_flag, 42);
+                if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
+                if (j < 2) {
+                    m_ref = m_new;                                 // nothing accumulated yet
+                } else if (__any_sync(0xffffffffu, raise)) {
+                    tcgen05_fence_after();
+                    const float f = raise ? ex2_approx(m_ref - m_new) : 1.0f;   // 0 for a row without a finite score so far
+                    for (int o0 = 0; o0 < d_h; o0 += 32) {
+                        float v[32];
+                        tmem_ld32(t_o + o0, v);
 #pragma unroll
-            for (int c = 0; c < AKV; c += 64) {
-                unsigned r0[32], r1[32];
-                tmem_ld32_issue(t_s + c, r0);
-                tmem_ld32_issue(t_s + c + 32, r1);
-                tmem_ld_wait(r0); tmem_ld_wait(r1);
-                if (masked) {
-                    tile_max32<true>(r0, lim_abs - (c0 + c), 0.f);
-                    tile_max32<true>(r1, lim_abs - (c0 + c + 32), 0.f);
+                        for (int q = 0; q < 32; ++q) v[q] *= f;
+                        tmem_st32(t_o + o0, v);
+                    }
+                    l *= f;
+                    if (raise) m_ref = m_new;
                 }
-                sum += exp_store(r0, sc, mref, prow + (c >> 6) * KB_BYTES, 0, i);
-                sum += exp_store(r1, sc, mref, prow + (c >> 6) * KB_BYTES, 4, i);
-            }
-            l += sum;
-            if (j == 2 && threadIdx.x == 64) ATRACE(23);
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the MMA reads P through the async proxy
-            tcgen05_fence_before();
-            __syncwarp();
-            if (lane == 0) { mbar_arrive(&sh.s_empty[half]); mbar_arrive(&sh.p_full[half]); }
-            if (threadIdx.x == 64) ATRACE(3 + min(j, 12));
-        }
-        // output rows of this tile's representatives, at their token positions
-        if (ok) {
-            bool got = mbar_wait(&sh.o_full, 0u, abort_flag, 43);
-            if (__all_sync(0xffffffffu, got)) {
-                if (threadIdx.x == 64) ATRACE(16);
-                tcgen05_fence_after();
-                // the two sets' statistics meet in the (now idle) P region
-                float2* xs = reinterpret_cast<float2*>(ps);
-                xs[half * AQ + i] = make_float2(m_ref, l);
+                if (k == 0 && j == 2 && threadIdx.x == 64) ATRACE(22);
+                // sweep 2: the probabilities
+                const float mref = m_ref > -INFINITY ? m_ref : 0.f;   // all scores -inf so far: every p is 0
+                unsigned char* prow = ps + half * 2 * KB_BYTES + i * 128;
+                float sum = 0.f;
+#pragma unroll
+                for (int c = 0; c < AKV; c += 64) {
+                    unsigned r0[32], r1[32];
+                    tmem_ld32_issue(t_s + c, r0);
+                    tmem_ld32_issue(t_s + c + 32, r1);
+                    tmem_ld_wait(r0); tmem_ld_wait(r1);
+                    if (masked) {
+                        tile_max32<true>(r0, lim_abs - (c0 + c), 0.f);
+                        tile_max32<true>(r1, lim_abs - (c0 + c + 32), 0.f);
+                    }
+                    sum += exp_store(r0, sc, mref, prow + (c >> 6) * KB_BYTES, 0, i);
+                    sum += exp_store(r1, sc, mref, prow + (c >> 6) * KB_BYTES, 4, i);
+                }
+                l += sum;
+                if (k == 0 && j == 2 && threadIdx.x == 64) ATRACE(23);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the MMA reads P through the async proxy
+                tcgen05_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&sh.x_put[quad]);
-                got = mbar_wait(&sh.x_put[quad], 0u, abort_flag, 45);
-                if (__all_sync(0xffffffffu, got)) {
-                    const float2 other = xs[(half ^ 1) * AQ + i];
-                    const float m = fmaxf(m_ref, other.x);
-                    const float f_own = m_ref > -INFINITY ? ex2_approx(m_ref - m) : 0.f;
-                    const float f_oth = other.x > -INFINITY ? ex2_approx(other.x - m) : 0.f;
-                    const float lt = l * f_own + other.y * f_oth;
-                    const float inv_l = lt > 0.f ? 1.0f / lt : 0.f;
-                    const float fa = (half == 0 ? f_own : f_oth) * inv_l;      // factor of the even tiles' accumulator
-                    const float fb = (half == 0 ? f_oth : f_own) * inv_l;
-                    const bool use_b = nkv > 1;                                  // was the odd accumulator ever written
-                    const int tok = qrow < n ? rep_idx[qrow] : -1;
-                    float* dst = (tok >= 0 && tok < T) ? out + (int64_t)tok * ldo + (int64_t)head * d_h : nullptr;
-                    for (int o0 = half * 32; o0 < d_h; o0 += 64) {
-                        float va[32], vb[32];
-                        tmem_ld32(tlane + 2 * AKV + o0, va);
-                        if (use_b) tmem_ld32(tlane + 3 * AKV + o0, vb);
-                        if (dst != nullptr) {
+                if (lane == 0) { mbar_arrive(&sh.s_empty[half]); mbar_arrive(&sh.p_full[half]); }
+                if (k == 0 && threadIdx.x == 64) ATRACE(3 + min(j, 12));
+            }
+            if (!ok) break;
+            base += (half == 0) ? (unsigned)(nkv + 1) >> 1 : (unsigned)nkv >> 1;
+            // output rows of this tile's representatives, at their token positions
+            bool got = mbar_wait(&sh.o_full, (unsigned)k & 1u, abort_flag, 43);
+            // (the statistics' slots are reused: everybody is done with the previous item's)
+            if (k > 0) got = got && mbar_wait(&sh.o_empty, (unsigned)(k - 1) & 1u, abort_flag, 48);
+            if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
+            if (k == 0 && threadIdx.x == 64) ATRACE(16);
+            tcgen05_fence_after();
+            sh.xstat[half][i] = make_float2(m_ref, l);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.x_put[quad]);
+            got = mbar_wait(&sh.x_put[quad], (unsigned)k & 1u, abort_flag, 45);
+            if (!__all_sync(0xffffffffu, got)) { ok = false; break; }
+            {
+                const float2 other = sh.xstat[half ^ 1][i];
+                const float m = fmaxf(m_ref, other.x);
+                const float f_own = m_ref > -INFINITY ? ex2_approx(m_ref - m) : 0.f;
+                const float f_oth = other.x > -INFINITY ? ex2_approx(other.x - m) : 0.f;
+                const float lt = l * f_own + other.y * f_oth;
+                const float inv_l = lt > 0.f ? 1.0f / lt : 0.f;
+                const float fa = (half == 0 ? f_own : f_oth) * inv_l;      // factor of the even tiles' accumulator
+                const float fb = (half == 0 ? f_oth : f_own) * inv_l;
+                const bool use_b = nkv > 1;                                  // was the odd accumulator written for this item
+                const int tok = qrow < n ? rep_idx[qrow] : -1;
+                float* dst = (tok >= 0 && tok < T) ? out + (int64_t)tok * ldo + (int64_t)head * d_h : nullptr;
+                for (int o0 = half * 32; o0 < d_h; o0 += 64) {
+                    float va[32], vb[32];
+                    tmem_ld32(tlane + 2 * AKV + o0, va);
+                    if (use_b) tmem_ld32(tlane + 3 * AKV + o0, vb);
+                    if (dst != nullptr) {
 #pragma unroll
-                            for (int q = 0; q < 32; q += 4) {
-                                if (o0 + q < d_h) {
-                                    float4 w = make_float4(va[q] * fa, va[q + 1] * fa, va[q + 2] * fa, va[q + 3] * fa);
-                                    if (use_b) {
-                                        w.x = fmaf(vb[q], fb, w.x); w.y = fmaf(vb[q + 1], fb, w.y);
-                                        w.z = fmaf(vb[q + 2], fb, w.z); w.w = fmaf(vb[q + 3], fb, w.w);
-                                    }
-                                    *reinterpret_cast<float4*>(dst + o0 + q) = w;
+                        for (int q = 0; q < 32; q += 4) {
+                            if (o0 + q < d_h) {
+                                float4 w = make_float4(va[q] * fa, va[q + 1] * fa, va[q + 2] * fa, va[q + 3] * fa);
+                                if (use_b) {
+                                    w.x = fmaf(vb[q], fb, w.x); w.y = fmaf(vb[q + 1], fb, w.y);
+                                    w.z = fmaf(vb[q + 2], fb, w.z); w.w = fmaf(vb[q + 3], fb, w.w);
                                 }
+                                *reinterpret_cast<float4*>(dst + o0 + q) = w;
                             }
                         }
                     }
                 }
             }
+            // the accumulators (and the statistics' slots) may be reused
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.o_empty);
+            if (k == 0 && threadIdx.x == 64) ATRACE(18);
         }
         tcgen05_fence_before();
     }
@@ -516,8 +556,10 @@ cudaError_t launch_attention_reps(ada_ctx* ctx, const void* Q, const void* K, co
     launch_k(ctx, k_attn_gather, dim3(Tp / 32, h), dim3(256), 0, s, (const __nv_bfloat16*)Q,
              (const __nv_bfloat16*)K, (const __nv_bfloat16*)V, T, Tp, h, d_h, ld, rep_idx, rep_cnt, Qr, Kr, Vt,
              ctx->status);
-    launch_k(ctx, k_attn_reps, dim3(Tp / AQ, h), dim3(ATT_THREADS), ATT_SMEM, s, maps, T, d_h, h, rep_idx, rep_cnt,
-             out, ldo, causal, ctx->status);
+    // persistent CTAs, at most one per SM; r (hence the number of work items) lives on the device
+    const int n_items_max = (Tp / AQ) * h;
+    launch_k(ctx, k_attn_reps, dim3(n_items_max < ctx->sm_count ? n_items_max : ctx->sm_count), dim3(ATT_THREADS),
+             ATT_SMEM, s, maps, T, d_h, h, rep_idx, rep_cnt, out, ldo, causal, ctx->status);
     if (nearest_idx != nullptr)
         launch_k(ctx, k_attn_expand, dim3((T + 7) / 8), dim3(256), 0, s, out, ldo, T, h * d_h, nearest_idx);
     return cudaGetLastError();
