@@ -88,7 +88,7 @@ def test_constant_values_pass_through(ada):
 
 
 def test_many_key_tiles_random(ada):
-    """r = 1400 of T = 2048: eleven key tiles per query tile, both softmax passes over all of them."""
+    """r = 1400 of T = 2048: eleven key tiles per query tile (six for one warp set, five for the other)."""
     rng = np.random.default_rng(5)
     T, h, d_h = 2048, 4, 128
     Q, K, V = (bf16_round(rng.standard_normal((T, h, d_h))) for _ in range(3))
@@ -96,6 +96,23 @@ def test_many_key_tiles_random(ada):
     R = sorted(rng.choice(T, 1400, replace=False).tolist())
     for causal in (False, True):
         run_case(ada, ctx, Q, K, V, R, None, causal)
+    ada.ada_destroy(ctx)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_more_work_items_than_sms(ada, causal):
+    """The CTAs are persistent: with 20 query tiles x 16 heads = 320 work items every CTA takes two
+    or three in a row, its rings, barriers and accumulators carried over (under the causal mask
+    with a different number of key tiles each time).  A second set with 7 query tiles leaves most
+    CTAs one item and some none."""
+    rng = np.random.default_rng(11 + causal)
+    T, h, d_h = 2560, 16, 32
+    Q, K, V = (bf16_round(rng.standard_normal((T, h, d_h))) for _ in range(3))
+    ctx = ada.ada_create(1, T, h * d_h, ada.ADA_BF16)
+    near = np.arange(T, dtype=np.int32)
+    run_case(ada, ctx, Q, K, V, list(range(T)), near, causal)
+    R = sorted(rng.choice(T, 800, replace=False).tolist())
+    run_case(ada, ctx, Q, K, V, R, None, causal)
     ada.ada_destroy(ctx)
 
 
