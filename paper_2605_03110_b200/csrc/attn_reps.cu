@@ -468,24 +468,41 @@ k_attn_reps(const __grid_constant__ AttnMaps maps, int T, int d_h, int h,
                 const bool use_b = nkv > 1;                                  // was the odd accumulator written for this item
                 const int tok = qrow < n ? rep_idx[qrow] : -1;
                 float* dst = (tok >= 0 && tok < T) ? out + (int64_t)tok * ldo + (int64_t)head * d_h : nullptr;
-                for (int o0 = half * 32; o0 < d_h; o0 += 64) {
+                // Rows leave through this set's own (now idle) P buffer: a thread owns a row, so its
+                // 32 columns go to shared memory (16-byte pieces permuted by row, free of bank
+                // conflicts both ways) and the warp then writes them out four rows at a time,
+                // 128 contiguous bytes per row, instead of 32 scattered 16-byte pieces per store.
+                unsigned char* stg = ps + half * 2 * KB_BYTES + quad * 8192;
+                const unsigned long long dst_bits = reinterpret_cast<unsigned long long>(dst);
+                int ci = 0;
+                for (int o0 = half * 32; o0 < d_h; o0 += 64, ++ci) {
                     float va[32], vb[32];
                     tmem_ld32(tlane + 2 * AKV + o0, va);
                     if (use_b) tmem_ld32(tlane + 3 * AKV + o0, vb);
-                    if (dst != nullptr) {
 #pragma unroll
-                        for (int q = 0; q < 32; q += 4) {
-                            if (o0 + q < d_h) {
-                                float4 w = make_float4(va[q] * fa, va[q + 1] * fa, va[q + 2] * fa, va[q + 3] * fa);
-                                if (use_b) {
-                                    w.x = fmaf(vb[q], fb, w.x); w.y = fmaf(vb[q + 1], fb, w.y);
-                                    w.z = fmaf(vb[q + 2], fb, w.z); w.w = fmaf(vb[q + 3], fb, w.w);
-                                }
-                                *reinterpret_cast<float4*>(dst + o0 + q) = w;
-                            }
+                    for (int q = 0; q < 32; q += 4) {
+                        float4 w = make_float4(va[q] * fa, va[q + 1] * fa, va[q + 2] * fa, va[q + 3] * fa);
+                        if (use_b) {
+                            w.x = fmaf(vb[q], fb, w.x); w.y = fmaf(vb[q + 1], fb, w.y);
+                            w.z = fmaf(vb[q + 2], fb, w.z); w.w = fmaf(vb[q + 3], fb, w.w);
                         }
+                        *reinterpret_cast<float4*>(stg + ci * 4096 + lane * 128 + ((((q >> 2) ^ lane) & 7) << 4)) = w;
                     }
                 }
+                __syncwarp();
+                ci = 0;
+                for (int o0 = half * 32; o0 < d_h; o0 += 64, ++ci) {
+#pragma unroll
+                    for (int it = 0; it < 8; ++it) {
+                        const int r = it * 4 + (lane >> 3), pc = lane & 7;
+                        const float4 w = *reinterpret_cast<const float4*>(stg + ci * 4096 + r * 128 + (((pc ^ r) & 7) << 4));
+                        const unsigned lo = __shfl_sync(0xffffffffu, (unsigned)dst_bits, r);
+                        const unsigned hi = __shfl_sync(0xffffffffu, (unsigned)(dst_bits >> 32), r);
+                        float* drow = reinterpret_cast<float*>(((unsigned long long)hi << 32) | lo);
+                        if (drow != nullptr && o0 + pc * 4 < d_h) *reinterpret_cast<float4*>(drow + o0 + pc * 4) = w;
+                    }
+                }
+                __syncwarp();
             }
             // the accumulators (and the statistics' slots) may be reused
             tcgen05_fence_before();
